@@ -1,0 +1,258 @@
+/*
+ * odma.h - C ABI of libodma: on-demand contiguous KV-cache allocation (ODMA) and the
+ * decode-attention path that streams the resulting slabs on NVIDIA B200 (sm_100a).
+ *
+ * The allocator follows the paper's design section (Section III): a request's KV cache
+ * lives in ONE contiguous slab whose size is the request's length bucket; bucket
+ * boundaries are re-derived from a sliding window of realised lengths (Section III-C,
+ * Eq. 2); a Large Bucket (safety pool) absorbs high-uncertainty requests and requests that
+ * outgrow their slab (Section III-D); reserve/release are the allocator's API (Section
+ * III-E).  The GPU kernels are the consumer the contiguous layout exists for (Section
+ * III-A: contiguous blocks so that attention streams at peak bandwidth).
+ *
+ * Conventions
+ *  - Every function returns an int32 status (ODMA_OK = 0); nothing throws.
+ *  - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *  - The pool's device memory belongs to the caller; the library never allocates or
+ *    frees it.  The library owns only small device scratch (split partials, staging for
+ *    odma_decode_step_host), allocated in odma_pool_create and freed in
+ *    odma_pool_destroy.
+ *  - Kernel launchers are asynchronous on the given stream (a cudaStream_t passed as
+ *    void*; NULL = the legacy default stream).  All device work of one pool must be
+ *    issued on one stream, or be ordered by the caller: a slab released on the host may
+ *    be handed out again while an earlier kernel still reads it otherwise.
+ *  - Host-side calls are not thread-safe; serialise calls on one pool.
+ *  - Lengths and capacities are in tokens.  One token occupies
+ *    layers * 2 * kv_heads * head_dim * elem_bytes bytes of the pool.
+ *
+ * Pool layout in device memory
+ *    The pool is layers*2 arrays (layer-major, K then V), each of T*kv_heads rows of
+ *    head_dim elements (T = pool capacity in tokens).  A slab {base, cap} owns rows
+ *    [base*kv_heads, (base+cap)*kv_heads) of every array, head-major inside the slab:
+ *        row(head, t) = base*kv_heads + head*cap + t,            0 <= t < cap
+ *    so the keys (or values) of one (request, layer, head) are one contiguous run of
+ *    len*head_dim*elem_bytes bytes.  Element address of array a = layer*2 + (0:K | 1:V):
+ *        dev_base + ((a*T*kv_heads + row) * head_dim + d) * elem_bytes
+ */
+#ifndef ODMA_H_
+#define ODMA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ODMA_MAX_BUCKETS 8
+
+enum {
+    ODMA_OK = 0,
+    ODMA_ERR_INVALID = 1,     /* bad argument, shape, alignment or configuration */
+    ODMA_ERR_NOMEM = 2,       /* no free run of the needed size (main or safety region) */
+    ODMA_ERR_UNKNOWN_REQ = 3, /* request id not live */
+    ODMA_ERR_DUP_REQ = 4,     /* request id already live */
+    ODMA_ERR_OVERFLOW = 5,    /* length beyond max_len, or beyond the slab on commit */
+    ODMA_ERR_CUDA = 6,        /* a CUDA runtime or driver call failed */
+    ODMA_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (status word) */
+};
+
+enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1 };
+
+/* kernels that odma_profile_read can report */
+enum { ODMA_K_APPEND = 0, ODMA_K_DECODE = 1, ODMA_K_COMBINE = 2, ODMA_K_MIGRATE = 3,
+       ODMA_K_PROBE = 4, ODMA_K_COUNT = 5 };
+
+typedef struct odma_pool odma_pool;   /* opaque */
+typedef struct odma_paged odma_paged; /* opaque: a page-16 copy of the pool (ablation) */
+
+/* Allocator and scratch configuration.  odma_config_default() fills the values the paper
+ * states (Section III-B: gamma = 0.2, tau = 0.8; Section III-C: 4 buckets, 10,000-request
+ * window, refresh every 1,000 requests) and this library's choices for what it leaves open. */
+typedef struct odma_config {
+    int32_t safety_pct;      /* share of the pool given to the Large Bucket, integer percent (10) */
+    int32_t max_len;         /* longest KV length of a request; multiple of granule (32768) */
+    int32_t granule;         /* G: slab bases and sizes are multiples of G tokens; must be 16 */
+    int32_t window;          /* W: realised lengths kept for the quantiles (10000) */
+    int32_t refresh;         /* R: boundaries re-derived every R completions (1000) */
+    int32_t n_levels;        /* B: number of quantile levels / adaptive buckets (4) */
+    int32_t p_num[ODMA_MAX_BUCKETS]; /* quantile levels p_i = p_num[i] / p_den ({1,2,3,4}/4) */
+    int32_t p_den;
+    int32_t gamma_permille;  /* gamma of L' = L(1 + gamma u), thousandths (200) */
+    int32_t tau_permille;    /* tau: u > tau routes to the Large Bucket, thousandths (800) */
+    int32_t growth;          /* migration asks for max(need, growth*len) tokens (2) */
+    int32_t large_fixed;     /* 1: every Large Bucket slab has max_len tokens (0) */
+    int32_t max_batch;       /* most requests per odma_build_tables call; sizes scratch (1024) */
+    int32_t max_group;       /* most query heads per KV head; sizes scratch (8) */
+    int32_t plan_ctas;       /* persistent CTAs the split plan targets; 0 = one per SM of the
+                                current device (148 when the pool has no device memory) */
+} odma_config;
+
+typedef struct odma_slab {
+    int32_t base_tok;  /* first token of the slab */
+    int32_t cap_tok;   /* tokens it can hold */
+    int32_t pool_id;   /* 0 main region, 1 Large Bucket */
+    int32_t bucket_id; /* index of the boundary it was sized by, -1 in the Large Bucket */
+    uint64_t epoch;    /* boundary epoch in force when the call returned */
+} odma_slab;
+
+typedef struct odma_stats {
+    int64_t total_tokens, safety_tokens, main_tokens; /* T, S, M */
+    int64_t live, reserved_live, used_live;           /* live requests, sum cap, sum len */
+    int64_t completed, sum_len_completed, sum_cap_completed; /* utilisation = len / cap */
+    int64_t migrations, nomem, routed_large;
+    int64_t safety_live, safety_peak;                 /* tokens held in the Large Bucket */
+    int64_t observed;                                 /* lengths logged so far */
+    uint64_t epoch;
+} odma_stats;
+
+/* Host-side description of one built batch (plain data, owned by the caller).  The device
+ * table it points to holds int32 words:
+ *   base[n], cap[n], len[n] (length AFTER this step's append), cu_new[n+1] (prefix sum of
+ *   the tokens appended this step), cta_begin[n_ctas+1], items[n_items][8], combine[n_combine][4].
+ *   item    = {request, kv_head, first_token, n_tokens, direct(1)|partial(0), slot, 0, 0}
+ *   combine = {request, kv_head, first_slot, n_slots}
+ * The off_* fields are word offsets of those arrays inside d_table. */
+typedef struct odma_tables {
+    void* d_table;
+    int32_t n, n_new_total, n_items, n_ctas, n_combine, words;
+    int32_t off_base, off_cap, off_len, off_cu_new, off_cta_begin, off_items, off_combine;
+    int32_t tile_tokens;
+    int64_t kv_tokens; /* sum of len */
+    uint64_t epoch;
+} odma_tables;
+
+void odma_config_default(odma_config* cfg);
+const char* odma_strerror(int32_t code);
+
+/* ---- pool (problem statement: one KV-cache pool carved into contiguous per-request slabs;
+ *      Section I-C, Section III-A) --------------------------------------------------------
+ * dev_base: device pointer to `bytes` bytes, 256-byte aligned, or NULL for a bookkeeping-only
+ * pool (allocator calls work, every device call returns ODMA_ERR_INVALID).  T =
+ * floor_G(bytes / token_bytes) tokens, the last floor_G(T*safety_pct/100) of them are the
+ * Large Bucket.  head_dim*elem_bytes must be a multiple of 16.  cfg NULL = defaults.
+ * Until odma_set_buckets or the first recalibration there is one bucket of max_len tokens.
+ * With device memory the call allocates the library's scratch (cudaMalloc) and must run
+ * with the pool's device current. */
+int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t kv_heads,
+                         int32_t head_dim, int32_t dtype, const odma_config* cfg, odma_pool** out);
+int32_t odma_pool_destroy(odma_pool* pool);
+
+/* ---- bucket boundaries (Section III-C, Eq. 2) ------------------------------------------
+ * Static / initial boundaries: n in [1, ODMA_MAX_BUCKETS], strictly increasing multiples of
+ * the granule, none above max_len.  They hold until the next recalibration. */
+int32_t odma_set_buckets(odma_pool* pool, const int32_t* boundaries, int32_t n);
+/* boundaries: host array of ODMA_MAX_BUCKETS entries; *n and *epoch receive count and epoch. */
+int32_t odma_get_buckets(const odma_pool* pool, int32_t* boundaries, int32_t* n, uint64_t* epoch);
+
+/* ---- reserve (Section III-E; bucket choice Section III-C; tail Section III-D) -----------
+ * predicted_len is the predicted TOTAL length (prompt + generation).  The slab has the size
+ * of the first boundary >= predicted_len and sits at the lowest free address of the main
+ * region; a length beyond the last boundary is served from the Large Bucket with
+ * ceil_G(predicted_len) tokens.  ODMA_ERR_NOMEM when nothing fits (ordinary requests never
+ * spill into the Large Bucket), ODMA_ERR_DUP_REQ for a live id. */
+int32_t odma_alloc(odma_pool* pool, uint64_t req, int32_t predicted_len, odma_slab* out);
+/* Section III-B: inflate L' = ceil(L_hat * (1 + gamma*u)) and, when u > tau, take the slab
+ * straight from the Large Bucket.  u_permille in [0, 1000]. */
+int32_t odma_alloc_uncertain(odma_pool* pool, uint64_t req, int32_t l_hat, int32_t u_permille,
+                             odma_slab* out);
+/* Sections III-D and IV-C, reactive migration: if needed_len exceeds the slab, reserve a
+ * Large Bucket slab of max(needed_len, growth*len) tokens (capped at max_len), launch the
+ * copy of the request's len tokens (all layers, K and V) on `stream`, then release the old
+ * slab.  *migrated = 1 when that happened.  ODMA_ERR_OVERFLOW beyond max_len;
+ * ODMA_ERR_NOMEM leaves the old slab in place. */
+int32_t odma_ensure_capacity(odma_pool* pool, uint64_t req, int32_t needed_len, void* stream,
+                             odma_slab* out, int32_t* migrated);
+/* release (Section III-E) and logging of the realised length (Section III-A): frees the
+ * slab, pushes the request's length into the window and, on every R-th completion,
+ * re-derives the boundaries.  New boundaries apply to later odma_alloc calls only
+ * (Section IV-C). */
+int32_t odma_free(odma_pool* pool, uint64_t req);
+
+/* Host mirror of the lengths: after a step's kernels have been issued, add n_new[i] (NULL =
+ * 1 each) tokens to each request's length.  ODMA_ERR_OVERFLOW if one would pass its slab
+ * (nothing is changed then). */
+int32_t odma_commit_step(odma_pool* pool, const uint64_t* reqs, int32_t n, const int32_t* n_new);
+int32_t odma_get_slab(const odma_pool* pool, uint64_t req, odma_slab* out, int32_t* len);
+int32_t odma_get_stats(const odma_pool* pool, odma_stats* out);
+
+/* ---- per-step tables -------------------------------------------------------------------
+ * Slab table, lengths and the split plan for a batch of n live requests, each about to
+ * append n_new[i] tokens (NULL = 1 each; 0 allowed).  Every request must already have room
+ * (odma_ensure_capacity).  The plan cuts the batch's KV streams (one per request and KV
+ * head) into equal shares of 64-token tiles, one share per persistent CTA.
+ * odma_plan_host writes the table to host memory (no CUDA call); odma_build_tables writes
+ * it to the caller's device buffer d_table with one asynchronous copy.  table_bytes must be
+ * at least odma_tables_bytes(pool, n). */
+uint64_t odma_tables_bytes(const odma_pool* pool, int32_t n);
+int32_t odma_plan_host(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                       int32_t* host_table, uint64_t table_bytes, odma_tables* out);
+int32_t odma_build_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                          void* d_table, uint64_t table_bytes, void* stream, odma_tables* out);
+
+/* ---- KV append (the per-step growth of each request's cache, Section II-A) --------------
+ * Writes the step's new K and V rows of `layer` behind each request's existing tokens:
+ * token j of request i goes to slab position len[i] - n_new[i] + j.  k_new, v_new: device,
+ * [n_new_total, kv_heads, head_dim] in the pool dtype, requests in table order, 16-byte
+ * aligned. */
+int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables,
+                       const void* k_new, const void* v_new, void* stream);
+
+/* ---- decode attention over the slabs (the bandwidth consumer, Sections III-A and V-B) ---
+ * out[i][h] = softmax_j(q[i][h] . K_i[h div g][j] / sqrt(head_dim)) V_i[h div g], j < len[i],
+ * g = q_heads / kv_heads.  q, out: device, [n, q_heads, head_dim] in the pool dtype, 16-byte
+ * aligned; lse: device fp32 [n, q_heads] or NULL (natural-log sum of exp of the scaled
+ * scores).  Accumulation and softmax are fp32.  Launches the split kernel and, when some
+ * stream was split, the combine kernel. */
+int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                              const odma_tables* tables, void* out, float* lse, void* stream);
+
+/* One decode step of one layer from HOST buffers: builds the tables for reqs (one new token
+ * each), copies h_q [n,q_heads,head_dim], h_k_new, h_v_new [n,kv_heads,head_dim] to the
+ * device, appends, attends and copies the result to h_out [n,q_heads,head_dim]; all
+ * asynchronous on `stream` (pinned host memory recommended).  Does not commit lengths. */
+int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
+                              int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
+                              void* h_out, void* stream);
+
+/* Synchronises `stream` and returns the device status word as an error code (ODMA_OK,
+ * ODMA_ERR_TIMEOUT, or ODMA_ERR_CUDA for a failed stream), clearing it. */
+int32_t odma_check_status(odma_pool* pool, void* stream);
+
+/* Failure detection, exercised without a fault: launches a one-thread kernel whose only wait
+ * can never be satisfied and gives up after limit_ms (1..1000); odma_check_status then returns
+ * ODMA_ERR_TIMEOUT and the context stays usable.  Every wait of the decode kernels is bounded
+ * the same way. */
+int32_t odma_selftest_timeout(odma_pool* pool, int32_t limit_ms, void* stream);
+
+/* ---- measurement aids -------------------------------------------------------------------
+ * Streams exactly the bytes odma_decode_attention would read for `layer`, through the same
+ * staging pipeline, and does no arithmetic: the ceiling for this access pattern. */
+int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const odma_tables* tables,
+                        void* stream);
+/* Per-kernel device time: while enabled every launch is bracketed by CUDA events on its
+ * stream.  odma_profile_read synchronises and returns the summed milliseconds and the
+ * number of launches of one kernel since profiling was enabled. */
+int32_t odma_profile_enable(odma_pool* pool, int32_t on);
+int32_t odma_profile_read(odma_pool* pool, int32_t kernel, double* total_ms, int64_t* launches);
+
+/* ---- page-16 ablation (paging is the layout the paper argues against, Sections I, II-A) --
+ * The same requests re-laid in 16-token pages: page p of (array a, head) is 16 rows at
+ * ((a*n_pages + p)*kv_heads + head)*16 of the caller's buffer d_pages.  odma_paged_build
+ * assigns ceil(len/16) pages to each request of `tables` (consecutive ids when shuffle_seed
+ * is 0, a seeded permutation of all pages otherwise), writes the page table
+ * [n][max_pages] to d_page_table and copies the slab contents of every layer into the
+ * pages.  odma_decode_attention_paged is odma_decode_attention reading through it. */
+int32_t odma_paged_create(odma_pool* pool, void* d_pages, uint64_t bytes, odma_paged** out);
+int32_t odma_paged_destroy(odma_paged* paged);
+int32_t odma_paged_build(odma_paged* paged, const odma_tables* tables, const int32_t* host_len,
+                         uint64_t shuffle_seed, int32_t* d_page_table, int32_t max_pages,
+                         void* stream);
+int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void* q,
+                                    int32_t q_heads, const odma_tables* tables,
+                                    const int32_t* d_page_table, int32_t max_pages, void* out,
+                                    float* lse, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ODMA_H_ */

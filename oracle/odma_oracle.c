@@ -450,6 +450,8 @@ int ora_ensure(ora_alloc* a, uint64_t id, int64_t need, int64_t* out5, int32_t* 
     }
     int32_t who = (int32_t)(r - a->reqs);
     mark(a, base, cap, who);        /* allocate ... */
+    int64_t u = safety_in_use(a);   /* peak occupancy counts the moment both slabs are held */
+    if (u > a->safety_peak) a->safety_peak = u;
     mark(a, r->base, r->cap, -1);   /* ... (copy) ... then release the old slab */
     r->base = base;
     r->cap = cap;
@@ -457,8 +459,6 @@ int ora_ensure(ora_alloc* a, uint64_t id, int64_t need, int64_t* out5, int32_t* 
     r->bucket = -1;
     r->migrations += 1;
     a->migrations += 1;
-    int64_t u = safety_in_use(a);
-    if (u > a->safety_peak) a->safety_peak = u;
     *migrated = 1;
     fill_slab(r, a->epoch, out5);
     return ORA_OK;

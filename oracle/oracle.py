@@ -279,6 +279,8 @@ class Allocator:
 
     def ensure(self, req, need):
         rc, slab, mig = self.ensure_capacity(req, need)
+        if rc == ERR_NOMEM:
+            return None
         if rc != OK:
             raise RuntimeError(f"oracle ensure_capacity({req},{need}) -> {rc}")
         return slab[:4], mig

@@ -1,0 +1,726 @@
+// C ABI of libodma (include/odma.h): argument checks, host bookkeeping, kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "allocator.hpp"
+#include "kernels.hpp"
+#include "odma.h"
+#include "planner.hpp"
+
+using namespace odma;
+
+namespace {
+
+constexpr int kStagingSlots = 4;
+constexpr int64_t kDefaultWaitLimitNs = 2000000000ll;   // 2 s: far above any kernel here
+
+struct ProfRecord {
+    int kernel;
+    cudaEvent_t start, stop;
+};
+
+struct Staging {
+    int32_t* host = nullptr;     // pinned
+    cudaEvent_t done = nullptr;  // recorded after the copy that read `host`
+    bool in_flight = false;
+};
+
+}  // namespace
+
+struct odma_pool {
+    Allocator alloc;
+    void* dev_base = nullptr;
+    uint64_t bytes = 0;
+    int32_t layers = 0, kv_heads = 0, head_dim = 0, dtype = 0, elem_bytes = 0;
+    int64_t rows_per_array = 0;
+    int32_t plan_ctas = 148;
+    int64_t slots_max = 0;
+    int64_t table_words_max = 0;
+    bool has_maps = false;
+    TensorMaps maps{};
+    float* part_o = nullptr;
+    float* part_ml = nullptr;
+    uint32_t* d_status = nullptr;
+    Staging staging[kStagingSlots];
+    int staging_next = 0;
+    // device staging of odma_decode_step_host
+    void* d_q = nullptr;
+    void* d_k_new = nullptr;
+    void* d_v_new = nullptr;
+    void* d_out = nullptr;
+    int32_t* d_step_table = nullptr;
+    // profiling
+    bool profiling = false;
+    std::vector<ProfRecord> prof;
+    // reusable host vectors
+    std::vector<int32_t> v_base, v_cap, v_len;
+};
+
+struct odma_paged {
+    odma_pool* pool = nullptr;
+    void* d_pages = nullptr;
+    int64_t n_pages = 0;
+    TensorMaps maps{};
+    bool has_maps = false;
+    int32_t* pinned = nullptr;
+    int64_t pinned_words = 0;
+};
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// Two views of a [rows x head_dim] bf16 row array: 64-row and 16-row boxes of 64 elements
+// (128 bytes, the widest inner extent the 128-byte swizzle allows).
+int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, TensorMaps* out) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || !fn)
+        return ODMA_ERR_CUDA;
+    auto encode = reinterpret_cast<EncodeTiledFn>(fn);
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(head_dim) * 2};
+    const cuuint32_t estride[2] = {1, 1};
+    const cuuint32_t box_big[2] = {64, 64}, box_small[2] = {64, 16};
+    if (encode(&out->big, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box_big, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return ODMA_ERR_CUDA;
+    if (encode(&out->small, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box_small, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return ODMA_ERR_CUDA;
+    return ODMA_OK;
+}
+
+struct ProfScope {
+    odma_pool* pool;
+    cudaStream_t stream;
+    cudaEvent_t stop = nullptr;
+    ProfScope(odma_pool* p, int kernel, cudaStream_t s) : pool(p), stream(s) {
+        if (!p->profiling) return;
+        ProfRecord r{kernel, nullptr, nullptr};
+        if (cudaEventCreate(&r.start) != cudaSuccess || cudaEventCreate(&r.stop) != cudaSuccess) return;
+        cudaEventRecord(r.start, s);
+        stop = r.stop;
+        p->prof.push_back(r);
+    }
+    ~ProfScope() {
+        if (stop) cudaEventRecord(stop, stream);
+    }
+};
+
+void clear_profile(odma_pool* p) {
+    for (auto& r : p->prof) {
+        cudaEventDestroy(r.start);
+        cudaEventDestroy(r.stop);
+    }
+    p->prof.clear();
+}
+
+void free_device_side(odma_pool* p) {
+    clear_profile(p);
+    cudaFree(p->part_o);
+    cudaFree(p->part_ml);
+    cudaFree(p->d_status);
+    cudaFree(p->d_q);
+    cudaFree(p->d_k_new);
+    cudaFree(p->d_v_new);
+    cudaFree(p->d_out);
+    cudaFree(p->d_step_table);
+    for (auto& s : p->staging) {
+        if (s.host) cudaFreeHost(s.host);
+        if (s.done) cudaEventDestroy(s.done);
+        s = Staging{};
+    }
+}
+
+// Gather slab, capacity and post-append length of every request of the batch.
+int32_t gather_batch(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n) {
+    pool->v_base.resize(n);
+    pool->v_cap.resize(n);
+    pool->v_len.resize(n);
+    for (int32_t i = 0; i < n; ++i) {
+        const Request* r = pool->alloc.find(reqs[i]);
+        if (!r) return ODMA_ERR_UNKNOWN_REQ;
+        const int64_t add = n_new ? n_new[i] : 1;
+        if (add < 0) return ODMA_ERR_INVALID;
+        if (r->len + add > r->cap) return ODMA_ERR_OVERFLOW;
+        if (r->len + add < 1) return ODMA_ERR_INVALID;
+        pool->v_base[i] = static_cast<int32_t>(r->base);
+        pool->v_cap[i] = static_cast<int32_t>(r->cap);
+        pool->v_len[i] = static_cast<int32_t>(r->len + add);
+    }
+    return ODMA_OK;
+}
+
+int32_t plan_into(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                  int32_t* host_table, uint64_t table_bytes, odma_tables* out) {
+    if (!pool || !reqs || !host_table || !out || n < 1) return ODMA_ERR_INVALID;
+    if (n > pool->alloc.config().max_batch) return ODMA_ERR_INVALID;
+    int32_t rc = gather_batch(pool, reqs, n_new, n);
+    if (rc != ODMA_OK) return rc;
+    PlanInput in;
+    in.n = n;
+    in.kv_heads = pool->kv_heads;
+    in.n_ctas = pool->plan_ctas;
+    in.base = pool->v_base.data();
+    in.cap = pool->v_cap.data();
+    in.len = pool->v_len.data();
+    in.n_new = n_new;
+    rc = plan_batch(in, host_table, static_cast<int64_t>(table_bytes / 4), out);
+    if (rc != ODMA_OK) return rc;
+    out->epoch = pool->alloc.epoch();
+    return ODMA_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int32_t check_tables(const odma_pool* pool, const odma_tables* t) {
+    if (!t || !t->d_table || t->n < 1 || t->n_items < 1 || t->n_ctas < 1) return ODMA_ERR_INVALID;
+    if (t->n_items > pool->slots_max) return ODMA_ERR_INVALID;
+    return ODMA_OK;
+}
+
+void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                        const odma_tables* t, void* out, float* lse, DecodeParams* p) {
+    const int32_t* tab = static_cast<const int32_t*>(t->d_table);
+    p->base = tab + t->off_base;
+    p->cap = tab + t->off_cap;
+    p->len = tab + t->off_len;
+    p->cta_begin = tab + t->off_cta_begin;
+    p->items = reinterpret_cast<const int4*>(tab + t->off_items);
+    p->q = q;
+    p->out = out;
+    p->lse = lse;
+    p->part_o = pool->part_o;
+    p->part_ml = pool->part_ml;
+    p->pool = pool->dev_base;
+    p->rows_per_array = pool->rows_per_array;
+    p->layer = layer;
+    p->q_heads = q_heads;
+    p->kv_heads = pool->kv_heads;
+    p->group = q_heads / pool->kv_heads;
+    p->head_dim = pool->head_dim;
+    p->scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(pool->head_dim)));
+    p->status = pool->d_status;
+    p->page_table = nullptr;
+    p->max_pages = 0;
+    p->wait_limit_ns = kDefaultWaitLimitNs;
+}
+
+int32_t check_decode_args(const odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                          const odma_tables* t, const void* out) {
+    if (!pool || !pool->dev_base) return ODMA_ERR_INVALID;
+    if (layer < 0 || layer >= pool->layers || !q || !out || !aligned16(q) || !aligned16(out))
+        return ODMA_ERR_INVALID;
+    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
+    if (q_heads / pool->kv_heads > pool->alloc.config().max_group) return ODMA_ERR_INVALID;
+    return check_tables(pool, t);
+}
+
+}  // namespace
+
+extern "C" {
+
+void odma_config_default(odma_config* cfg) {
+    if (!cfg) return;
+    std::memset(cfg, 0, sizeof *cfg);
+    cfg->safety_pct = 10;
+    cfg->max_len = 32768;
+    cfg->granule = 16;
+    cfg->window = 10000;
+    cfg->refresh = 1000;
+    cfg->n_levels = 4;
+    for (int i = 0; i < 4; ++i) cfg->p_num[i] = i + 1;
+    cfg->p_den = 4;
+    cfg->gamma_permille = 200;
+    cfg->tau_permille = 800;
+    cfg->growth = 2;
+    cfg->large_fixed = 0;
+    cfg->max_batch = 1024;
+    cfg->max_group = 8;
+    cfg->plan_ctas = 0;
+}
+
+const char* odma_strerror(int32_t code) {
+    switch (code) {
+        case ODMA_OK: return "ok";
+        case ODMA_ERR_INVALID: return "invalid argument";
+        case ODMA_ERR_NOMEM: return "no free run of the needed size";
+        case ODMA_ERR_UNKNOWN_REQ: return "unknown request";
+        case ODMA_ERR_DUP_REQ: return "request already live";
+        case ODMA_ERR_OVERFLOW: return "length beyond capacity";
+        case ODMA_ERR_CUDA: return "CUDA call failed";
+        case ODMA_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t kv_heads,
+                         int32_t head_dim, int32_t dtype, const odma_config* cfg_in, odma_pool** out) {
+    if (!out) return ODMA_ERR_INVALID;
+    *out = nullptr;
+    if (dtype != ODMA_DTYPE_F32 && dtype != ODMA_DTYPE_BF16) return ODMA_ERR_INVALID;
+    odma_config cfg;
+    if (cfg_in) cfg = *cfg_in; else odma_config_default(&cfg);
+    const int32_t esz = dtype == ODMA_DTYPE_F32 ? 4 : 2;
+    if (layers < 1 || kv_heads < 1 || head_dim < 1 || (static_cast<int64_t>(head_dim) * esz) % 16 != 0)
+        return ODMA_ERR_INVALID;
+    if (cfg.max_batch < 1 || cfg.max_group < 1 || cfg.plan_ctas < 0) return ODMA_ERR_INVALID;
+    if (dev_base && (reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0) return ODMA_ERR_INVALID;
+
+    odma_pool* p = new (std::nothrow) odma_pool();
+    if (!p) return ODMA_ERR_NOMEM;
+    int32_t rc = p->alloc.init(bytes, layers, kv_heads, head_dim, esz, cfg);
+    if (rc != ODMA_OK) {
+        delete p;
+        return rc;
+    }
+    p->dev_base = dev_base;
+    p->bytes = bytes;
+    p->layers = layers;
+    p->kv_heads = kv_heads;
+    p->head_dim = head_dim;
+    p->dtype = dtype;
+    p->elem_bytes = esz;
+    p->rows_per_array = p->alloc.T() * kv_heads;
+    if (p->rows_per_array * layers * 2 >= (int64_t(1) << 31)) {
+        delete p;
+        return ODMA_ERR_INVALID;
+    }
+    p->plan_ctas = cfg.plan_ctas > 0 ? cfg.plan_ctas : 148;
+    if (dev_base) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            delete p;
+            return ODMA_ERR_CUDA;
+        }
+        if (cfg.plan_ctas == 0) p->plan_ctas = sms;
+    }
+    p->slots_max = static_cast<int64_t>(cfg.max_batch) * kv_heads + p->plan_ctas;
+    p->table_words_max = plan_table_words(cfg.max_batch, kv_heads, p->plan_ctas);
+    if (dev_base) {
+        const size_t po = static_cast<size_t>(p->slots_max) * cfg.max_group * head_dim * 4;
+        const size_t pm = static_cast<size_t>(p->slots_max) * cfg.max_group * 2 * 4;
+        const size_t qb = static_cast<size_t>(cfg.max_batch) * kv_heads * cfg.max_group * head_dim * esz;
+        const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * esz;
+        bool ok = cudaMalloc(&p->part_o, po) == cudaSuccess && cudaMalloc(&p->part_ml, pm) == cudaSuccess &&
+                  cudaMalloc(&p->d_status, 4) == cudaSuccess && cudaMalloc(&p->d_q, qb) == cudaSuccess &&
+                  cudaMalloc(&p->d_out, qb) == cudaSuccess && cudaMalloc(&p->d_k_new, kb) == cudaSuccess &&
+                  cudaMalloc(&p->d_v_new, kb) == cudaSuccess &&
+                  cudaMalloc(&p->d_step_table, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
+                  cudaMemset(p->d_status, 0, 4) == cudaSuccess;
+        for (auto& s : p->staging) {
+            ok = ok && cudaMallocHost(&s.host, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) == cudaSuccess;
+        }
+        if (ok && dtype == ODMA_DTYPE_BF16 && tc_supported(head_dim, 1)) {
+            ok = make_tensor_maps(dev_base, p->rows_per_array * layers * 2, head_dim, &p->maps) == ODMA_OK;
+            p->has_maps = ok;
+        }
+        if (!ok) {
+            free_device_side(p);
+            delete p;
+            return ODMA_ERR_CUDA;
+        }
+    }
+    *out = p;
+    return ODMA_OK;
+}
+
+int32_t odma_pool_destroy(odma_pool* pool) {
+    if (!pool) return ODMA_ERR_INVALID;
+    if (pool->dev_base) free_device_side(pool);
+    delete pool;
+    return ODMA_OK;
+}
+
+int32_t odma_set_buckets(odma_pool* pool, const int32_t* boundaries, int32_t n) {
+    return pool ? pool->alloc.set_buckets(boundaries, n) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_get_buckets(const odma_pool* pool, int32_t* boundaries, int32_t* n, uint64_t* epoch) {
+    return pool ? pool->alloc.get_buckets(boundaries, n, epoch) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_alloc(odma_pool* pool, uint64_t req, int32_t predicted_len, odma_slab* out) {
+    return pool ? pool->alloc.reserve(req, predicted_len, out) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_alloc_uncertain(odma_pool* pool, uint64_t req, int32_t l_hat, int32_t u_permille,
+                             odma_slab* out) {
+    return pool ? pool->alloc.reserve_uncertain(req, l_hat, u_permille, out) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_ensure_capacity(odma_pool* pool, uint64_t req, int32_t needed_len, void* stream,
+                             odma_slab* out, int32_t* migrated) {
+    if (!pool) return ODMA_ERR_INVALID;
+    Migration mig{};
+    int32_t did = 0;
+    int32_t rc = pool->alloc.ensure(req, needed_len, out, &did, &mig);
+    if (migrated) *migrated = did;
+    if (rc != ODMA_OK || !did || !pool->dev_base || mig.len == 0) return rc;
+    MigrateParams mp;
+    mp.pool = pool->dev_base;
+    mp.rows_per_array = pool->rows_per_array;
+    mp.src_base = mig.src_base;
+    mp.src_cap = mig.src_cap;
+    mp.dst_base = mig.dst_base;
+    mp.dst_cap = mig.dst_cap;
+    mp.len = mig.len;
+    mp.arrays = pool->layers * 2;
+    mp.kv_heads = pool->kv_heads;
+    mp.row_vecs = pool->head_dim * pool->elem_bytes / 16;
+    ProfScope ps(pool, ODMA_K_MIGRATE, as_stream(stream));
+    return launch_migrate(mp, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
+}
+
+int32_t odma_free(odma_pool* pool, uint64_t req) {
+    return pool ? pool->alloc.release(req) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_commit_step(odma_pool* pool, const uint64_t* reqs, int32_t n, const int32_t* n_new) {
+    return pool ? pool->alloc.commit(reqs, n, n_new) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_get_slab(const odma_pool* pool, uint64_t req, odma_slab* out, int32_t* len) {
+    if (!pool) return ODMA_ERR_INVALID;
+    const Request* r = pool->alloc.find(req);
+    if (!r) return ODMA_ERR_UNKNOWN_REQ;
+    if (out) {
+        out->base_tok = static_cast<int32_t>(r->base);
+        out->cap_tok = static_cast<int32_t>(r->cap);
+        out->pool_id = r->pool;
+        out->bucket_id = r->bucket;
+        out->epoch = pool->alloc.epoch();
+    }
+    if (len) *len = static_cast<int32_t>(r->len);
+    return ODMA_OK;
+}
+
+int32_t odma_get_stats(const odma_pool* pool, odma_stats* out) {
+    if (!pool || !out) return ODMA_ERR_INVALID;
+    pool->alloc.stats(out);
+    return ODMA_OK;
+}
+
+uint64_t odma_tables_bytes(const odma_pool* pool, int32_t n) {
+    if (!pool || n < 1) return 0;
+    return static_cast<uint64_t>(plan_table_words(n, pool->kv_heads, pool->plan_ctas)) * 4u;
+}
+
+int32_t odma_plan_host(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                       int32_t* host_table, uint64_t table_bytes, odma_tables* out) {
+    return plan_into(pool, reqs, n_new, n, host_table, table_bytes, out);
+}
+
+int32_t odma_build_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                          void* d_table, uint64_t table_bytes, void* stream, odma_tables* out) {
+    if (!pool || !pool->dev_base || !d_table || !aligned16(d_table)) return ODMA_ERR_INVALID;
+    if (n < 1 || table_bytes < odma_tables_bytes(pool, n)) return ODMA_ERR_INVALID;
+    Staging& st = pool->staging[pool->staging_next];
+    pool->staging_next = (pool->staging_next + 1) % kStagingSlots;
+    if (st.in_flight && cudaEventSynchronize(st.done) != cudaSuccess) return ODMA_ERR_CUDA;
+    st.in_flight = false;
+    int32_t rc = plan_into(pool, reqs, n_new, n, st.host, static_cast<uint64_t>(pool->table_words_max) * 4, out);
+    if (rc != ODMA_OK) return rc;
+    if (cudaMemcpyAsync(d_table, st.host, static_cast<size_t>(out->words) * 4, cudaMemcpyHostToDevice,
+                        as_stream(stream)) != cudaSuccess ||
+        cudaEventRecord(st.done, as_stream(stream)) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    st.in_flight = true;
+    out->d_table = d_table;
+    return ODMA_OK;
+}
+
+int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables, const void* k_new,
+                       const void* v_new, void* stream) {
+    if (!pool || !pool->dev_base || layer < 0 || layer >= pool->layers) return ODMA_ERR_INVALID;
+    if (!tables || !tables->d_table || tables->n < 1) return ODMA_ERR_INVALID;
+    if (tables->n_new_total == 0) return ODMA_OK;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return ODMA_ERR_INVALID;
+    const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
+    AppendParams ap;
+    ap.base = tab + tables->off_base;
+    ap.cap = tab + tables->off_cap;
+    ap.len = tab + tables->off_len;
+    ap.cu_new = tab + tables->off_cu_new;
+    ap.pool = pool->dev_base;
+    ap.k_new = k_new;
+    ap.v_new = v_new;
+    ap.rows_per_array = pool->rows_per_array;
+    ap.layer = layer;
+    ap.n = tables->n;
+    ap.kv_heads = pool->kv_heads;
+    ap.n_new_total = tables->n_new_total;
+    ap.row_vecs = pool->head_dim * pool->elem_bytes / 16;
+    ProfScope ps(pool, ODMA_K_APPEND, as_stream(stream));
+    return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
+}
+
+int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                              const odma_tables* tables, void* out, float* lse, void* stream) {
+    int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
+    if (rc != ODMA_OK) return rc;
+    DecodeParams p;
+    fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
+    cudaError_t e;
+    {
+        ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
+        if (pool->has_maps && tc_supported(pool->head_dim, p.group))
+            e = launch_decode_tc(pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream));
+        else if (generic_supported(pool->head_dim))
+            e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
+        else
+            return ODMA_ERR_INVALID;
+    }
+    if (e != cudaSuccess) return ODMA_ERR_CUDA;
+    if (tables->n_combine > 0) {
+        ProfScope ps(pool, ODMA_K_COMBINE, as_stream(stream));
+        const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
+        e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,
+                           pool->part_o, pool->part_ml, out, lse, p.group, pool->head_dim, q_heads,
+                           pool->dtype, as_stream(stream));
+        if (e != cudaSuccess) return ODMA_ERR_CUDA;
+    }
+    return ODMA_OK;
+}
+
+int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
+                              int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
+                              void* h_out, void* stream) {
+    if (!pool || !pool->dev_base || !h_q || !h_k_new || !h_v_new || !h_out) return ODMA_ERR_INVALID;
+    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0 ||
+        q_heads / pool->kv_heads > pool->alloc.config().max_group)
+        return ODMA_ERR_INVALID;
+    odma_tables t;
+    int32_t rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
+                                   static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
+    if (rc != ODMA_OK) return rc;
+    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
+    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(pool->d_q, h_q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(pool->d_k_new, h_k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(pool->d_v_new, h_v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    rc = odma_append_kv(pool, layer, &t, pool->d_k_new, pool->d_v_new, stream);
+    if (rc != ODMA_OK) return rc;
+    rc = odma_decode_attention(pool, layer, pool->d_q, q_heads, &t, pool->d_out, nullptr, stream);
+    if (rc != ODMA_OK) return rc;
+    if (cudaMemcpyAsync(h_out, pool->d_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    return ODMA_OK;
+}
+
+int32_t odma_check_status(odma_pool* pool, void* stream) {
+    if (!pool || !pool->dev_base) return ODMA_ERR_INVALID;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return ODMA_ERR_CUDA;
+    uint32_t word = 0;
+    if (cudaMemcpy(&word, pool->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return ODMA_ERR_CUDA;
+    if (word != 0 && cudaMemset(pool->d_status, 0, 4) != cudaSuccess) return ODMA_ERR_CUDA;
+    return (word & kStatusTimeout) ? ODMA_ERR_TIMEOUT : ODMA_OK;
+}
+
+int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const odma_tables* tables,
+                        void* stream) {
+    if (!pool || !pool->dev_base || !pool->has_maps || layer < 0 || layer >= pool->layers)
+        return ODMA_ERR_INVALID;
+    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
+    int32_t rc = check_tables(pool, tables);
+    if (rc != ODMA_OK) return rc;
+    DecodeParams p;
+    // the probe moves the query bytes too; any valid device memory of that size will do
+    fill_decode_params(pool, layer, pool->d_q, q_heads, tables, pool->d_out, nullptr, &p);
+    if (!tc_supported(pool->head_dim, p.group) || p.group > pool->alloc.config().max_group)
+        return ODMA_ERR_INVALID;
+    ProfScope ps(pool, ODMA_K_PROBE, as_stream(stream));
+    return launch_decode_tc(pool->maps, p, kModeProbe, tables->n_ctas, as_stream(stream)) == cudaSuccess
+               ? ODMA_OK
+               : ODMA_ERR_CUDA;
+}
+
+int32_t odma_profile_enable(odma_pool* pool, int32_t on) {
+    if (!pool || !pool->dev_base) return ODMA_ERR_INVALID;
+    if (cudaDeviceSynchronize() != cudaSuccess) return ODMA_ERR_CUDA;
+    clear_profile(pool);
+    pool->profiling = on != 0;
+    return ODMA_OK;
+}
+
+int32_t odma_profile_read(odma_pool* pool, int32_t kernel, double* total_ms, int64_t* launches) {
+    if (!pool || !pool->dev_base || kernel < 0 || kernel >= ODMA_K_COUNT) return ODMA_ERR_INVALID;
+    double ms = 0.0;
+    int64_t count = 0;
+    for (auto& r : pool->prof) {
+        if (r.kernel != kernel) continue;
+        if (cudaEventSynchronize(r.stop) != cudaSuccess) return ODMA_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, r.start, r.stop) != cudaSuccess) return ODMA_ERR_CUDA;
+        ms += t;
+        count += 1;
+    }
+    if (total_ms) *total_ms = ms;
+    if (launches) *launches = count;
+    return ODMA_OK;
+}
+
+/* Launches a one-thread kernel whose only wait can never be satisfied and must give up after
+ * limit_ms; odma_check_status then reports ODMA_ERR_TIMEOUT.  Shows that a lost signal ends in
+ * an error code, not in a hung GPU. */
+int32_t odma_selftest_timeout(odma_pool* pool, int32_t limit_ms, void* stream) {
+    if (!pool || !pool->dev_base || limit_ms < 1 || limit_ms > 1000) return ODMA_ERR_INVALID;
+    return launch_wait_selftest(pool->d_status, static_cast<int64_t>(limit_ms) * 1000000ll,
+                                as_stream(stream)) == cudaSuccess
+               ? ODMA_OK
+               : ODMA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// page-16 ablation
+// ---------------------------------------------------------------------------------------------
+
+int32_t odma_paged_create(odma_pool* pool, void* d_pages, uint64_t bytes, odma_paged** out) {
+    if (!out) return ODMA_ERR_INVALID;
+    *out = nullptr;
+    if (!pool || !pool->dev_base || !d_pages || (reinterpret_cast<uintptr_t>(d_pages) & 255u) != 0)
+        return ODMA_ERR_INVALID;
+    const uint64_t page_bytes = static_cast<uint64_t>(pool->layers) * 2u * pool->kv_heads * 16u *
+                                pool->head_dim * pool->elem_bytes;
+    const int64_t n_pages = static_cast<int64_t>(bytes / page_bytes);
+    if (n_pages < 1 || n_pages * pool->kv_heads * 16 * pool->layers * 2 >= (int64_t(1) << 31))
+        return ODMA_ERR_INVALID;
+    odma_paged* pg = new (std::nothrow) odma_paged();
+    if (!pg) return ODMA_ERR_NOMEM;
+    pg->pool = pool;
+    pg->d_pages = d_pages;
+    pg->n_pages = n_pages;
+    if (pool->has_maps) {
+        if (make_tensor_maps(d_pages, n_pages * pool->kv_heads * 16 * pool->layers * 2, pool->head_dim,
+                             &pg->maps) != ODMA_OK) {
+            delete pg;
+            return ODMA_ERR_CUDA;
+        }
+        pg->has_maps = true;
+    }
+    *out = pg;
+    return ODMA_OK;
+}
+
+int32_t odma_paged_destroy(odma_paged* paged) {
+    if (!paged) return ODMA_ERR_INVALID;
+    if (paged->pinned) cudaFreeHost(paged->pinned);
+    delete paged;
+    return ODMA_OK;
+}
+
+int32_t odma_paged_build(odma_paged* paged, const odma_tables* tables, const int32_t* host_len,
+                         uint64_t shuffle_seed, int32_t* d_page_table, int32_t max_pages, void* stream) {
+    if (!paged || !tables || !tables->d_table || !host_len || !d_page_table || max_pages < 1)
+        return ODMA_ERR_INVALID;
+    odma_pool* pool = paged->pool;
+    const int32_t n = tables->n;
+    int64_t need = 0;
+    int32_t longest = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const int32_t pages = (host_len[i] + 15) / 16;
+        if (host_len[i] < 1 || pages > max_pages) return ODMA_ERR_INVALID;
+        need += pages;
+        longest = std::max(longest, host_len[i]);
+    }
+    if (need > paged->n_pages) return ODMA_ERR_NOMEM;
+    // page ids: 0,1,2,... in request order, or a seeded permutation of all pages of the buffer
+    std::vector<int32_t> ids(static_cast<size_t>(shuffle_seed ? paged->n_pages : need));
+    for (size_t i = 0; i < ids.size(); ++i) ids[i] = static_cast<int32_t>(i);
+    if (shuffle_seed) {
+        uint64_t s = shuffle_seed;
+        auto next = [&s]() {                 // splitmix64
+            uint64_t z = (s += 0x9E3779B97F4A7C15ull);
+            z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+            z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+            return z ^ (z >> 31);
+        };
+        for (size_t i = ids.size() - 1; i > 0; --i) std::swap(ids[i], ids[next() % (i + 1)]);
+    }
+    const int64_t words = static_cast<int64_t>(n) * max_pages;
+    if (words > paged->pinned_words) {
+        if (paged->pinned) cudaFreeHost(paged->pinned);
+        paged->pinned = nullptr;
+        if (cudaMallocHost(&paged->pinned, static_cast<size_t>(words) * 4) != cudaSuccess) return ODMA_ERR_CUDA;
+        paged->pinned_words = words;
+    }
+    std::fill(paged->pinned, paged->pinned + words, 0);
+    size_t k = 0;
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t pg = 0; pg < (host_len[i] + 15) / 16; ++pg)
+            paged->pinned[static_cast<size_t>(i) * max_pages + pg] = ids[k++];
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(d_page_table, paged->pinned, static_cast<size_t>(words) * 4, cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+        return ODMA_ERR_CUDA;
+    const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
+    ScatterPagesParams sp;
+    sp.base = tab + tables->off_base;
+    sp.cap = tab + tables->off_cap;
+    sp.len = tab + tables->off_len;
+    sp.page_table = d_page_table;
+    sp.pool = pool->dev_base;
+    sp.pages = paged->d_pages;
+    sp.rows_per_array = pool->rows_per_array;
+    sp.n_pages = paged->n_pages;
+    sp.n = n;
+    sp.max_pages = max_pages;
+    sp.arrays = pool->layers * 2;
+    sp.kv_heads = pool->kv_heads;
+    sp.row_vecs = pool->head_dim * pool->elem_bytes / 16;
+    if (launch_scatter_pages(sp, longest, s) != cudaSuccess) return ODMA_ERR_CUDA;
+    // the pinned table is reused by the next call: wait for the copy
+    return cudaStreamSynchronize(s) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
+}
+
+int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void* q, int32_t q_heads,
+                                    const odma_tables* tables, const int32_t* d_page_table,
+                                    int32_t max_pages, void* out, float* lse, void* stream) {
+    if (!paged || !paged->has_maps || !d_page_table || max_pages < 1) return ODMA_ERR_INVALID;
+    odma_pool* pool = paged->pool;
+    int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
+    if (rc != ODMA_OK) return rc;
+    DecodeParams p;
+    fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
+    if (!tc_supported(pool->head_dim, p.group)) return ODMA_ERR_INVALID;
+    p.pool = paged->d_pages;
+    p.rows_per_array = paged->n_pages * pool->kv_heads * 16;
+    p.page_table = d_page_table;
+    p.max_pages = max_pages;
+    cudaError_t e;
+    {
+        ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
+        e = launch_decode_tc(paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream));
+    }
+    if (e != cudaSuccess) return ODMA_ERR_CUDA;
+    if (tables->n_combine > 0) {
+        ProfScope ps(pool, ODMA_K_COMBINE, as_stream(stream));
+        const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
+        e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,
+                           pool->part_o, pool->part_ml, out, lse, p.group, pool->head_dim, q_heads,
+                           pool->dtype, as_stream(stream));
+        if (e != cudaSuccess) return ODMA_ERR_CUDA;
+    }
+    return ODMA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,97 @@
+// Device side of libodma: kernel parameter blocks and host launchers (kernels.cu).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace odma {
+
+// Status word bits written by kernels.
+constexpr uint32_t kStatusTimeout = 1u;
+
+struct DecodeParams {
+    // per-step tables (device)
+    const int32_t* base;
+    const int32_t* cap;
+    const int32_t* len;
+    const int32_t* cta_begin;
+    const int4* items;          // two int4 per item
+    // tensors
+    const void* q;              // [n, q_heads, head_dim]
+    void* out;                  // [n, q_heads, head_dim]
+    float* lse;                 // [n, q_heads] or nullptr
+    float* part_o;              // [slots, group, head_dim] unnormalised partial outputs
+    float* part_ml;             // [slots, group, 2] running max (log2 domain) and sum
+    const void* pool;           // base of the slab pool (or of the paged copy)
+    int64_t rows_per_array;     // T * kv_heads   (paged: n_pages * kv_heads * 16)
+    int32_t layer;
+    int32_t q_heads, kv_heads, group, head_dim;
+    float scale_log2;           // log2(e) / sqrt(head_dim)
+    uint32_t* status;
+    // page-16 ablation
+    const int32_t* page_table;  // [n, max_pages]
+    int32_t max_pages;
+    int64_t wait_limit_ns;
+};
+
+struct TensorMaps {
+    CUtensorMap big;    // box 64 rows x 64 elements
+    CUtensorMap small;  // box 16 rows x 64 elements
+};
+
+enum DecodeMode { kModeSlab = 0, kModePaged = 1, kModeProbe = 2 };
+
+// Returns false when (head_dim, group) has no tensor-core instantiation.
+bool tc_supported(int32_t head_dim, int32_t group);
+cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
+                             cudaStream_t stream);
+cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
+bool generic_supported(int32_t head_dim);
+
+cudaError_t launch_combine(const int4* combine, int n_combine, const float* part_o,
+                           const float* part_ml, void* out, float* lse, int group, int head_dim,
+                           int q_heads, int dtype, cudaStream_t stream);
+
+struct AppendParams {
+    const int32_t* base;
+    const int32_t* cap;
+    const int32_t* len;
+    const int32_t* cu_new;
+    void* pool;
+    const void* k_new;
+    const void* v_new;
+    int64_t rows_per_array;
+    int32_t layer, n, kv_heads, n_new_total;
+    int32_t row_vecs;           // 16-byte vectors per row
+};
+cudaError_t launch_append(const AppendParams& p, cudaStream_t stream);
+
+struct MigrateParams {
+    void* pool;
+    int64_t rows_per_array;
+    int64_t src_base, src_cap, dst_base, dst_cap, len;
+    int32_t arrays;             // layers * 2
+    int32_t kv_heads, row_vecs;
+};
+cudaError_t launch_migrate(const MigrateParams& p, cudaStream_t stream);
+
+struct ScatterPagesParams {
+    const int32_t* base;
+    const int32_t* cap;
+    const int32_t* len;
+    const int32_t* page_table;
+    const void* pool;
+    void* pages;
+    int64_t rows_per_array;      // slab pool
+    int64_t n_pages;
+    int32_t n, max_pages, arrays, kv_heads, row_vecs;
+};
+cudaError_t launch_scatter_pages(const ScatterPagesParams& p, int64_t max_len, cudaStream_t stream);
+
+// A one-thread kernel that waits on a barrier nobody signals, for at most limit_ns, then
+// sets the timeout bit: exercises the bounded-wait path without hanging anything.
+cudaError_t launch_wait_selftest(uint32_t* status, int64_t limit_ns, cudaStream_t stream);
+
+}  // namespace odma

@@ -293,6 +293,7 @@ class DriftResult:
     migrations: int = 0
     admitted: int = 0
     deferred: int = 0
+    preempted: int = 0
     boundary_log: List[Tuple[int, Tuple[int, ...]]] = field(default_factory=list)
 
 
@@ -304,8 +305,9 @@ def run_closed_loop(alloc, total_len: np.ndarray, predicted: np.ndarray, concurr
 
     `alloc` offers alloc(req, predicted) -> slab tuple (base, cap, pool, bucket)
     or None when memory is short, ensure(req, need) -> (slab tuple, migrated),
-    commit(reqs, n_new) for a list of requests, free(req) and
-    buckets() -> (tuple, epoch).  Request r is admitted with a prompt of
+    or None when the Large Bucket cannot take the request (the request is then
+    preempted: freed at its current length), commit(reqs, n_new) for a list of
+    requests, free(req) and buckets() -> (tuple, epoch).  Request r is admitted with a prompt of
     max(1, total_len[r] // 4) tokens already in its slab, gains one token per
     step, and is freed when it reaches total_len[r]; the next request of the
     trace takes its place.  Steps in which nothing happens to the allocator are
@@ -334,11 +336,18 @@ def run_closed_loop(alloc, total_len: np.ndarray, predicted: np.ndarray, concurr
                 break
             prompt = max(1, int(total_len[r]) // 4)
             if prompt > slab[1]:
-                slab, mig = alloc.ensure(r, prompt)
-                res.migrations += int(mig)
+                ans = alloc.ensure(r, prompt)
                 res.events += 1
                 if on_event:
-                    on_event("ensure", r, (slab, mig))
+                    on_event("ensure", r, ans)
+                if ans is None:
+                    alloc.free(r)
+                    res.events += 1
+                    res.preempted += 1
+                    nxt += 1
+                    continue
+                slab, mig = ans
+                res.migrations += int(mig)
             alloc.commit([r], prompt)
             live.append(r)
             cur.append(prompt)
@@ -358,14 +367,26 @@ def run_closed_loop(alloc, total_len: np.ndarray, predicted: np.ndarray, concurr
             k = min(k, int((k_cap - c)[grow].min()))
         if k <= 0:
             # some request stands at the end of its slab and still has tokens to produce
+            dropped = []
             for j, r in enumerate(live):
                 if cur[j] >= cap[j] and cur[j] < int(total_len[r]):
-                    slab, mig = alloc.ensure(r, cur[j] + 1)
-                    res.migrations += int(mig)
+                    ans = alloc.ensure(r, cur[j] + 1)
                     res.events += 1
-                    cap[j] = int(slab[1])
                     if on_event:
-                        on_event("ensure", r, (slab, mig))
+                        on_event("ensure", r, ans)
+                    if ans is None:
+                        alloc.free(r)
+                        res.events += 1
+                        res.preempted += 1
+                        dropped.append(j)
+                        continue
+                    slab, mig = ans
+                    res.migrations += int(mig)
+                    cap[j] = int(slab[1])
+            for j in reversed(dropped):
+                del live[j], cur[j], cap[j]
+            if dropped:
+                admit()
             continue
         alloc.commit(list(live), k)
         for j in range(len(cur)):

@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+from conftest import read_golden
+from helpers import (BF16_MAX_ABS, BF16_REL_L2, Session, assert_close, attention_errors, lib)
+from paper_2512_09427_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 500, 1000, 2771]
+
+
+def qwen_small(lens, layers=1, q_heads=28, kv_heads=4, head_dim=128, dtype=torch.bfloat16, seed=77):
+    """A Qwen-shaped workload over explicit context lengths with one static bucket ladder."""
+    ladder = (16, 64, 256, 1024, 4096)
+    ctx = np.asarray(lens, dtype=np.int64)
+    tokens = int(sum(min(b for b in ladder if b >= L + 1) for L in lens) * 1.5) + 8192
+    esz = 2 if dtype == torch.bfloat16 else 4
+    return wl.Workload(name="small", seed=seed, layers=layers, q_heads=q_heads, kv_heads=kv_heads,
+                       head_dim=head_dim, dtype=dtype, pool_bytes=tokens * layers * 2 * kv_heads * head_dim * esz,
+                       safety_pct=25, max_len=4096, context=ctx, predicted=ctx + 1, static_buckets=ladder)
+
+
+def run_decode(w, cfg_over=None, fill=None, scale=1.0, layers=None):
+    s = Session(w, fill=fill, **(cfg_over or {}))
+    if w.static_buckets:
+        assert s.pool.set_buckets(list(w.static_buckets)) == s.ls.oracle.set_buckets(list(w.static_buckets)) == 0
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    pre = [r for r in reqs if w.context[r] > 0]
+    if pre:
+        s.append(pre, [int(w.context[r]) for r in pre], scale=scale)
+    res = s.decode_step(reqs, w.q_heads, layers=layers, scale=scale)
+    return s, reqs, res
+
+
+def check_all(s, reqs, res, what=""):
+    worst = (0.0, 0.0)
+    for layer, (out, lse, q) in res.items():
+        ref, ref_lse, _ = s.oracle_out(layer, reqs, q, s.w.q_heads)
+        assert torch.isfinite(out.float()).all(), what
+        e = assert_close(out, ref, s.w.dtype, f"{what} layer {layer}")
+        worst = max(worst, e)
+        l = lse.double().cpu().numpy()
+        assert np.isfinite(l).all()
+        assert np.abs(l - ref_lse).max() <= (2e-2 if s.w.dtype == torch.bfloat16 else 1e-5), what
+    return worst
+
+
+# ---------------------------------------------------------------------------------------------
+
+
+@pytest.mark.parametrize("variant", ["a", "b"])
+def test_config1_allocation_append_and_attention(variant):
+    w = wl.config1(variant)
+    s, reqs, res = run_decode(w, fill=0x7B7B)       # sentinel-filled pool: canary for stray writes
+    # slab tables equal the hand-computed ones
+    rows = [r for r in read_golden("config1_alloc.txt") if r[0] == "1" + variant and r[1] == "ensure"]
+    for _, _, req, _, base, cap, pl, bucket, _ in rows:
+        rc, slab, ln = s.pool.get_slab(int(req))
+        assert slab[:4] == (int(base), int(cap), int(pl), int(bucket))
+        assert ln == int(w.context[int(req)]) + 1
+    if variant == "b":
+        assert s.pool.get_stats()["migrations"] == 1
+    check_all(s, reqs, res, "config1" + variant)
+    # the pool, read back through the documented layout, holds exactly the appended rows ...
+    touched = torch.zeros(s.T * w.kv_heads, dtype=torch.bool, device=s.dev)
+    for r in reqs:
+        k_ref, v_ref = s.kv.gathered(r, 0)
+        assert np.array_equal(s.pool_rows(0, 0, r).cpu().numpy(), k_ref)
+        assert np.array_equal(s.pool_rows(0, 1, r).cpu().numpy(), v_ref)
+        rc, slab, ln = s.pool.get_slab(r)
+        touched[slab[0] * w.kv_heads: slab[0] * w.kv_heads + ln] = True
+    # ... and nothing else was written (the migrated request's old slab [64,128) still holds its copy)
+    arr = s.mem.view(torch.int16)[: 2 * s.T * w.kv_heads * w.head_dim * 2].view(2, s.T * w.kv_heads, -1)
+    if variant == "b":
+        touched[64:128] = True
+    assert (arr[:, ~touched] == 0x7B7B).all()
+
+
+@pytest.mark.parametrize("ctas", [0, 1, 7])
+def test_bf16_ragged_lengths_span_tiles_and_splits(ctas):
+    w = qwen_small([L - 1 for L in RAGGED])
+    s, reqs, res = run_decode(w, cfg_over={"plan_ctas": ctas})
+    t = s.last_tables
+    if ctas == 7:
+        assert t.n_combine > 0                      # some streams were split and merged
+    if ctas == 1:
+        assert t.n_combine == 0
+    err = check_all(s, reqs, res, f"ragged ctas={ctas}")
+    print("bf16 ragged", ctas, err)
+
+
+def test_bf16_multi_layer_and_second_step():
+    w = qwen_small([40, 300, 64, 1, 130], layers=3)
+    s, reqs, res = run_decode(w)
+    check_all(s, reqs, res, "3 layers")
+    res2 = s.decode_step(reqs, w.q_heads, step=1)
+    check_all(s, reqs, res2, "second step")
+    for layer in range(3):
+        for r in reqs:
+            k_ref, v_ref = s.kv.gathered(r, layer)
+            assert np.array_equal(s.pool_rows(layer, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+            assert np.array_equal(s.pool_rows(layer, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
+@pytest.mark.parametrize("q_heads,kv_heads,head_dim", [(24, 2, 128), (24, 2, 64), (8, 8, 64), (14, 2, 128), (4, 4, 128)])
+def test_bf16_other_group_sizes_and_head_dims(q_heads, kv_heads, head_dim):
+    w = qwen_small([5, 63, 64, 200, 777], q_heads=q_heads, kv_heads=kv_heads, head_dim=head_dim)
+    s, reqs, res = run_decode(w, cfg_over={"max_group": 16, "plan_ctas": 5})
+    check_all(s, reqs, res, f"{q_heads}/{kv_heads}/{head_dim}")
+
+
+@pytest.mark.parametrize("dtype,q_heads,kv_heads,head_dim", [
+    (torch.float32, 28, 4, 128), (torch.float32, 2, 1, 64), (torch.float32, 6, 2, 32),
+    (torch.bfloat16, 40, 2, 128), (torch.bfloat16, 6, 2, 32)])
+def test_generic_path_fp32_and_wide_groups(dtype, q_heads, kv_heads, head_dim):
+    w = qwen_small([0, 31, 32, 100, 257, 900], q_heads=q_heads, kv_heads=kv_heads, head_dim=head_dim, dtype=dtype)
+    s, reqs, res = run_decode(w, cfg_over={"max_group": 32, "plan_ctas": 6})
+    check_all(s, reqs, res, f"generic {dtype} {q_heads}/{kv_heads}/{head_dim}")
+
+
+def test_nan_poisoned_pool_changes_nothing():
+    lens = [L - 1 for L in RAGGED]
+    w = qwen_small(lens)
+    s0, reqs, res0 = run_decode(w)
+    s1, _, res1 = run_decode(w, fill=0x7FC0)        # every untouched bf16 is a NaN
+    for layer in res0:
+        assert torch.isfinite(res1[layer][0].float()).all()
+        assert torch.equal(res0[layer][0], res1[layer][0])
+        assert torch.equal(res0[layer][1], res1[layer][1])
+
+
+def test_scores_scaled_by_eight_stay_stable():
+    w = qwen_small([100, 1000, 64])
+    s, reqs, res = run_decode(w, scale=8.0 ** 0.5)       # q and k both scaled: scores x 8
+    for layer, (out, lse, q) in res.items():
+        ref, ref_lse, _ = s.oracle_out(layer, reqs, q, w.q_heads)
+        assert torch.isfinite(out.float()).all()
+        err, rel = attention_errors(out, ref)
+        # softmax is nearly one-hot here: bf16 rounding of P matters less, of the output more
+        assert err <= 2e-2 and rel <= 1e-2, (err, rel)
+
+
+def test_migration_keeps_the_cache_and_attention_right():
+    # slabs exactly full before the step: every request migrates to the Large Bucket
+    w = qwen_small([16, 64, 256], layers=2)
+    w = wl.scaled(w, predicted=w.context.copy())
+    s, reqs, res = run_decode(w)
+    assert s.pool.get_stats()["migrations"] == 3
+    for r in reqs:
+        assert s.pool.get_slab(r)[1][2] == 1
+    check_all(s, reqs, res, "migrated")
+
+
+def test_paged_copy_gives_the_same_attention():
+    odma = lib()
+    lens = [L - 1 for L in RAGGED]
+    w = qwen_small(lens, layers=2)
+    s, reqs, res = run_decode(w, cfg_over={"plan_ctas": 9})
+    t = s.last_tables
+    host_len = [s.lens[r] for r in reqs]
+    max_pages = max(-(-L // 16) for L in host_len)
+    n_pages = sum(-(-L // 16) for L in host_len) + 37
+    page_bytes = w.layers * 2 * w.kv_heads * 16 * w.head_dim * 2
+    pages = torch.zeros(n_pages * page_bytes, dtype=torch.uint8, device=s.dev)
+    ptab = torch.zeros(len(reqs) * max_pages, dtype=torch.int32, device=s.dev)
+    paged = odma.Paged(s.pool, pages.data_ptr(), pages.numel())
+    for seed in (0, 12345):
+        pages.view(torch.int16).fill_(0x7FC0)
+        paged.build(t, host_len, seed, ptab.data_ptr(), max_pages, s.stream)
+        ids = ptab.view(len(reqs), max_pages).cpu().numpy()
+        used = np.concatenate([ids[i, : -(-L // 16)] for i, L in enumerate(host_len)])
+        assert len(set(used.tolist())) == len(used) and used.max() < n_pages
+        if seed == 0:
+            assert used.tolist() == list(range(len(used)))
+        else:
+            assert used.tolist() != sorted(used.tolist())
+        for layer, (out, lse, q) in res.items():
+            out_p = torch.full_like(out, float("nan"))
+            lse_p = torch.full_like(lse, float("nan"))
+            paged.decode_attention(layer, q.data_ptr(), w.q_heads, t, ptab.data_ptr(), max_pages,
+                                   out_p.data_ptr(), lse_p.data_ptr(), s.stream)
+            torch.cuda.synchronize()
+            assert s.pool.check_status(s.stream) == 0
+            assert torch.equal(out_p, out) and torch.equal(lse_p, lse)     # same arithmetic, other layout
+
+
+def test_read_probe_and_bounded_wait_selftest():
+    odma = lib()
+    w = qwen_small([100, 1000, 64])
+    s, reqs, res = run_decode(w)
+    s.pool.read_probe(0, w.q_heads, s.last_tables, s.stream)
+    assert s.pool.check_status(s.stream) == odma.OK
+    # a wait that nothing will ever satisfy gives up and reports, and the context lives on
+    assert s.pool.selftest_timeout(20, s.stream) == odma.OK
+    assert s.pool.check_status(s.stream) == odma.ERR_TIMEOUT
+    assert s.pool.check_status(s.stream) == odma.OK
+    res2 = s.decode_step(reqs, w.q_heads, step=1)
+    check_all(s, reqs, res2, "after the timeout self-test")
+
+
+def test_decode_step_from_host_buffers_matches_the_device_path():
+    w = qwen_small([10, 200, 64, 999])
+    s = Session(w)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    s.append(reqs, [int(c) for c in w.context])
+    for r in reqs:
+        s.ls.ensure(r, s.lens[r] + 1)
+    q = s.queries(0, reqs, w.q_heads).cpu().pin_memory()
+    k_new = torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu().pin_memory()
+    v_new = torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu().pin_memory()
+    out = torch.empty_like(q).pin_memory()
+    s.pool.decode_step_host(0, w.q_heads, reqs, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                            out.data_ptr(), s.stream)
+    torch.cuda.synchronize()
+    assert s.pool.check_status(s.stream) == 0
+    for i, r in enumerate(reqs):
+        s.kv.append(r, 0, k_new[i:i + 1], v_new[i:i + 1])
+    ref, _, _ = s.oracle_out(0, reqs, q, w.q_heads)
+    assert_close(out, ref, w.dtype, "host step")
+
+
+def test_profile_counts_launches():
+    odma = lib()
+    w = qwen_small([100, 1000, 64])
+    s, reqs, _ = run_decode(w, cfg_over={"plan_ctas": 4})
+    s.pool.profile_enable(True)
+    s.decode_step(reqs, w.q_heads, step=1)
+    ms, n = s.pool.profile_read(odma.K_DECODE)
+    assert n == 1 and ms > 0
+    assert s.pool.profile_read(odma.K_APPEND)[1] == 1
+    assert s.pool.profile_read(odma.K_COMBINE)[1] == (1 if s.last_tables.n_combine else 0)
+    s.pool.profile_enable(False)
+
+
+def test_config2_full_size_parity():
+    """The benchmark workload itself: 64 requests, log-normal contexts, learned quartile buckets."""
+    from helpers import warm_up
+    w = wl.config2()
+    s = Session(w)
+    warm_up(s.ls, w.warmup_lengths)
+    bounds, epoch = s.ls.buckets()
+    assert epoch == 10 and len(bounds) == 4
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    s.append(reqs, [int(c) for c in w.context])
+    res = s.decode_step(reqs, w.q_heads)
+    err = check_all(s, reqs, res, "config2")
+    st = s.ls.check_stats()
+    print("config2 parity", err, "buckets", bounds, "reserved", st["reserved_live"], "used", st["used_live"])

@@ -1,0 +1,83 @@
+"""Invariants of the host-built split plan (no GPU)."""
+import numpy as np
+import pytest
+
+from helpers import host_pool, lib
+from paper_2512_09427_b200 import workloads as wl
+
+
+def _plan(lens, kv_heads=4, ctas=148, max_len=32768 + 4096):
+    buckets = [64, 256, 1024, 4096, 16384, max_len]
+    tokens = sum(min(b for b in buckets if b >= L) for L in lens)
+    w = wl.scaled(wl.config5(batch=1), pool_bytes=int(tokens * 1.3 + 64) * 2 * kv_heads * 128 * 2,
+                  layers=1, kv_heads=kv_heads, max_len=max_len)
+    pool = host_pool(w, plan_ctas=ctas, max_batch=max(1024, len(lens)))
+    assert pool.set_buckets(buckets) == 0
+    reqs = list(range(len(lens)))
+    for r, L in zip(reqs, lens):
+        rc, slab = pool.alloc(r, int(L))
+        assert rc == 0, rc
+        if L > 1:
+            assert pool.commit_step([r], [int(L) - 1]) == 0
+    rc, t, words = pool.plan_host(reqs)
+    assert rc == 0
+    return pool, t, np.array(words, dtype=np.int64)
+
+
+@pytest.mark.parametrize("lens", [
+    [1], [64], [65], [17, 64, 100, 250], list(range(1, 200, 7)),
+    list(wl.config2().context + 1), list(wl.config3().context + 1), list(wl.config5().context + 1),
+    [16384] + [33] * 255,
+])
+@pytest.mark.parametrize("ctas", [1, 7, 148])
+def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
+    hkv = 4
+    pool, t, w = _plan(lens, hkv, ctas)
+    n = len(lens)
+    assert t.n == n and t.kv_tokens == sum(lens) and t.n_new_total == n and t.tile_tokens == 64
+    assert list(w[t.off_len:t.off_len + n]) == list(lens)
+    assert list(w[t.off_cu_new:t.off_cu_new + n + 1]) == list(range(n + 1))
+    items = w[t.off_items:t.off_items + 8 * t.n_items].reshape(-1, 8)
+    cta_begin = w[t.off_cta_begin:t.off_cta_begin + t.n_ctas + 1]
+    assert cta_begin[0] == 0 and cta_begin[-1] == t.n_items and (np.diff(cta_begin) >= 0).all()
+    assert t.n_ctas <= ctas
+    # coverage: per stream the items tile [0, len) in order with no gap or overlap
+    cover = {}
+    for k, (req, head, tok0, ntok, direct, slot, _, _) in enumerate(items):
+        assert slot == k and ntok >= 1 and tok0 % 64 == 0
+        cur = cover.get((req, head), 0)
+        assert tok0 == cur
+        cover[(req, head)] = tok0 + ntok
+        whole = tok0 == 0 and ntok == lens[req]
+        assert bool(direct) == whole
+        if tok0 + ntok < lens[req]:
+            assert ntok % 64 == 0                     # only a stream's last piece is ragged
+    assert cover == {(r, h): lens[r] for r in range(n) for h in range(hkv)}
+    # items are in (request, head, token) order, so a stream's slots are consecutive
+    keys = [(int(a), int(b), int(c)) for a, b, c in items[:, :3]]
+    assert keys == sorted(keys)
+    comb = w[t.off_combine:t.off_combine + 4 * t.n_combine].reshape(-1, 4)
+    split = {}
+    for k, (req, head, *_rest) in enumerate(items):
+        split.setdefault((int(req), int(head)), []).append(k)
+    want = [(r, h, ks[0], len(ks)) for (r, h), ks in sorted(split.items()) if len(ks) > 1]
+    assert [tuple(int(x) for x in c) for c in comb] == want
+    # balance: tiles per CTA within the snapping slack of the ideal share
+    tiles = np.array([sum(-(-int(items[k, 3]) // 64) for k in range(cta_begin[c], cta_begin[c + 1]))
+                      for c in range(t.n_ctas)])
+    total = sum(-(-L // 64) for L in lens) * hkv
+    assert tiles.sum() == total
+    ideal = total / t.n_ctas
+    assert tiles.max() <= np.ceil(ideal) + 2 and tiles.min() >= np.floor(ideal) - 2
+    assert t.words * 4 <= pool.tables_bytes(n)
+
+
+def test_plan_rejects_bad_batches():
+    odma = lib()
+    pool, t, w = _plan([10, 20])
+    assert pool.plan_host([0, 99])[0] == odma.ERR_UNKNOWN_REQ
+    # request 0 sits at length 9 in a slab of... fill it to the brim, then one more does not fit
+    rc, slab, ln = pool.get_slab(0)
+    assert pool.commit_step([0], [slab[1] - ln]) == 0
+    assert pool.plan_host([0, 1])[0] == odma.ERR_OVERFLOW
+    assert pool.plan_host([0, 1], [0, 1])[0] == odma.OK
