@@ -240,7 +240,8 @@ class Session:
         assert rc == 0
         base, cap = slab[0], slab[1]
         w = self.w
-        arr = self.mem.view(w.dtype).view(w.layers * 2, self.T * w.kv_heads, w.head_dim)[layer * 2 + kv]
+        n_elems = w.layers * 2 * self.T * w.kv_heads * w.head_dim
+        arr = self.mem.view(w.dtype)[:n_elems].view(w.layers * 2, self.T * w.kv_heads, w.head_dim)[layer * 2 + kv]
         heads = [arr[base * w.kv_heads + h * cap: base * w.kv_heads + h * cap + ln] for h in range(w.kv_heads)]
         return torch.stack(heads, dim=1)
 
