@@ -1,0 +1,537 @@
+"""Decode-step benchmark of the slab-KV attention path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config3|config5]
+                    [--impl ours|reference]
+
+One step = one pass of the whole device path over one batch: per-step tables (host split plan
++ one small copy), KV append of one new token per request, split decode attention over every
+request's slab and the log-sum-exp combine, for the layers the workload steps through.
+Prints one JSON line (rank 0).  `value` = decode tokens/s with every input resident in HBM;
+`e2e` = the same step from pinned HOST buffers through odma_decode_step_host, copies inside
+the timed region; `roofline` = the decode kernel's algorithmic KV bytes over its CUDA-event
+time against the measured copy bandwidth; `cpu_baseline` = the fp64 CPU checker timed on the
+host cores (a reported baseline).  `--impl reference` times the CPU checker alone.
+
+Multi-GPU (torchrun, one rank per GPU): independent replicas of the same step, no collective
+on the data path; timing is barrier + synchronize on both sides, max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2512_09427_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode tokens/s (slab-KV attention path: append + split decode + combine)"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 2**20
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per decode-kernel launch, from the ncu capture
+# summarised under profiles/ (None once the kernel has changed since the capture)
+TRAFFIC = {"config2": None}
+
+
+# ---------------------------------------------------------------------------------------------
+# workload set-up through the C ABI (no checker code on this path)
+# ---------------------------------------------------------------------------------------------
+
+def pick_workload(name: str, rank: int = 0, copies_override: int = 0):
+    """Returns (workload, layers stepped per step, number of rotating KV copies).
+
+    config2 is one layer; the pool is given several `layers`, each an independent copy of the
+    single-layer cache, and consecutive steps rotate over them so that no step finds its KV in
+    L2 (one copy is ~90 MB, L2 is 126 MB).  config3/config5 step through all their layers,
+    which together are far larger than L2."""
+    seed_off = 1000 * rank
+    if name == "config2":
+        base = wl.config2(seed=950902 + seed_off)
+        kv_bytes = int((base.context + 1).sum()) * 2 * base.kv_heads * base.head_dim * 2
+        copies = copies_override or max(4, -(-3 * L2_BYTES // kv_bytes))
+        w = wl.config2(layers=copies, seed=950902 + seed_off)
+        step_layers = 1
+    elif name == "config3":
+        w = wl.config3(seed=950903 + seed_off)
+        copies, step_layers = 1, w.layers
+    elif name == "config5":
+        w = wl.config5(seed=950905 + seed_off)
+        copies, step_layers = 1, w.layers
+    else:
+        raise SystemExit(f"unknown workload {name}")
+    return w, step_layers, copies
+
+
+class SlabDecode:
+    """A device pool filled with the workload's KV, plus the step's input buffers."""
+
+    def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0):
+        from paper_2512_09427_b200 import odma
+        self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
+        self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
+        cfg = odma.config_default()
+        cfg.safety_pct, cfg.max_len, cfg.granule = w.safety_pct, w.max_len, w.granule
+        cfg.window, cfg.refresh = w.window, w.refresh
+        pn, pd = w.quantiles
+        cfg.n_levels = len(pn)
+        for i, x in enumerate(pn):
+            cfg.p_num[i] = x
+        cfg.p_den = pd
+        cfg.max_batch = max(1024, w.batch)
+        cfg.plan_ctas = plan_ctas
+        self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
+                              self.dt, cfg)
+        self.reqs = list(range(w.batch))
+        self.reqs_c = (C.c_uint64 * w.batch)(*self.reqs)
+        self.zeros_c = (C.c_int32 * w.batch)()
+        self.migrations_at_fill = 0
+
+    def learn_boundaries(self):
+        """Static ladder, or boundaries learned from the warm-up window of realised lengths."""
+        w, pool = self.w, self.pool
+        if w.static_buckets:
+            assert pool.set_buckets(list(w.static_buckets)) == 0
+        if w.warmup_lengths is not None:
+            for i, L in enumerate(w.warmup_lengths):
+                r = (1 << 40) + i
+                rc, _ = pool.alloc(r, int(L))
+                assert rc == 0, rc
+                assert pool.commit_step([r], [int(L)]) == 0
+                assert pool.free(r) == 0
+        return pool.get_buckets()
+
+    def admit_and_fill(self):
+        """Reserve every request's slab and write its context tokens (seeded N(0,1)) on all layers."""
+        w, pool, odma = self.w, self.pool, self.odma
+        for r in self.reqs:
+            rc, _ = pool.alloc(r, int(w.predicted[r]))
+            assert rc == odma.OK, ("alloc", r, rc)
+            rc, _, _ = pool.ensure_capacity(r, int(w.context[r]) + 1, self.stream)
+            assert rc == odma.OK, ("ensure", r, rc)
+        table = torch.empty(pool.tables_bytes(w.batch), dtype=torch.uint8, device=self.dev)
+        ctx = [int(c) for c in w.context]
+        t = pool.build_tables(self.reqs, table.data_ptr(), table.numel(), self.stream, ctx)
+        chunk = max(1, (1 << 26) // (w.kv_heads * w.head_dim))      # tokens per generated piece
+        for layer in range(w.layers):
+            for kind, name in ((wl.KIND_K, "k"), (wl.KIND_V, "v")):
+                pieces = [wl.kv_rows(w.seed, layer, r, kind, t0, min(t0 + chunk, c), w.kv_heads,
+                                     w.head_dim, w.dtype, self.dev)
+                          for r, c in zip(self.reqs, ctx) for t0 in range(0, c, chunk)]
+                if name == "k":
+                    k_all = torch.cat(pieces)
+                else:
+                    v_all = torch.cat(pieces)
+            pool.append_kv(layer, t, k_all.data_ptr(), v_all.data_ptr(), self.stream)
+            torch.cuda.synchronize()
+            del k_all, v_all, pieces
+        assert pool.commit_step(self.reqs, ctx) == 0
+        self.migrations_at_fill = pool.get_stats()["migrations"]
+
+    def make_inputs(self, pinned: bool = False):
+        """Per layer: q [n,Hq,D] and the new token's K/V rows [n,Hkv,D] (seeded), and out."""
+        w = self.w
+        q = torch.stack([torch.stack([wl.q_rows(w.seed, l, r, 0, w.q_heads, w.head_dim, w.dtype, self.dev)
+                                      for r in self.reqs]) for l in range(w.layers)]).contiguous()
+        kn = torch.stack([torch.cat([wl.kv_rows(w.seed, l, r, wl.KIND_K, int(w.context[r]), int(w.context[r]) + 1,
+                                                w.kv_heads, w.head_dim, w.dtype, self.dev) for r in self.reqs])
+                          for l in range(w.layers)]).contiguous()
+        vn = torch.stack([torch.cat([wl.kv_rows(w.seed, l, r, wl.KIND_V, int(w.context[r]), int(w.context[r]) + 1,
+                                                w.kv_heads, w.head_dim, w.dtype, self.dev) for r in self.reqs])
+                          for l in range(w.layers)]).contiguous()
+        out = torch.zeros_like(q)
+        if pinned:
+            return tuple(x.cpu().pin_memory() for x in (q, kn, vn, out))
+        return q, kn, vn, out
+
+    def step(self, i: int, q, kn, vn, out, tables=None):
+        """Step i from device buffers: the layers it touches, one C call, then the length commit."""
+        L = self.step_layers
+        l0 = (i * L) % self.w.layers
+        self.pool.decode_step(l0, L, self.w.q_heads, self.reqs_c, q[l0].data_ptr(), kn[l0].data_ptr(),
+                              vn[l0].data_ptr(), out[l0].data_ptr(), 0, self.stream, tables)
+        self.commit_none()
+
+    def commit_none(self):
+        """Every timed step repeats the SAME decode step (token `context` appended, context+1
+        keys attended), so that K steps measure one workload rather than a growing one: the
+        host-side length commit runs, with zero growth."""
+        rc = self.odma._lib.odma_commit_step(self.pool._h, self.reqs_c, self.w.batch, self.zeros_c)
+        assert rc == 0, rc
+
+    def step_host(self, i: int, hq, hkn, hvn, hout):
+        """Step i from pinned host buffers; the result is on the host when this returns."""
+        L = self.step_layers
+        l0 = (i * L) % self.w.layers
+        for l in range(l0, l0 + L):
+            self.pool.decode_step_host(l, self.w.q_heads, self.reqs_c, hq[l].data_ptr(), hkn[l].data_ptr(),
+                                       hvn[l].data_ptr(), hout[l].data_ptr(), self.stream)
+        torch.cuda.current_stream().synchronize()
+        self.commit_none()
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+_CLOCK_FIELDS = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+                 "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+                 "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+class ClockSampler:
+    """nvidia-smi in a child process, one CSV line every 50 ms, read-only queries."""
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False).name
+        self.f = open(self.path, "w")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={_CLOCK_FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        self.windows = []
+
+    def mark(self, t0: float, t1: float):
+        self.windows.append((t0, t1))
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.f.close()
+        from datetime import datetime
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 10:
+                continue
+            try:
+                ts = datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                mhz, mx = float(parts[2]), float(parts[3])
+            except ValueError:
+                continue
+            if not any(a - 0.05 <= ts <= b + 0.05 for a, b in self.windows):
+                continue
+            sm.append(mhz)
+            smax.append(mx)
+            for nm, val in zip(names, parts[6:10]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU checker legs (the only place this file touches oracle/)
+# ---------------------------------------------------------------------------------------------
+
+def _host_batch(w: wl.Workload, reqs, layer=0):
+    """(q, K list, V list) of the decode step of `reqs` on one layer, generated on the CPU."""
+    q = torch.stack([wl.q_rows(w.seed, layer, r, 0, w.q_heads, w.head_dim, w.dtype) for r in reqs])
+    Ks = [wl.kv_rows(w.seed, layer, r, wl.KIND_K, 0, int(w.context[r]) + 1, w.kv_heads, w.head_dim, w.dtype) for r in reqs]
+    Vs = [wl.kv_rows(w.seed, layer, r, wl.KIND_V, 0, int(w.context[r]) + 1, w.kv_heads, w.head_dim, w.dtype) for r in reqs]
+    return q, Ks, Vs
+
+
+def checker_sample(w: wl.Workload, step_layers: int, budget_s: float):
+    """Times the CPU checker on a bounded sample of the step: the first m requests of the
+    batch on one layer (requests are i.i.d., so any prefix has the batch's length law), with m
+    chosen from a one-request probe so that the sample takes about `budget_s` seconds."""
+    from oracle import oracle as ora
+    ora.build()
+    code = ora.dtype_code(w.dtype)
+    q, Ks, Vs = _host_batch(w, [0])
+    t0 = time.perf_counter()
+    _, _, threads = ora.decode_attention(q, Ks, Vs, w.q_heads, w.kv_heads, w.head_dim, code)
+    probe = max(time.perf_counter() - t0, 1e-6)
+    per_tok = probe / float(w.context[0] + 1)             # one request runs on one thread
+    total = np.cumsum(w.context + 1)
+    cores = os.cpu_count() or 1
+    m = int(np.searchsorted(total * per_tok / min(cores, w.batch), budget_s) + 1)
+    m = max(1, min(w.batch, m))
+    return m, threads
+
+
+def checker_time_step(w: wl.Workload, m: int, step_layers: int):
+    """One timed pass of the CPU checker over the first m requests (one layer); the step time
+    of the full workload's layer count is extrapolated by the caller."""
+    from oracle import oracle as ora
+    code = ora.dtype_code(w.dtype)
+    reqs = list(range(m))
+    q, Ks, Vs = _host_batch(w, reqs)
+    store = ora.KVStore(1, w.kv_heads, w.head_dim, code)
+    for r, k, v in zip(reqs, Ks, Vs):
+        store.append(r, 0, k[:-1], v[:-1])
+        store.gathered(r, 0)
+    t0 = time.perf_counter()
+    for r, k, v in zip(reqs, Ks, Vs):                      # the step's append ...
+        store.append(r, 0, k[-1:], v[-1:])
+    _, _, threads = store.decode_attention(0, reqs, q, w.q_heads)     # ... and attention
+    dt = time.perf_counter() - t0
+    return dt, threads
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU checker as it stands, on the host cores, same metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total = args.steps + args.warmup
+    w, step_layers, copies = pick_workload(args.workload)
+    per_step_budget = max(0.02, min(15.0, 150.0 / max(total, 1)))
+    m, _ = checker_sample(w, step_layers, per_step_budget)
+    times, threads = [], 0
+    for i in range(total):
+        dt, threads = checker_time_step(w, m, step_layers)
+        if i >= args.warmup:
+            times.append(dt)
+    t_step = sum(times) / len(times) * step_layers         # all stepped layers cost the same
+    value = m / t_step
+    sample = (f"first {m} of {w.batch} requests ({int((w.context[:m] + 1).sum())} of "
+              f"{int((w.context + 1).sum())} KV tokens), one layer timed"
+              + (f", x{step_layers} layers" if step_layers > 1 else ""))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, args.workload, step_layers, copies),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# the GPU arm
+# ---------------------------------------------------------------------------------------------
+
+def workload_config(w, name, step_layers, copies):
+    desc = {"config2": "configs[1]: Qwen-7B-shaped single layer, 28q/4kv heads, head_dim 128, bf16, batch 64, "
+                       "contexts lognormal(median 512, sigma 0.8) in [16,8192], quartile buckets",
+            "config3": "configs[2]: 28-layer Qwen-7B-shaped pool of 40 GB, batch 256, Pareto(1.5, 32) lengths, "
+                       "noisy predictions, 10% safety pool",
+            "config5": "configs[4]: long-reasoning decode, batch 32, contexts U[16384,32768], 28 layers"}[name]
+    kv_bytes_layer = int((w.context + 1).sum()) * 2 * w.kv_heads * w.head_dim * w.elem_bytes
+    return {"workload": desc, "batch": w.batch, "layers_per_step": step_layers,
+            "kv_tokens": int((w.context + 1).sum()), "kv_bytes_per_layer": kv_bytes_layer,
+            "l2": (f"steps rotate over {copies} independent KV copies ({copies * kv_bytes_layer >> 20} MiB > L2)"
+                   if copies > 1 else f"one step streams {step_layers * kv_bytes_layer >> 20} MiB of KV (> L2)")}
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    phases = set(args.phases.split(","))
+    K, W = args.steps, args.warmup
+    w, step_layers, copies = pick_workload(args.workload, rank, args.copies)
+    sd = SlabDecode(w, step_layers, dev)
+    bounds, epoch = sd.learn_boundaries()
+    sd.admit_and_fill()
+    q, kn, vn, out = sd.make_inputs()
+    torch.cuda.synchronize()
+
+    odma = sd.odma
+    tables = odma.Tables()
+    clocks = ClockSampler(local) if "clocks" in phases else None
+    peak, peak_kind = measured_peak()
+    row_bytes = w.head_dim * w.elem_bytes
+    n = w.batch
+    step_no = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # ---- warm-up, then exactly K timed steps -------------------------------------------------
+    for _ in range(W):
+        sd.step(step_no, q, kn, vn, out, tables)
+        step_no += 1
+    barrier()
+    t_wall0 = time.time()
+    ev0.record()
+    for _ in range(K):
+        sd.step(step_no, q, kn, vn, out, tables)
+        step_no += 1
+    ev1.record()
+    barrier()
+    if clocks:
+        clocks.mark(t_wall0, time.time())
+    ms = ev0.elapsed_time(ev1)
+    assert sd.pool.check_status(sd.stream) == odma.OK
+    launches_per_step = step_layers * (2 + (1 if tables.n_combine > 0 else 0))
+    kv_bytes_per_launch = tables.kv_tokens * 2 * w.kv_heads * row_bytes
+    step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes)
+
+    # ---- the same steps with every launch bracketed by CUDA events (per-kernel time) ----------
+    roofline, kernels_us = None, None
+    if "kernels" in phases:
+        prof_steps = max(3, min(K, 500))
+        sd.pool.profile_enable(True)
+        t0w = time.time()
+        for _ in range(prof_steps):
+            sd.step(step_no, q, kn, vn, out, tables)
+            step_no += 1
+        torch.cuda.synchronize()
+        if clocks:
+            clocks.mark(t0w, time.time())
+        dec_ms, dec_n = sd.pool.profile_read(odma.K_DECODE)
+        app_ms, app_n = sd.pool.profile_read(odma.K_APPEND)
+        cmb_ms, cmb_n = sd.pool.profile_read(odma.K_COMBINE)
+        sd.pool.profile_enable(False)
+        achieved = kv_bytes_per_launch / (dec_ms / dec_n * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": TRAFFIC.get(args.workload),
+                    "bytes_per_launch": kv_bytes_per_launch, "us_per_launch": dec_ms / dec_n * 1e3,
+                    "launches_timed": dec_n}
+        kernels_us = {"append": app_ms / max(app_n, 1) * 1e3, "decode": dec_ms / dec_n * 1e3,
+                      "combine": cmb_ms / cmb_n * 1e3 if cmb_n else 0.0}
+
+    # ---- end to end from pinned host buffers ---------------------------------------------------
+    e2e = None
+    if "e2e" in phases:
+        e2e_steps = max(3, min(K, 200))
+        hq, hkn, hvn, hout = sd.make_inputs(pinned=True)
+        for _ in range(3):
+            sd.step_host(step_no, hq, hkn, hvn, hout)
+            step_no += 1
+        barrier()
+        t0w = time.time()
+        ev0.record()
+        for _ in range(e2e_steps):
+            sd.step_host(step_no, hq, hkn, hvn, hout)
+            step_no += 1
+        ev1.record()
+        barrier()
+        if clocks:
+            clocks.mark(t0w, time.time())
+        e2e_ms = ev0.elapsed_time(ev1)
+        assert sd.pool.check_status(sd.stream) == odma.OK
+    else:
+        e2e_steps, e2e_ms = 1, float("nan")
+
+    # ---- if the timed passes were too short for the 50 ms sampler, repeat the same step under it
+    clk = None
+    if clocks:
+        if sum(b - a for a, b in clocks.windows) < 1.0:
+            t0w = time.time()
+            while time.time() - t0w < 1.2:
+                for _ in range(20):
+                    sd.step(step_no, q, kn, vn, out, tables)
+                    step_no += 1
+            torch.cuda.synchronize()
+            clocks.mark(t0w, time.time())
+        clk = clocks.stop()
+
+    # ---- max over ranks ------------------------------------------------------------------------
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, dev)
+    value = world * n * K / (ms * 1e-3)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+            "config": workload_config(w, args.workload, step_layers, copies),
+            "step_gbs": step_bytes / (ms / K * 1e-3) / 1e9,
+            "gpu_launches": int(launches_per_step * K),
+            "plan": {"ctas": tables.n_ctas, "items": tables.n_items, "combine": tables.n_combine},
+            "buckets": list(bounds), "migrations_at_fill": sd.migrations_at_fill}
+    if e2e_ms == e2e_ms:
+        h2d = step_layers * (n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes + tables.words * 4)
+        d2h = step_layers * n * w.q_heads * row_bytes
+        line["e2e"] = {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+                       "ms_per_step": e2e_ms / e2e_steps}
+    if roofline:
+        line["roofline"], line["kernels_us"] = roofline, kernels_us
+    if clk:
+        line["clocks"] = clk
+    if rank == 0 and world == 1 and "cpu" in phases:
+        m, _ = checker_sample(w, step_layers, 4.0)
+        dts = []
+        threads = 0
+        for _ in range(3):
+            dt, threads = checker_time_step(w, m, step_layers)
+            dts.append(dt)
+        t_step = min(dts) * step_layers
+        line["cpu_baseline"] = {"value": m / t_step, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"first {m} of {w.batch} requests, one layer, best of 3"
+                                          + (f", x{step_layers} layers" if step_layers > 1 else "")}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    t = torch.nan_to_num(t, nan=-1.0)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) if v >= 0 else float("nan") for v in t]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--phases", default="timed,kernels,e2e,clocks,cpu",
+                    help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
+                         "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline)")
+    ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

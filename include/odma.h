@@ -214,6 +214,18 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
                               int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
                               void* h_out, void* stream);
 
+/* The same step from DEVICE buffers, for n_layers consecutive layers starting at `layer`:
+ * builds the tables once into the pool's own table buffer, then for each layer appends one
+ * token per request and attends, all asynchronous on `stream`.  Buffers are layer-major:
+ * d_q, d_out [n_layers, n, q_heads, head_dim]; d_k_new, d_v_new [n_layers, n, kv_heads,
+ * head_dim]; lse device fp32 [n_layers, n, q_heads] or NULL.  tables_out (host, nullable)
+ * receives the description of the built batch; its d_table stays valid until the next
+ * odma_decode_step / odma_decode_step_host on this pool.  Does not commit lengths. */
+int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32_t q_heads,
+                         const uint64_t* reqs, int32_t n, const void* d_q, const void* d_k_new,
+                         const void* d_v_new, void* d_out, float* lse, void* stream,
+                         odma_tables* tables_out);
+
 /* Synchronises `stream` and returns the device status word as an error code (ODMA_OK,
  * ODMA_ERR_TIMEOUT, or ODMA_ERR_CUDA for a failed stream), clearing it. */
 int32_t odma_check_status(odma_pool* pool, void* stream);

@@ -527,6 +527,31 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
     return ODMA_OK;
 }
 
+int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32_t q_heads,
+                         const uint64_t* reqs, int32_t n, const void* d_q, const void* d_k_new,
+                         const void* d_v_new, void* d_out, float* lse, void* stream,
+                         odma_tables* tables_out) {
+    if (!pool || !pool->dev_base || !d_q || !d_k_new || !d_v_new || !d_out) return ODMA_ERR_INVALID;
+    if (n_layers < 1 || layer < 0 || layer + n_layers > pool->layers) return ODMA_ERR_INVALID;
+    odma_tables t;
+    int32_t rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
+                                   static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
+    if (rc != ODMA_OK) return rc;
+    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
+    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    for (int32_t l = 0; l < n_layers; ++l) {
+        rc = odma_append_kv(pool, layer + l, &t, static_cast<const uint8_t*>(d_k_new) + l * kb,
+                            static_cast<const uint8_t*>(d_v_new) + l * kb, stream);
+        if (rc != ODMA_OK) return rc;
+        rc = odma_decode_attention(pool, layer + l, static_cast<const uint8_t*>(d_q) + l * qb, q_heads, &t,
+                                   static_cast<uint8_t*>(d_out) + l * qb,
+                                   lse ? lse + static_cast<size_t>(l) * n * q_heads : nullptr, stream);
+        if (rc != ODMA_OK) return rc;
+    }
+    if (tables_out) *tables_out = t;
+    return ODMA_OK;
+}
+
 int32_t odma_check_status(odma_pool* pool, void* stream) {
     if (!pool || !pool->dev_base) return ODMA_ERR_INVALID;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return ODMA_ERR_CUDA;

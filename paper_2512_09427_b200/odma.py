@@ -82,6 +82,8 @@ _SIGS = {
     "odma_append_kv": (_i32, [_vp, _i32, C.POINTER(Tables), _vp, _vp, _vp]),
     "odma_decode_attention": (_i32, [_vp, _i32, _vp, _i32, C.POINTER(Tables), _vp, _vp, _vp]),
     "odma_decode_step_host": (_i32, [_vp, _i32, _i32, _u64p, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "odma_decode_step": (_i32, [_vp, _i32, _i32, _i32, _u64p, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                C.POINTER(Tables)]),
     "odma_check_status": (_i32, [_vp, _vp]),
     "odma_selftest_timeout": (_i32, [_vp, _i32, _vp]),
     "odma_read_probe": (_i32, [_vp, _i32, _i32, C.POINTER(Tables), _vp]),
@@ -180,8 +182,9 @@ class Pool:
     def free(self, req: int) -> int:
         return _lib.odma_free(self._h, req)
 
-    def commit_step(self, reqs: Sequence[int], n_new: Optional[Sequence[int]] = None) -> int:
-        return _lib.odma_commit_step(self._h, _u64arr(reqs), len(reqs), _i32arr(n_new))
+    def commit_step(self, reqs, n_new: Optional[Sequence[int]] = None) -> int:
+        arr = reqs if isinstance(reqs, C.Array) else _u64arr(reqs)
+        return _lib.odma_commit_step(self._h, arr, len(arr), _i32arr(n_new))
 
     def get_slab(self, req: int):
         s, ln = Slab(), C.c_int32()
@@ -228,6 +231,14 @@ class Pool:
         arr = reqs if isinstance(reqs, C.Array) else _u64arr(reqs)
         _check(_lib.odma_decode_step_host(self._h, layer, q_heads, arr, len(arr), h_q, h_k_new, h_v_new,
                                           h_out, stream or None), "odma_decode_step_host")
+
+    def decode_step(self, layer: int, n_layers: int, q_heads: int, reqs, d_q: int, d_k_new: int,
+                    d_v_new: int, d_out: int, lse: int = 0, stream: int = 0,
+                    tables: Optional[Tables] = None) -> None:
+        arr = reqs if isinstance(reqs, C.Array) else _u64arr(reqs)
+        _check(_lib.odma_decode_step(self._h, layer, n_layers, q_heads, arr, len(arr), d_q, d_k_new,
+                                     d_v_new, d_out, lse or None, stream or None,
+                                     C.byref(tables) if tables is not None else None), "odma_decode_step")
 
     def check_status(self, stream: int = 0) -> int:
         return _lib.odma_check_status(self._h, stream or None)
