@@ -77,7 +77,8 @@ def pick_workload(name: str, rank: int = 0, copies_override: int = 0):
 class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
-    def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0):
+    def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0,
+                 per_sm: int = 1, fused: int = 1):
         from paper_2512_09427_b200 import odma
         self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
         self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
@@ -91,6 +92,7 @@ class SlabDecode:
         cfg.p_den = pd
         cfg.max_batch = max(1024, w.batch)
         cfg.plan_ctas = plan_ctas
+        cfg.ctas_per_sm, cfg.fused_combine = per_sm, fused
         self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
         self.stream = torch.cuda.current_stream().cuda_stream
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,

@@ -83,8 +83,13 @@ typedef struct odma_config {
     int32_t large_fixed;     /* 1: every Large Bucket slab has max_len tokens (0) */
     int32_t max_batch;       /* most requests per odma_build_tables call; sizes scratch (1024) */
     int32_t max_group;       /* most query heads per KV head; sizes scratch (8) */
-    int32_t plan_ctas;       /* persistent CTAs the split plan targets; 0 = one per SM of the
-                                current device (148 when the pool has no device memory) */
+    int32_t plan_ctas;       /* persistent CTAs the split plan targets; 0 = ctas_per_sm per SM of
+                                the current device (148 SMs when the pool has no device memory) */
+    int32_t ctas_per_sm;     /* CTAs of the decode kernel resident on one SM: 1 or 2; sets the
+                                depth of each CTA's staging pipeline (1) */
+    int32_t fused_combine;   /* 1: the CTA that delivers the last piece of a split stream merges
+                                the pieces inside the decode kernel; 0: a separate combine kernel
+                                is launched after it (1) */
 } odma_config;
 
 typedef struct odma_slab {
@@ -108,15 +113,20 @@ typedef struct odma_stats {
 /* Host-side description of one built batch (plain data, owned by the caller).  The device
  * table it points to holds int32 words:
  *   base[n], cap[n], len[n] (length AFTER this step's append), cu_new[n+1] (prefix sum of
- *   the tokens appended this step), cta_begin[n_ctas+1], items[n_items][8], combine[n_combine][4].
- *   item    = {request, kv_head, first_token, n_tokens, direct(1)|partial(0), slot, 0, 0}
+ *   the tokens appended this step), cta[n_ctas][12], items[n_items][8], combine[n_combine][4].
+ *   cta     = {item_begin, item_end, 0, 0, copy of items[item_begin]}: CTA c works through
+ *             items [item_begin, item_end)
+ *   item    = {request, kv_head, first_token, n_tokens, direct(1)|partial(0), slot,
+ *              first row of the piece inside one K/V array, combine record (-1 if direct)}
  *   combine = {request, kv_head, first_slot, n_slots}
  * The off_* fields are word offsets of those arrays inside d_table. */
 typedef struct odma_tables {
     void* d_table;
     int32_t n, n_new_total, n_items, n_ctas, n_combine, words;
-    int32_t off_base, off_cap, off_len, off_cu_new, off_cta_begin, off_items, off_combine;
+    int32_t off_base, off_cap, off_len, off_cu_new, off_cta, off_items, off_combine;
     int32_t tile_tokens;
+    int32_t one_new_each; /* 1 when every request appends exactly one token (decode step) */
+    int32_t reserved;
     int64_t kv_tokens; /* sum of len */
     uint64_t epoch;
 } odma_tables;

@@ -40,6 +40,7 @@ struct odma_pool {
     int32_t layers = 0, kv_heads = 0, head_dim = 0, dtype = 0, elem_bytes = 0;
     int64_t rows_per_array = 0;
     int32_t plan_ctas = 148;
+    uint32_t* d_counters = nullptr;   // per split stream: pieces delivered (fused combine)
     int64_t slots_max = 0;
     int64_t table_words_max = 0;
     bool has_maps = false;
@@ -135,6 +136,7 @@ void free_device_side(odma_pool* p) {
     cudaFree(p->part_o);
     cudaFree(p->part_ml);
     cudaFree(p->d_status);
+    cudaFree(p->d_counters);
     cudaFree(p->d_q);
     cudaFree(p->d_k_new);
     cudaFree(p->d_v_new);
@@ -200,8 +202,10 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->base = tab + t->off_base;
     p->cap = tab + t->off_cap;
     p->len = tab + t->off_len;
-    p->cta_begin = tab + t->off_cta_begin;
+    p->cta = reinterpret_cast<const int4*>(tab + t->off_cta);
     p->items = reinterpret_cast<const int4*>(tab + t->off_items);
+    p->combine = reinterpret_cast<const int4*>(tab + t->off_combine);
+    p->counters = pool->alloc.config().fused_combine ? pool->d_counters : nullptr;
     p->q = q;
     p->out = out;
     p->lse = lse;
@@ -213,6 +217,7 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->q_heads = q_heads;
     p->kv_heads = pool->kv_heads;
     p->group = q_heads / pool->kv_heads;
+    p->stages = tc_stages(pool->head_dim, p->group, pool->alloc.config().ctas_per_sm);
     p->head_dim = pool->head_dim;
     p->scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(pool->head_dim)));
     p->status = pool->d_status;
@@ -253,6 +258,8 @@ void odma_config_default(odma_config* cfg) {
     cfg->max_batch = 1024;
     cfg->max_group = 8;
     cfg->plan_ctas = 0;
+    cfg->ctas_per_sm = 1;
+    cfg->fused_combine = 1;
 }
 
 const char* odma_strerror(int32_t code) {
@@ -280,6 +287,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
     if (layers < 1 || kv_heads < 1 || head_dim < 1 || (static_cast<int64_t>(head_dim) * esz) % 16 != 0)
         return ODMA_ERR_INVALID;
     if (cfg.max_batch < 1 || cfg.max_group < 1 || cfg.plan_ctas < 0) return ODMA_ERR_INVALID;
+    if (cfg.ctas_per_sm < 1 || cfg.ctas_per_sm > 2) return ODMA_ERR_INVALID;
     if (dev_base && (reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0) return ODMA_ERR_INVALID;
 
     odma_pool* p = new (std::nothrow) odma_pool();
@@ -301,7 +309,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
         delete p;
         return ODMA_ERR_INVALID;
     }
-    p->plan_ctas = cfg.plan_ctas > 0 ? cfg.plan_ctas : 148;
+    p->plan_ctas = cfg.plan_ctas > 0 ? cfg.plan_ctas : 148 * cfg.ctas_per_sm;
     if (dev_base) {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -309,7 +317,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
             delete p;
             return ODMA_ERR_CUDA;
         }
-        if (cfg.plan_ctas == 0) p->plan_ctas = sms;
+        if (cfg.plan_ctas == 0) p->plan_ctas = sms * cfg.ctas_per_sm;
     }
     p->slots_max = static_cast<int64_t>(cfg.max_batch) * kv_heads + p->plan_ctas;
     p->table_words_max = plan_table_words(cfg.max_batch, kv_heads, p->plan_ctas);
@@ -320,6 +328,8 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
         const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * esz;
         bool ok = cudaMalloc(&p->part_o, po) == cudaSuccess && cudaMalloc(&p->part_ml, pm) == cudaSuccess &&
                   cudaMalloc(&p->d_status, 4) == cudaSuccess && cudaMalloc(&p->d_q, qb) == cudaSuccess &&
+                  cudaMalloc(&p->d_counters, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
+                  cudaMemset(p->d_counters, 0, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
                   cudaMalloc(&p->d_out, qb) == cudaSuccess && cudaMalloc(&p->d_k_new, kb) == cudaSuccess &&
                   cudaMalloc(&p->d_v_new, kb) == cudaSuccess &&
                   cudaMalloc(&p->d_step_table, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
@@ -468,6 +478,7 @@ int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables
     ap.kv_heads = pool->kv_heads;
     ap.n_new_total = tables->n_new_total;
     ap.row_vecs = pool->head_dim * pool->elem_bytes / 16;
+    ap.one_new_each = tables->one_new_each;
     ProfScope ps(pool, ODMA_K_APPEND, as_stream(stream));
     return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
@@ -479,17 +490,22 @@ int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int
     DecodeParams p;
     fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
     cudaError_t e;
+    bool fused = false;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
-        if (pool->has_maps && tc_supported(pool->head_dim, p.group))
+        if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
+            if (p.stages < 2) return ODMA_ERR_INVALID;
+            fused = p.counters != nullptr;
             e = launch_decode_tc(pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream));
-        else if (generic_supported(pool->head_dim))
+        } else if (generic_supported(pool->head_dim)) {
+            p.counters = nullptr;
             e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
-        else
+        } else {
             return ODMA_ERR_INVALID;
+        }
     }
     if (e != cudaSuccess) return ODMA_ERR_CUDA;
-    if (tables->n_combine > 0) {
+    if (tables->n_combine > 0 && !fused) {
         ProfScope ps(pool, ODMA_K_COMBINE, as_stream(stream));
         const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
         e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,
@@ -557,7 +573,12 @@ int32_t odma_check_status(odma_pool* pool, void* stream) {
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return ODMA_ERR_CUDA;
     uint32_t word = 0;
     if (cudaMemcpy(&word, pool->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return ODMA_ERR_CUDA;
-    if (word != 0 && cudaMemset(pool->d_status, 0, 4) != cudaSuccess) return ODMA_ERR_CUDA;
+    if (word != 0) {
+        // a kernel that gave up may have left split streams half counted
+        if (cudaMemset(pool->d_status, 0, 4) != cudaSuccess ||
+            cudaMemset(pool->d_counters, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess)
+            return ODMA_ERR_CUDA;
+    }
     return (word & kStatusTimeout) ? ODMA_ERR_TIMEOUT : ODMA_OK;
 }
 
@@ -571,7 +592,7 @@ int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const o
     DecodeParams p;
     // the probe moves the query bytes too; any valid device memory of that size will do
     fill_decode_params(pool, layer, pool->d_q, q_heads, tables, pool->d_out, nullptr, &p);
-    if (!tc_supported(pool->head_dim, p.group) || p.group > pool->alloc.config().max_group)
+    if (!tc_supported(pool->head_dim, p.group) || p.group > pool->alloc.config().max_group || p.stages < 2)
         return ODMA_ERR_INVALID;
     ProfScope ps(pool, ODMA_K_PROBE, as_stream(stream));
     return launch_decode_tc(pool->maps, p, kModeProbe, tables->n_ctas, as_stream(stream)) == cudaSuccess
@@ -726,7 +747,7 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
     if (rc != ODMA_OK) return rc;
     DecodeParams p;
     fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
-    if (!tc_supported(pool->head_dim, p.group)) return ODMA_ERR_INVALID;
+    if (!tc_supported(pool->head_dim, p.group) || p.stages < 2) return ODMA_ERR_INVALID;
     p.pool = paged->d_pages;
     p.rows_per_array = paged->n_pages * pool->kv_heads * 16;
     p.page_table = d_page_table;
@@ -737,7 +758,7 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
         e = launch_decode_tc(paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream));
     }
     if (e != cudaSuccess) return ODMA_ERR_CUDA;
-    if (tables->n_combine > 0) {
+    if (tables->n_combine > 0 && p.counters == nullptr) {
         ProfScope ps(pool, ODMA_K_COMBINE, as_stream(stream));
         const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
         e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,

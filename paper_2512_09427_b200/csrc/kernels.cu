@@ -14,7 +14,11 @@
 
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "odma.h"
+
+#pragma nv_diag_suppress 128   // the probe instantiation leaves the merge code unreachable
 
 namespace odma {
 namespace {
@@ -139,37 +143,97 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // keys and 64 values of one stream, written by TMA with the 128-byte swizzle so that ldmatrix
 // reads are conflict-free.  Consumer warp w owns keys [16w, 16w+16) of every tile and keeps its
 // own running (max, sum, output); the four are merged through shared memory when the item ends.
-// The query heads of the group are the M rows of the MMA tiles (rows >= group are zero).
+//
+// The contraction is arranged with the KEYS on the M side of the MMA tiles and the query heads
+// of the GQA group on the N side (8 heads per n-tile, rows >= group are zero):
+//     S^T[16 keys x 8 heads]  = K[16 keys x D]   . Q^T[D x 8 heads]
+//     O^T[D x 8 heads]       += V^T[D x 16 keys] . P^T[16 keys x 8 heads]
+// so a group of 7 heads wastes one column in eight instead of nine rows in sixteen, and the
+// softmax weights go from the first product's accumulator to the second product's B operand
+// with one 8x8 register transpose (movmatrix) per eight keys.
 
 constexpr int kConsumerWarps = 4;
-constexpr int kTcThreads = (kConsumerWarps + 1) * 32;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kTcThreads = kConsumerThreads + 32;
 constexpr int kTile = 64;
+constexpr int kMaxStages = 8;
 
-template <int D, bool HI>
+template <int D, int NT>
 struct TcConfig {
-    static constexpr int kRows = HI ? 16 : 8;
+    static constexpr int kRows = NT * 8;
     static constexpr int kKvTileBytes = kTile * D * 2;
     static constexpr int kStageBytes = 2 * kKvTileBytes;
-    static constexpr int kQBytes = 16 * D * 2;
-    static constexpr int kMoStride = D + 8;
-    static constexpr int kMergeBytes = kConsumerWarps * kRows * (kMoStride + 2) * 4;
-    static constexpr int kFixedBytes = 2 * kQBytes + kMergeBytes + 64 /*desc*/ + 256 /*barriers*/;
-    static constexpr int kBudget = 227 * 1024 - 1024 /*alignment slack*/;
-    static constexpr int kStagesFit = (kBudget - kFixedBytes) / kStageBytes;
-    static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kFixedBytes + 1024;
+    static constexpr int kQBytes = kRows * D * 2;
+    static constexpr int kMoStride = D + 4;
+    static constexpr int kMergeFloats = kConsumerWarps * kRows * kMoStride;
+    static constexpr int kMlFloats = kConsumerWarps * kRows * 2;
+    static constexpr int kFixedBytes =
+        2 * kQBytes + (kMergeFloats + kMlFloats) * 4 + 2 * 8 * 4 /*desc*/ + (2 * kMaxStages + 8) * 8 /*barriers*/ + 64;
+    static constexpr int kAlignSlack = 1024;
+    static int smem_bytes(int stages) { return stages * kStageBytes + kFixedBytes + kAlignSlack; }
 };
 
-template <int D, bool HI, int MODE>
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+
+__device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float c, float d) {
+    *reinterpret_cast<uint2*>(p) = make_uint2(pack_bf16(a, b), pack_bf16(c, d));
+}
+
+// Log-sum-exp merge of the `ns` partial results of one (request, KV head) stream, slots
+// [slot0, slot0+ns): out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), M = max_s m_s.
+// Thread `tid` of `nthreads` takes two groups of four output elements of one query head.
+// Partials are read through L2 (they may have been written by other SMs a moment ago).
+template <typename T>
+__device__ __forceinline__ void combine_stream(const float* part_o, const float* part_ml, int slot0,
+                                               int ns, int req, int head, int group, int D,
+                                               int q_heads, T* out, float* lse, int tid, int nthreads) {
+    const int per_row = D >> 3;
+    for (int idx = tid; idx < group * per_row; idx += nthreads) {
+        const int r = idx / per_row, c = idx - r * per_row;
+        const int d0 = c * 4, d1 = (D >> 1) + c * 4;
+        float M = -INFINITY;
+#pragma unroll 4
+        for (int s = 0; s < ns; ++s)
+            M = fmaxf(M, __ldcg(part_ml + (static_cast<size_t>(slot0 + s) * group + r) * 2));
+        float L = 0.f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll 2
+        for (int s = 0; s < ns; ++s) {
+            const size_t prow = static_cast<size_t>(slot0 + s) * group + r;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(part_ml + prow * 2));
+            const float e = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+            const float4 x = ldcg4(part_o + prow * D + d0), y = ldcg4(part_o + prow * D + d1);
+            L = fmaf(ml.y, e, L);
+            a.x = fmaf(x.x, e, a.x); a.y = fmaf(x.y, e, a.y); a.z = fmaf(x.z, e, a.z); a.w = fmaf(x.w, e, a.w);
+            b.x = fmaf(y.x, e, b.x); b.y = fmaf(y.y, e, b.y); b.z = fmaf(y.z, e, b.z); b.w = fmaf(y.w, e, b.w);
+        }
+        const float inv = 1.f / L;
+        const size_t row = static_cast<size_t>(req) * q_heads + static_cast<size_t>(head) * group + r;
+        store4(out + row * D + d0, a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+        store4(out + row * D + d1, b.x * inv, b.y * inv, b.z * inv, b.w * inv);
+        if (c == 0 && lse) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+    }
+}
+
+template <int D, int NT, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                  const __grid_constant__ CUtensorMap tm_small, const DecodeParams p) {
-    using Cfg = TcConfig<D, HI>;
-    constexpr int STAGES = Cfg::kStages;
+    using Cfg = TcConfig<D, NT>;
     constexpr int ROWS = Cfg::kRows;
     constexpr int HALVES = D / 64;                 // 128-byte column blocks per row
     constexpr int HALF_BYTES = kTile * 128;
-    constexpr int MO_STRIDE = Cfg::kMoStride;
+    constexpr int MO = Cfg::kMoStride;
+    const int STAGES = p.stages;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
@@ -177,23 +241,38 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     uint8_t* kv = smem;
     uint8_t* qbuf = kv + STAGES * Cfg::kStageBytes;
     float* mrg_o = reinterpret_cast<float*>(qbuf + 2 * Cfg::kQBytes);
-    float* mrg_ml = mrg_o + kConsumerWarps * ROWS * MO_STRIDE;
-    int* desc = reinterpret_cast<int*>(mrg_ml + kConsumerWarps * ROWS * 2);
+    float* mrg_ml = mrg_o + Cfg::kMergeFloats;
+    int* desc = reinterpret_cast<int*>(mrg_ml + Cfg::kMlFloats);
     uint64_t* bars = reinterpret_cast<uint64_t*>(desc + 16);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 6);
+    volatile int* flags = reinterpret_cast<volatile int*>(bars + 2 * kMaxStages + 8);
+    volatile int* abort_flag = flags;            // flags[0]: a wait timed out somewhere in the CTA
+    volatile int* last_flag = flags + 1;         // flags[1]: this CTA completes a split stream
 
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (STAGES + s); };
-    auto qfull_bar = [&](uint32_t s) { return bar0 + 8u * (2 * STAGES + s); };
-    auto qempty_bar = [&](uint32_t s) { return bar0 + 8u * (2 * STAGES + 2 + s); };
-    const uint32_t mready_bar = bar0 + 8u * (2 * STAGES + 4);
-    const uint32_t mdone_bar = bar0 + 8u * (2 * STAGES + 5);
+    auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kMaxStages + s); };
+    auto qfull_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + s); };
+    auto qempty_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 + s); };
+    const uint32_t mready_bar = bar0 + 8u * (2 * kMaxStages + 4);
+    const uint32_t mdone_bar = bar0 + 8u * (2 * kMaxStages + 5);
+    const uint32_t cfence_bar = bar0 + 8u * (2 * kMaxStages + 6);
+    const uint32_t cflag_bar = bar0 + 8u * (2 * kMaxStages + 7);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int64_t limit = p.wait_limit_ns;
+    const int cta = blockIdx.x;
 
+    // the producer's first loads are in flight while the barriers are being set up
+    int4 rec = make_int4(0, 0, 0, 0), first_a = rec, first_b = rec;
+    if (tid == kConsumerThreads) {
+        const int4* r = p.cta + 3 * cta;
+        rec = __ldg(r);
+        first_a = __ldg(r + 1);
+        first_b = __ldg(r + 2);
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_big)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_small)) : "memory");
+    }
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
@@ -205,25 +284,27 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         }
         mbar_init(mready_bar, kConsumerWarps);
         mbar_init(mdone_bar, kConsumerWarps);
-        *abort_flag = 0;
+        mbar_init(cfence_bar, kConsumerWarps);
+        mbar_init(cflag_bar, kConsumerWarps);
+        flags[0] = 0;
+        flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // query rows >= group stay zero for the whole kernel; TMA only ever writes rows < group
+    // query rows >= group stay zero for the whole kernel; the bulk copy only writes rows < group
     for (int i = tid; i < 2 * Cfg::kQBytes / 16; i += kTcThreads)
         reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
 
-    const int cta = blockIdx.x;
-    const int it_begin = p.cta_begin[cta], it_end = p.cta_begin[cta + 1];
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
+            const int it_begin = rec.x, it_end = rec.y;
             uint32_t stage = 0, phase = 0;
-            uint32_t issued[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // loads issued per stage (drain on abort)
+            uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
             bool ok = true;
             const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
             const int64_t v_array = k_array + p.rows_per_array;
@@ -234,32 +315,32 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 if (!ok) break;
                 int* dsc = desc + qs * 8;
                 if (it >= it_end) {                      // end marker
-                    dsc[3] = 0;
+                    dsc[2] = 0;
                     mbar_arrive(qfull_bar(qs));
                     break;
                 }
-                const int4 a = p.items[2 * it], b = p.items[2 * it + 1];
+                int4 a = first_a, b = first_b;
+                if (it != it_begin) {
+                    a = __ldg(p.items + 2 * it);
+                    b = __ldg(p.items + 2 * it + 1);
+                }
                 const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
                 dsc[0] = req;
                 dsc[1] = head;
-                dsc[2] = tok0;
-                dsc[3] = ntok;
-                dsc[4] = b.x;
-                dsc[5] = b.y;
+                dsc[2] = ntok;
+                dsc[3] = b.x;     // direct
+                dsc[4] = b.y;     // slot
+                dsc[5] = b.w;     // combine record
                 const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
                 mbar_expect_tx(qfull_bar(qs), q_bytes);
                 bulk_load(q_u32 + qs * Cfg::kQBytes,
                           static_cast<const uint8_t*>(p.q) +
                               (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
                           q_bytes, qfull_bar(qs));
-                int64_t row = 0;
+                const int64_t row = b.z;
                 const int32_t* pages = nullptr;
-                if (MODE == kModePaged) {
+                if (MODE == kModePaged)
                     pages = p.page_table + static_cast<size_t>(req) * p.max_pages + tok0 / 16;
-                } else {
-                    row = static_cast<int64_t>(p.base[req]) * p.kv_heads +
-                          static_cast<int64_t>(head) * p.cap[req] + tok0;
-                }
                 const int ntiles = (ntok + kTile - 1) / kTile;
                 for (int t = 0; t < ntiles; ++t) {
                     ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit);
@@ -299,8 +380,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                             }
                         }
                     }
-                    issued[stage] += 1;
-                    if (++stage == STAGES) {
+                    issued_any |= 1u << stage;
+                    issued_odd ^= 1u << stage;
+                    if (++stage == static_cast<uint32_t>(STAGES)) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -310,8 +392,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 // Something timed out.  Before the CTA's shared memory can be handed to another
                 // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
                 for (int s = 0; s < STAGES; ++s)
-                    if (issued[s])
-                        mbar_wait_slow(full_bar(s), (issued[s] - 1u) & 1u, nullptr, p.status,
+                    if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
+                        mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
                                        limit / 4 + 1);
             }
         }
@@ -322,38 +404,55 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     // ---------------------------------------------------------------------- consumers
     const int qd = lane >> 2, qt = lane & 3;          // row within 8, position within the quad
     const int mi = lane >> 3, r8 = lane & 7;          // ldmatrix: matrix id, row within it
-    const uint32_t k_lane_off = (warp * 16 + (mi >> 1) * 8 + r8) * 128;
-    const uint32_t xk = (mi & 1) ^ r8;
-    const uint32_t v_lane_off = (warp * 16 + (mi & 1) * 8 + r8) * 128;
-    const uint32_t xv = (mi >> 1) ^ r8;
-    const uint32_t q_lane_off = ((mi & 1) * 8 + r8) * (D * 2) + (mi >> 1) * 16;
-    const int kidx0 = warp * 16 + qt * 2;             // first of this thread's key columns
+    // K tile as the A operand: matrices (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15)
+    const uint32_t k_lane_off = (warp * 16 + (mi & 1) * 8 + r8) * 128;
+    const uint32_t xk = (mi >> 1) ^ r8;
+    // V tile, transposed on load, as the A operand: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
+    const uint32_t v_lane_off = (warp * 16 + (mi >> 1) * 8 + r8) * 128;
+    const uint32_t xv = (mi & 1) ^ r8;
+    // Q as the B operand: four consecutive 16-byte chunks of head r8
+    const uint32_t q_lane_off = r8 * (D * 2) + mi * 16;
+    const int key_lo = warp * 16 + qd;                // the thread's two key rows: key_lo, key_lo + 8
+    const int vkey0 = warp * 16 + qt * 2;             // keys of its value fragments: vkey0, +1, +8, +9
     const float scale = p.scale_log2;
     const int group = p.group;
 
-    uint32_t stage = 0, phase = 0;
+    uint32_t stage = 0, phase = 0, n_split = 0;
     bool ok = true;
     for (uint32_t k_item = 0; ok; ++k_item) {
         const uint32_t qs = k_item & 1u;
         ok = mbar_wait(qfull_bar(qs), (k_item >> 1) & 1u, abort_flag, p.status, limit);
         if (!ok) break;
         const int* dsc = desc + qs * 8;
-        const int req = dsc[0], head = dsc[1], ntok = dsc[3], direct = dsc[4], slot = dsc[5];
+        const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3], slot = dsc[4], comb = dsc[5];
         if (ntok == 0) break;
 
-        uint32_t qa[D / 16][4];
+        uint32_t qb[NT][D / 16][2];
         if (MODE != kModeProbe) {
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk)
-                ldmatrix_x4(qa[kk], q_u32 + qs * Cfg::kQBytes + q_lane_off + kk * 32);
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int j = 0; j < D / 32; ++j) {
+                    uint32_t r[4];
+                    ldmatrix_x4(r, q_u32 + qs * Cfg::kQBytes + nt * 8 * (D * 2) + q_lane_off + j * 64);
+                    qb[nt][2 * j][0] = r[0];
+                    qb[nt][2 * j][1] = r[1];
+                    qb[nt][2 * j + 1][0] = r[2];
+                    qb[nt][2 * j + 1][1] = r[3];
+                }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(qempty_bar(qs));
 
-        float o[D / 8][4];
+        float o[NT][D / 16][4];
+        float m_run[NT][2], l_run[NT][2];
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-        float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+            for (int i = 0; i < D / 16; ++i) o[nt][i][0] = o[nt][i][1] = o[nt][i][2] = o[nt][i][3] = 0.f;
+            m_run[nt][0] = m_run[nt][1] = -INFINITY;
+            l_run[nt][0] = l_run[nt][1] = 0.f;
+        }
 
         const int ntiles = (ntok + kTile - 1) / kTile;
         for (int t = 0; t < ntiles; ++t) {
@@ -363,93 +462,87 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             if (MODE != kModeProbe && warp * 16 < valid) {
                 const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
                 const uint32_t vbase = kbase + Cfg::kKvTileBytes;
-                // ---- S = Q K^T for this warp's 16 keys (two n-tiles of 8 keys)
-                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                // ---- S^T = K Q^T for this warp's 16 keys; two accumulators shorten the chain
+                float s[NT][4], s2[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) s[nt][i] = s2[nt][i] = 0.f;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    uint32_t b[4];
-                    ldmatrix_x4(b, kbase + (kk >> 2) * HALF_BYTES + k_lane_off +
-                                       ((((kk & 3) * 2) ^ xk) << 4));
-                    mma_bf16(s0, qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[0], b[1]);
-                    mma_bf16(s1, qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[2], b[3]);
+                    uint32_t a[4];
+                    ldmatrix_x4(a, kbase + (kk >> 2) * HALF_BYTES + k_lane_off + ((((kk & 3) * 2) ^ xk) << 4));
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        if (kk & 1)
+                            mma_bf16(s2[nt], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
+                        else
+                            mma_bf16(s[nt], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
+                    }
                 }
                 // ---- keys at or beyond the item's end: scores are selected to -inf (never
                 //      added to), value rows are zeroed in registers below
-                uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
                 const bool ragged = valid < kTile;
+                const bool in_lo = key_lo < valid, in_hi = key_lo + 8 < valid;
+                uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
                 if (ragged) {
-                    const bool in0 = kidx0 < valid, in1 = kidx0 + 1 < valid;
-                    const bool in8 = kidx0 + 8 < valid, in9 = kidx0 + 9 < valid;
-                    if (!in0) s0[0] = s0[2] = -INFINITY;
-                    if (!in1) s0[1] = s0[3] = -INFINITY;
-                    if (!in8) s1[0] = s1[2] = -INFINITY;
-                    if (!in9) s1[1] = s1[3] = -INFINITY;
-                    vm0 = (in0 ? 0x0000FFFFu : 0u) | (in1 ? 0xFFFF0000u : 0u);
-                    vm1 = (in8 ? 0x0000FFFFu : 0u) | (in9 ? 0xFFFF0000u : 0u);
+                    vm0 = (vkey0 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 1 < valid ? 0xFFFF0000u : 0u);
+                    vm1 = (vkey0 + 8 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 9 < valid ? 0xFFFF0000u : 0u);
                 }
-                // ---- online softmax, fp32, row max shared across the quad by shuffles
-                uint32_t pa0, pa1 = 0u, pa2, pa3 = 0u;
-                {
-                    float mx = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-                    const float m_new = fmaxf(m_lo, mx * scale);
-                    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                    const float corr = exp2f(m_lo - m_use);
-                    const float p0 = exp2f(fmaf(s0[0], scale, -m_use));
-                    const float p1 = exp2f(fmaf(s0[1], scale, -m_use));
-                    const float p2 = exp2f(fmaf(s1[0], scale, -m_use));
-                    const float p3 = exp2f(fmaf(s1[1], scale, -m_use));
-                    l_lo = fmaf(l_lo, corr, (p0 + p1) + (p2 + p3));
-                    m_lo = m_new;
+                // ---- online softmax, fp32; a head's maximum is shared by the eight lanes that
+                //      hold its keys (shuffles over the lane bits that select the key row)
+                uint32_t pb[NT][2];
 #pragma unroll
-                    for (int i = 0; i < D / 8; ++i) {
-                        o[i][0] *= corr;
-                        o[i][1] *= corr;
+                for (int nt = 0; nt < NT; ++nt) {
+                    float c0 = s[nt][0] + s2[nt][0], c1 = s[nt][1] + s2[nt][1];
+                    float c2 = s[nt][2] + s2[nt][2], c3 = s[nt][3] + s2[nt][3];
+                    if (!in_lo) c0 = c1 = -INFINITY;
+                    if (!in_hi) c2 = c3 = -INFINITY;
+                    float mx0 = fmaxf(c0, c2), mx1 = fmaxf(c1, c3);
+#pragma unroll
+                    for (int off = 4; off < 32; off <<= 1) {
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, off));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, off));
                     }
-                    pa0 = pack_bf16(p0, p1);
-                    pa2 = pack_bf16(p2, p3);
-                }
-                if (HI) {
-                    float mx = fmaxf(fmaxf(s0[2], s0[3]), fmaxf(s1[2], s1[3]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-                    const float m_new = fmaxf(m_hi, mx * scale);
-                    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                    const float corr = exp2f(m_hi - m_use);
-                    const float p0 = exp2f(fmaf(s0[2], scale, -m_use));
-                    const float p1 = exp2f(fmaf(s0[3], scale, -m_use));
-                    const float p2 = exp2f(fmaf(s1[2], scale, -m_use));
-                    const float p3 = exp2f(fmaf(s1[3], scale, -m_use));
-                    l_hi = fmaf(l_hi, corr, (p0 + p1) + (p2 + p3));
-                    m_hi = m_new;
+                    const float mn0 = fmaxf(m_run[nt][0], mx0 * scale), mn1 = fmaxf(m_run[nt][1], mx1 * scale);
+                    const float mu0 = (mn0 == -INFINITY) ? 0.f : mn0, mu1 = (mn1 == -INFINITY) ? 0.f : mn1;
+                    const float corr0 = exp2f(m_run[nt][0] - mu0), corr1 = exp2f(m_run[nt][1] - mu1);
+                    const float p0 = exp2f(fmaf(c0, scale, -mu0)), p1 = exp2f(fmaf(c1, scale, -mu1));
+                    const float p2 = exp2f(fmaf(c2, scale, -mu0)), p3 = exp2f(fmaf(c3, scale, -mu1));
+                    l_run[nt][0] = fmaf(l_run[nt][0], corr0, p0 + p2);
+                    l_run[nt][1] = fmaf(l_run[nt][1], corr1, p1 + p3);
+                    m_run[nt][0] = mn0;
+                    m_run[nt][1] = mn1;
 #pragma unroll
-                    for (int i = 0; i < D / 8; ++i) {
-                        o[i][2] *= corr;
-                        o[i][3] *= corr;
+                    for (int i = 0; i < D / 16; ++i) {
+                        o[nt][i][0] *= corr0;
+                        o[nt][i][1] *= corr1;
+                        o[nt][i][2] *= corr0;
+                        o[nt][i][3] *= corr1;
                     }
-                    pa1 = pack_bf16(p0, p1);
-                    pa3 = pack_bf16(p2, p3);
+                    // P[key][head] -> P^T fragments: (head qd; keys 2qt, 2qt+1) and (+8, +9)
+                    pb[nt][0] = movmatrix_trans(pack_bf16(p0, p1));
+                    pb[nt][1] = movmatrix_trans(pack_bf16(p2, p3));
                 }
-                // ---- O += P V
+                // ---- O^T += V^T P^T
 #pragma unroll
-                for (int jj = 0; jj < D / 16; ++jj) {
-                    uint32_t b[4];
-                    ldmatrix_x4_trans(b, vbase + (jj >> 2) * HALF_BYTES + v_lane_off +
-                                             ((((jj & 3) * 2) ^ xv) << 4));
+                for (int dt = 0; dt < D / 16; ++dt) {
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, vbase + (dt >> 2) * HALF_BYTES + v_lane_off + ((((dt & 3) * 2) ^ xv) << 4));
                     if (ragged) {
-                        b[0] &= vm0;
-                        b[1] &= vm1;
-                        b[2] &= vm0;
-                        b[3] &= vm1;
+                        a[0] &= vm0;
+                        a[1] &= vm0;
+                        a[2] &= vm1;
+                        a[3] &= vm1;
                     }
-                    mma_bf16(o[2 * jj], pa0, pa1, pa2, pa3, b[0], b[1]);
-                    mma_bf16(o[2 * jj + 1], pa0, pa1, pa2, pa3, b[2], b[3]);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        mma_bf16(o[nt][dt], a[0], a[1], a[2], a[3], pb[nt][0], pb[nt][1]);
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar(stage));
-            if (++stage == STAGES) {
+            if (++stage == static_cast<uint32_t>(STAGES)) {
                 stage = 0;
                 phase ^= 1u;
             }
@@ -458,68 +551,101 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         if (MODE == kModeProbe) continue;
 
         // ---- merge the four warps' partial results and write the item's result
-        l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 1);
-        l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 2);
-        if (HI) {
-            l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 1);
-            l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 2);
-        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                l_run[nt][0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][0], off);
+                l_run[nt][1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][1], off);
+            }
         if (k_item > 0) {
             ok = mbar_wait(mdone_bar, (k_item - 1u) & 1u, abort_flag, p.status, limit);
             if (!ok) break;
         }
-        float* mo = mrg_o + warp * ROWS * MO_STRIDE;
+        float* mo = mrg_o + warp * ROWS * MO;
         float* mml = mrg_ml + warp * ROWS * 2;
-        if (qd < group) {
 #pragma unroll
-            for (int i = 0; i < D / 8; ++i)
-                *reinterpret_cast<float2*>(mo + qd * MO_STRIDE + i * 8 + qt * 2) =
-                    make_float2(o[i][0], o[i][1]);
-            if (qt == 0) {
-                mml[qd * 2] = m_lo;
-                mml[qd * 2 + 1] = l_lo;
+        for (int nt = 0; nt < NT; ++nt) {
+            const int h0 = nt * 8 + qt * 2;
+#pragma unroll
+            for (int dt = 0; dt < D / 16; ++dt) {
+                const int d = dt * 16 + qd;
+                mo[h0 * MO + d] = o[nt][dt][0];
+                mo[(h0 + 1) * MO + d] = o[nt][dt][1];
+                mo[h0 * MO + d + 8] = o[nt][dt][2];
+                mo[(h0 + 1) * MO + d + 8] = o[nt][dt][3];
             }
-        }
-        if (HI && qd + 8 < group) {
-#pragma unroll
-            for (int i = 0; i < D / 8; ++i)
-                *reinterpret_cast<float2*>(mo + (qd + 8) * MO_STRIDE + i * 8 + qt * 2) =
-                    make_float2(o[i][2], o[i][3]);
-            if (qt == 0) {
-                mml[(qd + 8) * 2] = m_hi;
-                mml[(qd + 8) * 2 + 1] = l_hi;
+            if (qd == 0) {
+                mml[h0 * 2] = m_run[nt][0];
+                mml[h0 * 2 + 1] = l_run[nt][0];
+                mml[h0 * 2 + 2] = m_run[nt][1];
+                mml[h0 * 2 + 3] = l_run[nt][1];
             }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(mready_bar);
         ok = mbar_wait(mready_bar, k_item & 1u, abort_flag, p.status, limit);
         if (!ok) break;
-        for (int idx = tid; idx < group * D; idx += kConsumerWarps * 32) {
-            const int r = idx / D, d = idx - r * D;
+        constexpr int PER_ROW = D / 8;
+        for (int idx = tid; idx < group * PER_ROW; idx += kConsumerThreads) {
+            const int r = idx / PER_ROW, c = idx - r * PER_ROW;
+            const int d0 = c * 4, d1 = D / 2 + c * 4;
             float mw[kConsumerWarps], M = -INFINITY;
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w) {
                 mw[w] = mrg_ml[(w * ROWS + r) * 2];
                 M = fmaxf(M, mw[w]);
             }
-            float L = 0.f, O = 0.f;
+            float L = 0.f;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w) {
-                const float e = exp2f(mw[w] - M);       // exp2(-inf) = 0 for warps without keys
+                const float e = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);   // warps without keys
+                const float4 x = *reinterpret_cast<const float4*>(mrg_o + (w * ROWS + r) * MO + d0);
+                const float4 y = *reinterpret_cast<const float4*>(mrg_o + (w * ROWS + r) * MO + d1);
                 L = fmaf(mrg_ml[(w * ROWS + r) * 2 + 1], e, L);
-                O = fmaf(mrg_o[(w * ROWS + r) * MO_STRIDE + d], e, O);
+                a.x = fmaf(x.x, e, a.x); a.y = fmaf(x.y, e, a.y); a.z = fmaf(x.z, e, a.z); a.w = fmaf(x.w, e, a.w);
+                b.x = fmaf(y.x, e, b.x); b.y = fmaf(y.y, e, b.y); b.z = fmaf(y.z, e, b.z); b.w = fmaf(y.w, e, b.w);
             }
             if (direct) {
+                const float inv = 1.f / L;
                 const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
-                reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(O / L);
-                if (d == 0 && p.lse) p.lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+                store4(out + row * D + d0, a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+                store4(out + row * D + d1, b.x * inv, b.y * inv, b.z * inv, b.w * inv);
+                if (c == 0 && p.lse) p.lse[row] = (M + log2f(L)) * 0.6931471805599453f;
             } else {
                 const size_t prow = static_cast<size_t>(slot) * group + r;
-                p.part_o[prow * D + d] = O;
-                if (d == 0) {
-                    p.part_ml[prow * 2] = M;
-                    p.part_ml[prow * 2 + 1] = L;
-                }
+                *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = a;
+                *reinterpret_cast<float4*>(p.part_o + prow * D + d1) = b;
+                if (c == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(M, L);
+            }
+        }
+        if (!direct && p.counters != nullptr) {
+            // ---- the CTA that delivers a split stream's last piece merges all of them: every
+            //      thread's partial stores are fenced, one thread counts this piece in, and the
+            //      CTA that sees the count complete reads the pieces back through L2
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cfence_bar);
+            ok = mbar_wait(cfence_bar, n_split & 1u, abort_flag, p.status, limit);
+            if (!ok) break;
+            const int4 cr = __ldg(p.combine + comb);         // {request, head, first slot, pieces}
+            if (tid == 0) {
+                const uint32_t seen = atomicAdd(p.counters + comb, 1u);
+                const int last = seen + 1u == static_cast<uint32_t>(cr.w);
+                if (last) p.counters[comb] = 0u;              // ready for the next launch
+                *last_flag = last;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cflag_bar);
+            ok = mbar_wait(cflag_bar, n_split & 1u, abort_flag, p.status, limit);
+            if (!ok) break;
+            ++n_split;
+            if (*last_flag) {
+                __threadfence();
+                combine_stream(p.part_o, p.part_ml, cr.z, cr.w, cr.x, cr.y, group, D, p.q_heads,
+                               reinterpret_cast<__nv_bfloat16*>(p.out), p.lse, tid, kConsumerThreads);
             }
         }
         __syncwarp();
@@ -582,7 +708,8 @@ decode_generic_kernel(const DecodeParams p) {
     T* outg = static_cast<T*>(p.out);
     const float scale = p.scale_log2;
 
-    for (int it = p.cta_begin[cta]; it < p.cta_begin[cta + 1]; ++it) {
+    const int4 rec = __ldg(p.cta + 3 * cta);
+    for (int it = rec.x; it < rec.y; ++it) {
         const int4 a = p.items[2 * it], b = p.items[2 * it + 1];
         const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w, direct = b.x, slot = b.y;
         const int64_t row0 = static_cast<int64_t>(p.base[req]) * p.kv_heads +
@@ -715,23 +842,8 @@ combine_kernel(const int4* __restrict__ combine, const float* __restrict__ part_
                const float* __restrict__ part_ml, T* __restrict__ out, float* __restrict__ lse,
                int group, int D, int q_heads) {
     const int4 rec = combine[blockIdx.x];
-    const int req = rec.x, head = rec.y, slot0 = rec.z, ns = rec.w;
-    for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
-        const int r = idx / D, d = idx - r * D;
-        float M = -INFINITY;
-        for (int s = 0; s < ns; ++s)
-            M = fmaxf(M, part_ml[(static_cast<size_t>(slot0 + s) * group + r) * 2]);
-        float L = 0.f, O = 0.f;
-        for (int s = 0; s < ns; ++s) {
-            const size_t prow = static_cast<size_t>(slot0 + s) * group + r;
-            const float e = exp2f(part_ml[prow * 2] - M);
-            L = fmaf(part_ml[prow * 2 + 1], e, L);
-            O = fmaf(part_o[prow * D + d], e, O);
-        }
-        const size_t row = static_cast<size_t>(req) * q_heads + static_cast<size_t>(head) * group + r;
-        store_out(out + row * D + d, O / L);
-        if (d == 0 && lse) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
-    }
+    combine_stream(part_o, part_ml, rec.z, rec.w, rec.x, rec.y, group, D, q_heads, out, lse,
+                   static_cast<int>(threadIdx.x), static_cast<int>(blockDim.x));
 }
 
 // =============================================================================================
@@ -749,13 +861,17 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const AppendParams p) {
         const int tok = static_cast<int>(rem / vecs_per_tok);
         const int within = static_cast<int>(rem - tok * vecs_per_tok);
         const int head = within / p.row_vecs, vec = within - head * p.row_vecs;
-        // request owning new token `tok`: last r with cu_new[r] <= tok
-        int lo = 0, hi = p.n;
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (p.cu_new[mid] <= tok) lo = mid; else hi = mid;
+        // request owning new token `tok`: last r with cu_new[r] <= tok (tok itself when every
+        // request appends exactly one token, the decode case)
+        int req = tok;
+        if (!p.one_new_each) {
+            int lo = 0, hi = p.n;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (p.cu_new[mid] <= tok) lo = mid; else hi = mid;
+            }
+            req = lo;
         }
-        const int req = lo;
         const int n_new = p.cu_new[req + 1] - p.cu_new[req];
         const int pos = p.len[req] - n_new + (tok - p.cu_new[req]);
         const int64_t row = static_cast<int64_t>(p.base[req]) * p.kv_heads +
@@ -813,28 +929,42 @@ __global__ void wait_selftest_kernel(uint32_t* status, int64_t limit_ns) {
 // launch helpers
 // ---------------------------------------------------------------------------------------------
 
-template <int D, bool HI, int MODE>
+constexpr int kSmemPerSm = 233472;        // shared memory of one SM
+constexpr int kSmemPerCtaMax = 232448;    // most one CTA may ask for
+constexpr int kSmemCtaReserve = 1024;     // what the system keeps per resident CTA
+
+template <int D, int NT, int MODE>
 cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_ctas, cudaStream_t stream) {
-    using Cfg = TcConfig<D, HI>;
+    using Cfg = TcConfig<D, NT>;
     static bool configured = false;
-    auto kern = decode_tc_kernel<D, HI, MODE>;
+    auto kern = decode_tc_kernel<D, NT, MODE>;
+    const int smem = Cfg::smem_bytes(p.stages);
+    if (p.stages < 2 || p.stages > kMaxStages || smem > kSmemPerCtaMax) return cudaErrorInvalidValue;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<n_ctas, kTcThreads, Cfg::kSmemBytes, stream>>>(maps.big, maps.small, p);
+    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p);
     return cudaGetLastError();
 }
 
-template <int D, bool HI>
+template <int D, int NT>
 cudaError_t launch_tc_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s) {
     switch (mode) {
-        case kModeSlab: return launch_tc_inst<D, HI, kModeSlab>(maps, p, n_ctas, s);
-        case kModePaged: return launch_tc_inst<D, HI, kModePaged>(maps, p, n_ctas, s);
-        case kModeProbe: return launch_tc_inst<D, HI, kModeProbe>(maps, p, n_ctas, s);
+        case kModeSlab: return launch_tc_inst<D, NT, kModeSlab>(maps, p, n_ctas, s);
+        case kModePaged: return launch_tc_inst<D, NT, kModePaged>(maps, p, n_ctas, s);
+        case kModeProbe: return launch_tc_inst<D, NT, kModeProbe>(maps, p, n_ctas, s);
     }
     return cudaErrorInvalidValue;
+}
+
+template <int D, int NT>
+int32_t tc_stages_inst(int32_t ctas_per_sm) {
+    using Cfg = TcConfig<D, NT>;
+    const int budget = std::min(kSmemPerSm / ctas_per_sm - kSmemCtaReserve, kSmemPerCtaMax);
+    const int n = (budget - Cfg::kFixedBytes - Cfg::kAlignSlack) / Cfg::kStageBytes;
+    return n < 2 ? 0 : (n > kMaxStages ? kMaxStages : n);
 }
 
 template <typename T>
@@ -856,15 +986,22 @@ bool tc_supported(int32_t head_dim, int32_t group) {
 
 bool generic_supported(int32_t head_dim) { return head_dim == 32 || head_dim == 64 || head_dim == 128; }
 
+int32_t tc_stages(int32_t head_dim, int32_t group, int32_t ctas_per_sm) {
+    if (!tc_supported(head_dim, group) || ctas_per_sm < 1) return 0;
+    const bool two = group > 8;
+    if (head_dim == 128) return two ? tc_stages_inst<128, 2>(ctas_per_sm) : tc_stages_inst<128, 1>(ctas_per_sm);
+    return two ? tc_stages_inst<64, 2>(ctas_per_sm) : tc_stages_inst<64, 1>(ctas_per_sm);
+}
+
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
                              cudaStream_t stream) {
-    const bool hi = p.group > 8;
+    const bool two = p.group > 8;
     if (p.head_dim == 128)
-        return hi ? launch_tc_mode<128, true>(maps, p, mode, n_ctas, stream)
-                  : launch_tc_mode<128, false>(maps, p, mode, n_ctas, stream);
+        return two ? launch_tc_mode<128, 2>(maps, p, mode, n_ctas, stream)
+                   : launch_tc_mode<128, 1>(maps, p, mode, n_ctas, stream);
     if (p.head_dim == 64)
-        return hi ? launch_tc_mode<64, true>(maps, p, mode, n_ctas, stream)
-                  : launch_tc_mode<64, false>(maps, p, mode, n_ctas, stream);
+        return two ? launch_tc_mode<64, 2>(maps, p, mode, n_ctas, stream)
+                   : launch_tc_mode<64, 1>(maps, p, mode, n_ctas, stream);
     return cudaErrorInvalidValue;
 }
 

@@ -16,8 +16,11 @@ struct DecodeParams {
     const int32_t* base;
     const int32_t* cap;
     const int32_t* len;
-    const int32_t* cta_begin;
+    const int4* cta;            // three int4 per CTA: {item_begin, item_end, 0, 0}, first item
     const int4* items;          // two int4 per item
+    const int4* combine;        // one int4 per split stream: {request, head, first slot, pieces}
+    uint32_t* counters;         // per split stream: pieces delivered so far (zero between launches);
+                                // nullptr = the caller merges with launch_combine instead
     // tensors
     const void* q;              // [n, q_heads, head_dim]
     void* out;                  // [n, q_heads, head_dim]
@@ -34,6 +37,7 @@ struct DecodeParams {
     const int32_t* page_table;  // [n, max_pages]
     int32_t max_pages;
     int64_t wait_limit_ns;
+    int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
 };
 
 struct TensorMaps {
@@ -45,6 +49,8 @@ enum DecodeMode { kModeSlab = 0, kModePaged = 1, kModeProbe = 2 };
 
 // Returns false when (head_dim, group) has no tensor-core instantiation.
 bool tc_supported(int32_t head_dim, int32_t group);
+// Pipeline stages that fit when `ctas_per_sm` CTAs share one SM's shared memory (0: none fit).
+int32_t tc_stages(int32_t head_dim, int32_t group, int32_t ctas_per_sm);
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
                              cudaStream_t stream);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
@@ -65,6 +71,7 @@ struct AppendParams {
     int64_t rows_per_array;
     int32_t layer, n, kv_heads, n_new_total;
     int32_t row_vecs;           // 16-byte vectors per row
+    int32_t one_new_each;       // every request appends exactly one token: token index = request
 };
 cudaError_t launch_append(const AppendParams& p, cudaStream_t stream);
 

@@ -19,7 +19,7 @@ int64_t plan_table_words(int32_t n, int32_t kv_heads, int32_t n_ctas) {
     int64_t w = 0;
     w += align4(n) * 3;                 // base, cap, len
     w += align4(n + 1);                 // cu_new
-    w += align4(n_ctas + 1);            // cta_begin
+    w += kCtaWords * n_ctas;            // per-CTA records
     w += 8 * (streams + n_ctas);        // items
     w += 4 * std::min<int64_t>(streams, n_ctas);   // combine records
     return w;
@@ -49,12 +49,14 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     t.off_cap = w;        w += align4(n);
     t.off_len = w;        w += align4(n);
     t.off_cu_new = w;     w += align4(n + 1);
-    t.off_cta_begin = w;  w += align4(ctas + 1);
+    t.off_cta = w;        w += kCtaWords * ctas;
     t.off_items = w;
     int32_t* items = table + t.off_items;
 
     int32_t cu = 0;
+    bool one_each = true;
     for (int32_t i = 0; i < n; ++i) {
+        one_each = one_each && (!in.n_new || in.n_new[i] == 1);
         table[t.off_base + i] = in.base[i];
         table[t.off_cap + i] = in.cap[i];
         table[t.off_len + i] = in.len[i];
@@ -86,7 +88,8 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     int64_t pos = 0;
     int32_t stream_first_item = 0;
     for (int32_t c = 0; c < ctas; ++c) {
-        table[t.off_cta_begin + c] = n_items;
+        int32_t* rec = table + t.off_cta + kCtaWords * c;
+        rec[0] = n_items;
         while (pos < cut[c + 1]) {
             const int64_t per = (in.len[r] + kTileTokens - 1) / kTileTokens;
             const int64_t stream_hi = stream_lo + per;
@@ -100,14 +103,18 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
             it[3] = static_cast<int32_t>(tok1 - tok0);
             it[4] = (pos == stream_lo && end == stream_hi) ? 1 : 0;    // whole stream: direct
             it[5] = n_items;                                           // slot = item index
-            it[6] = 0;
-            it[7] = 0;
+            // first row of the piece inside one K (or V) array of the pool
+            it[6] = static_cast<int32_t>(static_cast<int64_t>(in.base[r]) * hkv +
+                                         static_cast<int64_t>(head) * in.cap[r] + tok0);
+            it[7] = -1;                                                // combine record, set below
             if (pos == stream_lo) stream_first_item = n_items;
             ++n_items;
             pos = end;
             if (end == stream_hi) {                                    // stream finished
                 const int32_t pieces = n_items - stream_first_item;
                 if (pieces > 1) {
+                    const int32_t ci = static_cast<int32_t>(comb.size() / 4);
+                    for (int32_t k = stream_first_item; k < n_items; ++k) items[8 * k + 7] = ci;
                     comb.push_back(r);
                     comb.push_back(head);
                     comb.push_back(stream_first_item);
@@ -120,8 +127,14 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
                 }
             }
         }
+        rec[1] = n_items;
+        rec[2] = rec[3] = 0;
     }
-    table[t.off_cta_begin + ctas] = n_items;
+    // a copy of each CTA's first item rides in its record: one load starts the CTA's stream
+    for (int32_t c = 0; c < ctas; ++c) {
+        int32_t* rec = table + t.off_cta + kCtaWords * c;
+        for (int k = 0; k < 8; ++k) rec[4 + k] = rec[0] < rec[1] ? items[8 * rec[0] + k] : 0;
+    }
     w = t.off_items + 8 * n_items;
     t.off_combine = w;
     std::copy(comb.begin(), comb.end(), table + w);
@@ -135,6 +148,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     t.n_combine = static_cast<int32_t>(comb.size() / 4);
     t.words = w;
     t.tile_tokens = kTileTokens;
+    t.one_new_each = one_each ? 1 : 0;
     t.kv_tokens = kv_tokens;
     t.epoch = 0;
     *out = t;

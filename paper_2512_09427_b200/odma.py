@@ -31,7 +31,7 @@ class Config(C.Structure):
                 ("p_num", C.c_int32 * MAX_BUCKETS), ("p_den", C.c_int32),
                 ("gamma_permille", C.c_int32), ("tau_permille", C.c_int32), ("growth", C.c_int32),
                 ("large_fixed", C.c_int32), ("max_batch", C.c_int32), ("max_group", C.c_int32),
-                ("plan_ctas", C.c_int32)]
+                ("plan_ctas", C.c_int32), ("ctas_per_sm", C.c_int32), ("fused_combine", C.c_int32)]
 
 
 class Slab(C.Structure):
@@ -55,7 +55,8 @@ class Stats(C.Structure):
 class Tables(C.Structure):
     _fields_ = [("d_table", C.c_void_p)] + [(k, C.c_int32) for k in
                 ("n", "n_new_total", "n_items", "n_ctas", "n_combine", "words", "off_base", "off_cap",
-                 "off_len", "off_cu_new", "off_cta_begin", "off_items", "off_combine", "tile_tokens")] + \
+                 "off_len", "off_cu_new", "off_cta", "off_items", "off_combine", "tile_tokens", "one_new_each",
+                 "reserved")] + \
                [("kv_tokens", C.c_int64), ("epoch", C.c_uint64)]
 
 

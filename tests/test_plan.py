@@ -35,16 +35,28 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
     pool, t, w = _plan(lens, hkv, ctas)
     n = len(lens)
     assert t.n == n and t.kv_tokens == sum(lens) and t.n_new_total == n and t.tile_tokens == 64
+    assert t.one_new_each == 1
     assert list(w[t.off_len:t.off_len + n]) == list(lens)
     assert list(w[t.off_cu_new:t.off_cu_new + n + 1]) == list(range(n + 1))
     items = w[t.off_items:t.off_items + 8 * t.n_items].reshape(-1, 8)
-    cta_begin = w[t.off_cta_begin:t.off_cta_begin + t.n_ctas + 1]
+    recs = w[t.off_cta:t.off_cta + 12 * t.n_ctas].reshape(-1, 12)
+    # CTA c owns items [recs[c,0], recs[c,1]), shares are consecutive, and each record carries a
+    # copy of its first item
+    cta_begin = np.concatenate([recs[:, 0], recs[-1:, 1]])
+    assert (recs[1:, 0] == recs[:-1, 1]).all() and (recs[:, 2:4] == 0).all()
     assert cta_begin[0] == 0 and cta_begin[-1] == t.n_items and (np.diff(cta_begin) >= 0).all()
+    for c in range(t.n_ctas):
+        if recs[c, 0] < recs[c, 1]:
+            assert list(recs[c, 4:]) == list(items[recs[c, 0]])
     assert t.n_ctas <= ctas
     # coverage: per stream the items tile [0, len) in order with no gap or overlap
     cover = {}
-    for k, (req, head, tok0, ntok, direct, slot, _, _) in enumerate(items):
+    rc, slabs = 0, {r: pool.get_slab(r)[1] for r in range(n)}
+    for k, (req, head, tok0, ntok, direct, slot, row, ci) in enumerate(items):
         assert slot == k and ntok >= 1 and tok0 % 64 == 0
+        base, cap = slabs[req][0], slabs[req][1]
+        assert row == base * hkv + head * cap + tok0        # the documented row(head, t) formula
+        assert (ci == -1) == bool(direct)
         cur = cover.get((req, head), 0)
         assert tok0 == cur
         cover[(req, head)] = tok0 + ntok
@@ -62,6 +74,8 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
         split.setdefault((int(req), int(head)), []).append(k)
     want = [(r, h, ks[0], len(ks)) for (r, h), ks in sorted(split.items()) if len(ks) > 1]
     assert [tuple(int(x) for x in c) for c in comb] == want
+    for ci, (req, head, first, pieces) in enumerate(want):
+        assert (items[first:first + pieces, 7] == ci).all()
     # balance: tiles per CTA within the snapping slack of the ideal share
     tiles = np.array([sum(-(-int(items[k, 3]) // 64) for k in range(cta_begin[c], cta_begin[c + 1]))
                       for c in range(t.n_ctas)])
