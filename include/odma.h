@@ -53,7 +53,8 @@ enum {
     ODMA_ERR_DUP_REQ = 4,     /* request id already live */
     ODMA_ERR_OVERFLOW = 5,    /* length beyond max_len, or beyond the slab on commit */
     ODMA_ERR_CUDA = 6,        /* a CUDA runtime or driver call failed */
-    ODMA_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (status word) */
+    ODMA_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (status word) */
+    ODMA_ERR_TOO_LARGE = 8    /* odma_decode_attention_static: batch beyond its fixed scratch */
 };
 
 enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1 };
@@ -235,6 +236,36 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
                          const uint64_t* reqs, int32_t n, const void* d_q, const void* d_k_new,
                          const void* d_v_new, void* d_out, float* lse, void* stream,
                          odma_tables* tables_out);
+
+/* ---- decode attention that allocates nothing (the paper has no counterpart: this entry point
+ *      exists for how the library is deployed, not for the method) ------------------------
+ * For callers that cannot allocate device memory when they reach this call: a serving
+ * process whose memory manager has already claimed the whole GPU, a plug-in that runs under
+ * a host framework which owns every allocation, code on a path where cudaMalloc (which
+ * synchronises the device) is forbidden.  The result is the one odma_decode_attention
+ * gives, but the partial results of split streams are kept in ONE fixed array of device
+ * memory that is part of the library image (about 2.1 MB on every GPU that loads the
+ * library, until the process exits) rather than in scratch allocated by odma_pool_create,
+ * and the call itself performs no cudaMalloc, cudaFree or other allocating call.
+ *   pool      any pool handle; it supplies the geometry only (layers, kv_heads, head_dim,
+ *             dtype, capacity T).  A pool created with dev_base = NULL (its creation makes
+ *             no CUDA call) is enough; plan the batch with odma_plan_host and copy the
+ *             table words into device memory of your own.
+ *   dev_base  device, 256-byte aligned: the KV memory, laid out as described at the top.
+ *   tables    the descriptor odma_plan_host filled, with d_table set to your device copy
+ *             of the table (16-byte aligned).
+ *   q, out, lse, stream: as for odma_decode_attention.
+ * Limits: at most 512 items in the plan (tables->n_items), at most 8 query heads per KV head,
+ * head_dim 32, 64 or 128; beyond them the call returns ODMA_ERR_TOO_LARGE and launches
+ * nothing.  It runs the plain-ALU decode kernel and the combine kernel for every dtype.
+ * The first call on a device looks up the array's device address (a CUDA runtime query, no
+ * allocation): make that first call before any stream capture, with the device current.
+ * Every call on a GPU uses the same array and leaves its partial results there; a call
+ * reads only slots it has written itself, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, no ordering) race on it. */
+int32_t odma_decode_attention_static(const odma_pool* pool, const void* dev_base, int32_t layer,
+                                     const void* q, int32_t q_heads, const odma_tables* tables,
+                                     void* out, float* lse, void* stream);
 
 /* Synchronises `stream` and returns the device status word as an error code (ODMA_OK,
  * ODMA_ERR_TIMEOUT, or ODMA_ERR_CUDA for a failed stream), clearing it. */

@@ -272,6 +272,7 @@ const char* odma_strerror(int32_t code) {
         case ODMA_ERR_OVERFLOW: return "length beyond capacity";
         case ODMA_ERR_CUDA: return "CUDA call failed";
         case ODMA_ERR_TIMEOUT: return "device-side wait timed out";
+        case ODMA_ERR_TOO_LARGE: return "batch beyond the fixed scratch array of odma_decode_attention_static";
     }
     return "unknown status";
 }
@@ -566,6 +567,31 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
     }
     if (tables_out) *tables_out = t;
     return ODMA_OK;
+}
+
+int32_t odma_decode_attention_static(const odma_pool* pool, const void* dev_base, int32_t layer,
+                                     const void* q, int32_t q_heads, const odma_tables* tables,
+                                     void* out, float* lse, void* stream) {
+    if (!pool || !dev_base || !q || !out || !tables || !tables->d_table) return ODMA_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0 || !aligned16(q) || !aligned16(out) ||
+        !aligned16(tables->d_table))
+        return ODMA_ERR_INVALID;
+    if (layer < 0 || layer >= pool->layers) return ODMA_ERR_INVALID;
+    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
+    if (tables->n < 1 || tables->n_items < 1 || tables->n_ctas < 1) return ODMA_ERR_INVALID;
+    if (!generic_supported(pool->head_dim)) return ODMA_ERR_INVALID;
+    const int32_t group = q_heads / pool->kv_heads;
+    if (tables->n_items > kStaticSlots || group > kStaticGroup || pool->head_dim > kStaticHeadDim)
+        return ODMA_ERR_TOO_LARGE;
+    DecodeParams p;
+    fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
+    p.pool = dev_base;
+    p.status = nullptr;       // the kernels of this path wait on nothing
+    const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
+    cudaError_t e = launch_decode_static(p, pool->dtype, tables->n_ctas,
+                                         reinterpret_cast<const int4*>(tab + tables->off_combine),
+                                         tables->n_combine, as_stream(stream));
+    return e == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
 
 int32_t odma_check_status(odma_pool* pool, void* stream) {

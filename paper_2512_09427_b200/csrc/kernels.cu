@@ -1051,6 +1051,41 @@ cudaError_t launch_scatter_pages(const ScatterPagesParams& p, int64_t max_len, c
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// decode attention with the split partials in a fixed device array instead of allocated scratch
+// ---------------------------------------------------------------------------------------------
+
+// One array per GPU that loads the library, held until the process exits: room for
+// kStaticSlots pieces of kStaticGroup query heads, each head_dim outputs plus (max, sum).
+constexpr int kStaticFloats = kStaticSlots * kStaticGroup * (kStaticHeadDim + 2);
+static __device__ __align__(256) float g_static_partials[kStaticFloats];
+
+cudaError_t launch_decode_static(DecodeParams p, int dtype, int n_ctas, const int4* combine,
+                                 int n_combine, cudaStream_t stream) {
+    // In host code the array's name is not a device address; the address is asked for once
+    // per device, with that device current, and kept.
+    static float* scratch_of_device[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!scratch_of_device[dev]) {
+        float* ptr = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_partials);
+        if (e != cudaSuccess) return e;
+        scratch_of_device[dev] = ptr;
+    }
+    // partial outputs first, then the (max, sum) pairs; every slot a launch reads it has
+    // written itself, so nothing has to start at zero
+    p.part_o = scratch_of_device[dev];
+    p.part_ml = scratch_of_device[dev] + static_cast<size_t>(kStaticSlots) * kStaticGroup * kStaticHeadDim;
+    p.counters = nullptr;
+    e = launch_decode_generic(p, dtype, n_ctas, stream);
+    if (e != cudaSuccess) return e;
+    return launch_combine(combine, n_combine, p.part_o, p.part_ml, p.out, p.lse, p.group, p.head_dim,
+                          p.q_heads, dtype, stream);
+}
+
 cudaError_t launch_wait_selftest(uint32_t* status, int64_t limit_ns, cudaStream_t stream) {
     wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
     return cudaGetLastError();

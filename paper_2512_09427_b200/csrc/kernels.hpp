@@ -97,6 +97,16 @@ struct ScatterPagesParams {
 };
 cudaError_t launch_scatter_pages(const ScatterPagesParams& p, int64_t max_len, cudaStream_t stream);
 
+// Limits of launch_decode_static: pieces (items) per batch, query heads per KV head, head_dim.
+constexpr int kStaticSlots = 512;
+constexpr int kStaticGroup = 8;
+constexpr int kStaticHeadDim = 128;
+// The generic decode kernel and the combine kernel with the split partials kept in a
+// file-scope device array (no allocation).  The first call on a device looks the array's
+// address up; calls that overlap on one GPU share the array and race.
+cudaError_t launch_decode_static(DecodeParams p, int dtype, int n_ctas, const int4* combine,
+                                 int n_combine, cudaStream_t stream);
+
 // A one-thread kernel that waits on a barrier nobody signals, for at most limit_ns, then
 // sets the timeout bit: exercises the bounded-wait path without hanging anything.
 cudaError_t launch_wait_selftest(uint32_t* status, int64_t limit_ns, cudaStream_t stream);

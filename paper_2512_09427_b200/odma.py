@@ -20,7 +20,7 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 MAX_BUCKETS = 8
-OK, ERR_INVALID, ERR_NOMEM, ERR_UNKNOWN_REQ, ERR_DUP_REQ, ERR_OVERFLOW, ERR_CUDA, ERR_TIMEOUT = range(8)
+OK, ERR_INVALID, ERR_NOMEM, ERR_UNKNOWN_REQ, ERR_DUP_REQ, ERR_OVERFLOW, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(9)
 DTYPE_F32, DTYPE_BF16 = 0, 1
 K_APPEND, K_DECODE, K_COMBINE, K_MIGRATE, K_PROBE = range(5)
 
@@ -85,6 +85,7 @@ _SIGS = {
     "odma_decode_step_host": (_i32, [_vp, _i32, _i32, _u64p, _i32, _vp, _vp, _vp, _vp, _vp]),
     "odma_decode_step": (_i32, [_vp, _i32, _i32, _i32, _u64p, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
                                 C.POINTER(Tables)]),
+    "odma_decode_attention_static": (_i32, [_vp, _vp, _i32, _vp, _i32, C.POINTER(Tables), _vp, _vp, _vp]),
     "odma_check_status": (_i32, [_vp, _vp]),
     "odma_selftest_timeout": (_i32, [_vp, _i32, _vp]),
     "odma_read_probe": (_i32, [_vp, _i32, _i32, C.POINTER(Tables), _vp]),
@@ -240,6 +241,14 @@ class Pool:
         _check(_lib.odma_decode_step(self._h, layer, n_layers, q_heads, arr, len(arr), d_q, d_k_new,
                                      d_v_new, d_out, lse or None, stream or None,
                                      C.byref(tables) if tables is not None else None), "odma_decode_step")
+
+    def decode_attention_static(self, dev_base: int, layer: int, q: int, q_heads: int, tables: Tables,
+                                out: int, lse: int = 0, stream: int = 0) -> int:
+        """odma_decode_attention_static: same result as decode_attention, no device allocation
+        anywhere on the call (split partials live in a fixed array inside the library).
+        Returns the status code (ERR_TOO_LARGE beyond the array's limits)."""
+        return _lib.odma_decode_attention_static(self._h, dev_base, layer, q, q_heads, C.byref(tables),
+                                                 out, lse or None, stream or None)
 
     def check_status(self, stream: int = 0) -> int:
         return _lib.odma_check_status(self._h, stream or None)
