@@ -116,9 +116,10 @@ typedef struct odma_stats {
  *   base[n], cap[n], len[n] (length AFTER this step's append), cu_new[n+1] (prefix sum of
  *   the tokens appended this step), cta[n_ctas][12], items[n_items][8], combine[n_combine][4].
  *   cta     = {item_begin, item_end, 0, 0, copy of items[item_begin]}: CTA c works through
- *             items [item_begin, item_end)
+ *             items [item_begin, item_end), pieces of split streams first
  *   item    = {request, kv_head, first_token, n_tokens, direct(1)|partial(0), slot,
- *              first row of the piece inside one K/V array, combine record (-1 if direct)}
+ *              first row of the piece inside one K/V array, combine record (-1 if direct)};
+ *             slots number all pieces in (request, head, token) order
  *   combine = {request, kv_head, first_slot, n_slots}
  * The off_* fields are word offsets of those arrays inside d_table. */
 typedef struct odma_tables {

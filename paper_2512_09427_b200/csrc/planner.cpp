@@ -65,60 +65,74 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     }
     table[t.off_cu_new + n] = cu;
 
-    // cut points: equal shares, moved to a stream boundary when they fall inside a short stream
+    // Cut points.  Shares are equal in COST, not in tiles: starting a stream (its query, its
+    // first rows in a new part of memory, its merge at the end) costs about as much as
+    // streaming kStreamCostTiles more tiles, so a stream of `per` tiles weighs per +
+    // kStreamCostTiles.  A cut that falls into a stream's start-up part moves to the stream's
+    // start, one that falls inside a short stream moves to its nearer end.
+    std::vector<int64_t> first_cost(static_cast<size_t>(n) + 1, 0);
+    for (int32_t i = 0; i < n; ++i)
+        first_cost[i + 1] = first_cost[i] + ((first_tile[i + 1] - first_tile[i]) / hkv + kStreamCostTiles) * hkv;
+    const int64_t total_cost = first_cost[n];
     std::vector<int64_t> cut(static_cast<size_t>(ctas) + 1);
     cut[0] = 0;
     cut[ctas] = total;
     int32_t req = 0;
     for (int32_t c = 1; c < ctas; ++c) {
-        int64_t x = total * c / ctas;
-        while (first_tile[req + 1] <= x) ++req;                     // request holding tile x
+        const int64_t xc = total_cost * c / ctas;
+        while (first_cost[req + 1] <= xc) ++req;                    // request holding cost unit xc
         const int64_t per = (first_tile[req + 1] - first_tile[req]) / hkv;   // tiles per stream
-        const int64_t s0 = first_tile[req] + (x - first_tile[req]) / per * per;
-        const int64_t s1 = s0 + per;
+        const int64_t per_cost = per + kStreamCostTiles;
+        const int64_t sh = (xc - first_cost[req]) / per_cost;       // stream of that request
+        const int64_t off = (xc - first_cost[req]) - sh * per_cost - kStreamCostTiles;
+        const int64_t s0 = first_tile[req] + sh * per, s1 = s0 + per;
+        int64_t x = s0 + std::max<int64_t>(off, 0);
         if (per <= kSnapTiles) x = (x - s0 <= s1 - x) ? s0 : s1;
         cut[c] = std::max(x, cut[c - 1]);
     }
 
-    // walk the tile sequence once, emitting one item per (share, stream) overlap
-    int32_t n_items = 0;
+    // walk the tile sequence once, emitting one piece per (share, stream) overlap, in stream
+    // order; a piece's slot (where its partial result goes) is its index in that order
+    struct Piece { int32_t w[8]; };
+    std::vector<Piece> pieces;
+    std::vector<int32_t> share_begin(static_cast<size_t>(ctas) + 1, 0);
     std::vector<int32_t> comb;      // {req, head, first_slot, n_slots}
     int32_t r = 0, head = 0;
     int64_t stream_lo = 0;          // first tile of the current stream
     int64_t pos = 0;
-    int32_t stream_first_item = 0;
+    int32_t stream_first = 0;
     for (int32_t c = 0; c < ctas; ++c) {
-        int32_t* rec = table + t.off_cta + kCtaWords * c;
-        rec[0] = n_items;
+        share_begin[c] = static_cast<int32_t>(pieces.size());
         while (pos < cut[c + 1]) {
             const int64_t per = (in.len[r] + kTileTokens - 1) / kTileTokens;
             const int64_t stream_hi = stream_lo + per;
             const int64_t end = std::min(stream_hi, cut[c + 1]);
             const int64_t tok0 = (pos - stream_lo) * kTileTokens;
             const int64_t tok1 = std::min<int64_t>((end - stream_lo) * kTileTokens, in.len[r]);
-            int32_t* it = items + 8 * n_items;
-            it[0] = r;
-            it[1] = head;
-            it[2] = static_cast<int32_t>(tok0);
-            it[3] = static_cast<int32_t>(tok1 - tok0);
-            it[4] = (pos == stream_lo && end == stream_hi) ? 1 : 0;    // whole stream: direct
-            it[5] = n_items;                                           // slot = item index
+            const int32_t k = static_cast<int32_t>(pieces.size());
+            Piece pc;
+            pc.w[0] = r;
+            pc.w[1] = head;
+            pc.w[2] = static_cast<int32_t>(tok0);
+            pc.w[3] = static_cast<int32_t>(tok1 - tok0);
+            pc.w[4] = (pos == stream_lo && end == stream_hi) ? 1 : 0;    // whole stream: direct
+            pc.w[5] = k;                                                 // slot
             // first row of the piece inside one K (or V) array of the pool
-            it[6] = static_cast<int32_t>(static_cast<int64_t>(in.base[r]) * hkv +
-                                         static_cast<int64_t>(head) * in.cap[r] + tok0);
-            it[7] = -1;                                                // combine record, set below
-            if (pos == stream_lo) stream_first_item = n_items;
-            ++n_items;
+            pc.w[6] = static_cast<int32_t>(static_cast<int64_t>(in.base[r]) * hkv +
+                                           static_cast<int64_t>(head) * in.cap[r] + tok0);
+            pc.w[7] = -1;                                                // combine record, set below
+            if (pos == stream_lo) stream_first = k;
+            pieces.push_back(pc);
             pos = end;
-            if (end == stream_hi) {                                    // stream finished
-                const int32_t pieces = n_items - stream_first_item;
-                if (pieces > 1) {
+            if (end == stream_hi) {                                      // stream finished
+                const int32_t n_pieces = static_cast<int32_t>(pieces.size()) - stream_first;
+                if (n_pieces > 1) {
                     const int32_t ci = static_cast<int32_t>(comb.size() / 4);
-                    for (int32_t k = stream_first_item; k < n_items; ++k) items[8 * k + 7] = ci;
+                    for (int32_t j = stream_first; j < stream_first + n_pieces; ++j) pieces[j].w[7] = ci;
                     comb.push_back(r);
                     comb.push_back(head);
-                    comb.push_back(stream_first_item);
-                    comb.push_back(pieces);
+                    comb.push_back(stream_first);
+                    comb.push_back(n_pieces);
                 }
                 stream_lo = stream_hi;
                 if (++head == hkv) {
@@ -127,12 +141,26 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
                 }
             }
         }
-        rec[1] = n_items;
-        rec[2] = rec[3] = 0;
     }
-    // a copy of each CTA's first item rides in its record: one load starts the CTA's stream
+    share_begin[ctas] = static_cast<int32_t>(pieces.size());
+    const int32_t n_items = static_cast<int32_t>(pieces.size());
+
+    // Each CTA works through the pieces of split streams first (at most its first and its last
+    // piece), then through the whole streams: partial results are delivered early, so the
+    // merge of a split stream overlaps with streaming instead of trailing the kernel.
+    int32_t out_i = 0;
     for (int32_t c = 0; c < ctas; ++c) {
         int32_t* rec = table + t.off_cta + kCtaWords * c;
+        rec[0] = out_i;
+        for (int pass = 0; pass < 2; ++pass)
+            for (int32_t k = share_begin[c]; k < share_begin[c + 1]; ++k)
+                if ((pieces[k].w[4] == 0) == (pass == 0)) {
+                    std::copy(pieces[k].w, pieces[k].w + 8, items + 8 * out_i);
+                    ++out_i;
+                }
+        rec[1] = out_i;
+        rec[2] = rec[3] = 0;
+        // a copy of the CTA's first item rides in its record: one load starts its stream
         for (int k = 0; k < 8; ++k) rec[4 + k] = rec[0] < rec[1] ? items[8 * rec[0] + k] : 0;
     }
     w = t.off_items + 8 * n_items;

@@ -10,6 +10,7 @@ namespace odma {
 
 constexpr int32_t kTileTokens = 64;   // tokens staged per pipeline stage
 constexpr int32_t kSnapTiles = 2;     // streams this short are never cut in two
+constexpr int32_t kStreamCostTiles = 1;  // a stream's start-up weighs as much as this many tiles
 constexpr int32_t kCtaWords = 12;     // per-CTA record: {item_begin, item_end, 0, 0, first item[8]}
 
 struct PlanInput {

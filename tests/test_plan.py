@@ -49,11 +49,18 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
         if recs[c, 0] < recs[c, 1]:
             assert list(recs[c, 4:]) == list(items[recs[c, 0]])
     assert t.n_ctas <= ctas
-    # coverage: per stream the items tile [0, len) in order with no gap or overlap
+    # within a CTA's share the pieces of split streams come first
+    for c in range(t.n_ctas):
+        d = items[cta_begin[c]:cta_begin[c + 1], 4]
+        assert list(d) == sorted(d) and (d == 0).sum() <= 2
+    # slots number the pieces in (request, head, token) order; per stream they tile [0, len)
+    # in order with no gap or overlap
+    by_slot = items[np.argsort(items[:, 5])]
+    assert list(by_slot[:, 5]) == list(range(t.n_items))
     cover = {}
-    rc, slabs = 0, {r: pool.get_slab(r)[1] for r in range(n)}
-    for k, (req, head, tok0, ntok, direct, slot, row, ci) in enumerate(items):
-        assert slot == k and ntok >= 1 and tok0 % 64 == 0
+    slabs = {r: pool.get_slab(r)[1] for r in range(n)}
+    for req, head, tok0, ntok, direct, slot, row, ci in by_slot:
+        assert ntok >= 1 and tok0 % 64 == 0
         base, cap = slabs[req][0], slabs[req][1]
         assert row == base * hkv + head * cap + tok0        # the documented row(head, t) formula
         assert (ci == -1) == bool(direct)
@@ -65,24 +72,27 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
         if tok0 + ntok < lens[req]:
             assert ntok % 64 == 0                     # only a stream's last piece is ragged
     assert cover == {(r, h): lens[r] for r in range(n) for h in range(hkv)}
-    # items are in (request, head, token) order, so a stream's slots are consecutive
-    keys = [(int(a), int(b), int(c)) for a, b, c in items[:, :3]]
+    keys = [(int(a), int(b), int(c)) for a, b, c in by_slot[:, :3]]
     assert keys == sorted(keys)
     comb = w[t.off_combine:t.off_combine + 4 * t.n_combine].reshape(-1, 4)
     split = {}
-    for k, (req, head, *_rest) in enumerate(items):
-        split.setdefault((int(req), int(head)), []).append(k)
+    for req, head, _, _, _, slot, _, _ in by_slot:
+        split.setdefault((int(req), int(head)), []).append(int(slot))
     want = [(r, h, ks[0], len(ks)) for (r, h), ks in sorted(split.items()) if len(ks) > 1]
     assert [tuple(int(x) for x in c) for c in comb] == want
     for ci, (req, head, first, pieces) in enumerate(want):
-        assert (items[first:first + pieces, 7] == ci).all()
-    # balance: tiles per CTA within the snapping slack of the ideal share
+        assert (by_slot[first:first + pieces, 7] == ci).all()
+    # balance: shares are equal in cost, a stream weighing its tiles plus one for its start-up
+    # (a cut never lands inside that start-up part, and short streams are never cut)
     tiles = np.array([sum(-(-int(items[k, 3]) // 64) for k in range(cta_begin[c], cta_begin[c + 1]))
                       for c in range(t.n_ctas)])
+    starts = np.array([sum(1 for k in range(cta_begin[c], cta_begin[c + 1]) if items[k, 2] == 0)
+                       for c in range(t.n_ctas)])
     total = sum(-(-L // 64) for L in lens) * hkv
-    assert tiles.sum() == total
-    ideal = total / t.n_ctas
-    assert tiles.max() <= np.ceil(ideal) + 2 and tiles.min() >= np.floor(ideal) - 2
+    assert tiles.sum() == total and starts.sum() == n * hkv
+    cost = tiles + starts
+    ideal = cost.sum() / t.n_ctas
+    assert cost.max() <= np.ceil(ideal) + 3 and cost.min() >= np.floor(ideal) - 3
     assert t.words * 4 <= pool.tables_bytes(n)
 
 
