@@ -217,7 +217,8 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->q_heads = q_heads;
     p->kv_heads = pool->kv_heads;
     p->group = q_heads / pool->kv_heads;
-    p->stages = tc_stages(pool->head_dim, p->group, pool->alloc.config().ctas_per_sm);
+    tc_shape(pool->head_dim, p->group, pool->alloc.config().ctas_per_sm, &p->stages, &p->q_slots);
+    p->fin_warps = pool->alloc.config().ctas_per_sm == 1 ? 4 : 2;   // two CTAs share the register file
     p->head_dim = pool->head_dim;
     p->scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(pool->head_dim)));
     p->status = pool->d_status;

@@ -15,6 +15,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "odma.h"
 
@@ -139,13 +140,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // decode attention, tensor-core path (bf16, head_dim 64 or 128, group <= 16)
 // =============================================================================================
 //
-// Roles: warps 0..3 consume, warp 4 (one lane) produces.  A pipeline stage holds one tile of 64
-// keys and 64 values of one stream, written by TMA with the 128-byte swizzle so that ldmatrix
-// reads are conflict-free.  Consumer warp w owns keys [16w, 16w+16) of every tile and keeps its
-// own running (max, sum, output); the four are merged through shared memory when the item ends.
+// Roles: warps 0..3 consume, warp 4 (one lane) produces, warps 5.. finish.  A pipeline stage
+// holds one tile of 64 keys and 64 values of one stream, written by TMA with the 128-byte
+// swizzle so that ldmatrix reads are conflict-free.  Consumer warp w owns keys [16w, 16w+16) of
+// every tile and keeps its own running (max, sum, output).  When an item ends the four warps
+// drop their partial results into one of two merge buffers and go straight on to the next
+// item; the finisher warps merge the four, write the item's result (or partial result) to
+// global memory and, for a split stream, count the piece in and merge all pieces if it was
+// the last one.  Queries and item descriptors travel through a ring of 4..8 slots so the
+// producer can run several short items ahead of the consumers.
 //
 // The contraction is arranged with the KEYS on the M side of the MMA tiles and the query heads
-// of the GQA group on the N side (8 heads per n-tile, rows >= group are zero):
+// of the GQA group on the N side (8 heads per n-tile; columns >= group hold whatever the
+// query slot holds and are never written out: a column of the product depends on that column
+// of the B operand only):
 //     S^T[16 keys x 8 heads]  = K[16 keys x D]   . Q^T[D x 8 heads]
 //     O^T[D x 8 heads]       += V^T[D x 16 keys] . P^T[16 keys x 8 heads]
 // so a group of 7 heads wastes one column in eight instead of nine rows in sixteen, and the
@@ -154,9 +162,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kTcThreads = kConsumerThreads + 32;
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kFinisherWarp0 = kConsumerWarps + 1;
+constexpr int kMaxFinisherWarps = 4;              // 2 when two CTAs share an SM (register file)
+constexpr int kTcThreads = kConsumerThreads + 32 + kMaxFinisherWarps * 32;
 constexpr int kTile = 64;
 constexpr int kMaxStages = 8;
+constexpr int kMinQSlots = 4, kMaxQSlots = 8;
+constexpr int kMergeBufs = 2;
+constexpr int kNumBars = 2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs + 2;
 
 template <int D, int NT>
 struct TcConfig {
@@ -167,10 +181,13 @@ struct TcConfig {
     static constexpr int kMoStride = D + 4;
     static constexpr int kMergeFloats = kConsumerWarps * kRows * kMoStride;
     static constexpr int kMlFloats = kConsumerWarps * kRows * 2;
-    static constexpr int kFixedBytes =
-        2 * kQBytes + (kMergeFloats + kMlFloats) * 4 + 2 * 8 * 4 /*desc*/ + (2 * kMaxStages + 8) * 8 /*barriers*/ + 64;
+    // merge buffers (+ their item headers), descriptor ring, barriers, flags
+    static constexpr int kFixedBytes = kMergeBufs * ((kMergeFloats + kMlFloats) * 4 + 32) +
+                                       kMaxQSlots * 32 + kNumBars * 8 + 64;
     static constexpr int kAlignSlack = 1024;
-    static int smem_bytes(int stages) { return stages * kStageBytes + kFixedBytes + kAlignSlack; }
+    static int smem_bytes(int stages, int q_slots) {
+        return stages * kStageBytes + q_slots * kQBytes + kFixedBytes + kAlignSlack;
+    }
 };
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
@@ -188,39 +205,45 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float
     *reinterpret_cast<uint2*>(p) = make_uint2(pack_bf16(a, b), pack_bf16(c, d));
 }
 
+// One step of the log-sum-exp merge: folds a piece (m, l, x) into the running (M, L, a), all
+// maxima in the log2 domain.  Pieces are always folded in slot order, so the result does not
+// depend on which CTA happens to do the merge.
+__device__ __forceinline__ void lse_fold(float& M, float& L, float4& a, float m, float l, const float4& x) {
+    const float mn = fmaxf(M, m);
+    const float e0 = M == -INFINITY ? 0.f : exp2f(M - mn);
+    const float e1 = m == -INFINITY ? 0.f : exp2f(m - mn);
+    L = fmaf(L, e0, l * e1);
+    a.x = fmaf(a.x, e0, x.x * e1);
+    a.y = fmaf(a.y, e0, x.y * e1);
+    a.z = fmaf(a.z, e0, x.z * e1);
+    a.w = fmaf(a.w, e0, x.w * e1);
+    M = mn;
+}
+
 // Log-sum-exp merge of the `ns` partial results of one (request, KV head) stream, slots
 // [slot0, slot0+ns): out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), M = max_s m_s.
-// Thread `tid` of `nthreads` takes two groups of four output elements of one query head.
+// Thread `tid` of `nthreads` takes groups of four output elements of one query head.
 // Partials are read through L2 (they may have been written by other SMs a moment ago).
 template <typename T>
 __device__ __forceinline__ void combine_stream(const float* part_o, const float* part_ml, int slot0,
                                                int ns, int req, int head, int group, int D,
                                                int q_heads, T* out, float* lse, int tid, int nthreads) {
-    const int per_row = D >> 3;
+    const int per_row = D >> 2;
     for (int idx = tid; idx < group * per_row; idx += nthreads) {
-        const int r = idx / per_row, c = idx - r * per_row;
-        const int d0 = c * 4, d1 = (D >> 1) + c * 4;
-        float M = -INFINITY;
+        const int r = idx / per_row, d0 = (idx - r * per_row) * 4;
+        float M = -INFINITY, L = 0.f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-        for (int s = 0; s < ns; ++s)
-            M = fmaxf(M, __ldcg(part_ml + (static_cast<size_t>(slot0 + s) * group + r) * 2));
-        float L = 0.f;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-#pragma unroll 2
         for (int s = 0; s < ns; ++s) {
             const size_t prow = static_cast<size_t>(slot0 + s) * group + r;
             const float2 ml = __ldcg(reinterpret_cast<const float2*>(part_ml + prow * 2));
-            const float e = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
-            const float4 x = ldcg4(part_o + prow * D + d0), y = ldcg4(part_o + prow * D + d1);
-            L = fmaf(ml.y, e, L);
-            a.x = fmaf(x.x, e, a.x); a.y = fmaf(x.y, e, a.y); a.z = fmaf(x.z, e, a.z); a.w = fmaf(x.w, e, a.w);
-            b.x = fmaf(y.x, e, b.x); b.y = fmaf(y.y, e, b.y); b.z = fmaf(y.z, e, b.z); b.w = fmaf(y.w, e, b.w);
+            const float4 x = ldcg4(part_o + prow * D + d0);
+            lse_fold(M, L, a, ml.x, ml.y, x);
         }
         const float inv = 1.f / L;
         const size_t row = static_cast<size_t>(req) * q_heads + static_cast<size_t>(head) * group + r;
         store4(out + row * D + d0, a.x * inv, a.y * inv, a.z * inv, a.w * inv);
-        store4(out + row * D + d1, b.x * inv, b.y * inv, b.z * inv, b.w * inv);
-        if (c == 0 && lse) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+        if (d0 == 0 && lse) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
     }
 }
 
@@ -233,30 +256,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     constexpr int HALVES = D / 64;                 // 128-byte column blocks per row
     constexpr int HALF_BYTES = kTile * 128;
     constexpr int MO = Cfg::kMoStride;
-    const int STAGES = p.stages;
+    const uint32_t STAGES = static_cast<uint32_t>(p.stages);
+    const uint32_t QSLOTS = static_cast<uint32_t>(p.q_slots);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* kv = smem;
     uint8_t* qbuf = kv + STAGES * Cfg::kStageBytes;
-    float* mrg_o = reinterpret_cast<float*>(qbuf + 2 * Cfg::kQBytes);
-    float* mrg_ml = mrg_o + Cfg::kMergeFloats;
-    int* desc = reinterpret_cast<int*>(mrg_ml + Cfg::kMlFloats);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(desc + 16);
-    volatile int* flags = reinterpret_cast<volatile int*>(bars + 2 * kMaxStages + 8);
-    volatile int* abort_flag = flags;            // flags[0]: a wait timed out somewhere in the CTA
-    volatile int* last_flag = flags + 1;         // flags[1]: this CTA completes a split stream
+    float* mrg_o = reinterpret_cast<float*>(qbuf + QSLOTS * Cfg::kQBytes);
+    float* mrg_ml = mrg_o + kMergeBufs * Cfg::kMergeFloats;
+    int* mrg_hdr = reinterpret_cast<int*>(mrg_ml + kMergeBufs * Cfg::kMlFloats);   // 8 ints per buffer
+    int* desc = mrg_hdr + kMergeBufs * 8;                                           // 8 ints per slot
+    uint64_t* bars = reinterpret_cast<uint64_t*>(desc + kMaxQSlots * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars);
+    volatile int* last_flag = abort_flag + 1;    // finishers: this CTA delivered a stream's last piece
 
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kMaxStages + s); };
     auto qfull_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + s); };
-    auto qempty_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 + s); };
-    const uint32_t mready_bar = bar0 + 8u * (2 * kMaxStages + 4);
-    const uint32_t mdone_bar = bar0 + 8u * (2 * kMaxStages + 5);
-    const uint32_t cfence_bar = bar0 + 8u * (2 * kMaxStages + 6);
-    const uint32_t cflag_bar = bar0 + 8u * (2 * kMaxStages + 7);
+    auto qempty_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + kMaxQSlots + s); };
+    auto mready_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + s); };
+    auto mdone_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + kMergeBufs + s); };
+    const uint32_t fstored_bar = bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs);
+    const uint32_t fcounted_bar = fstored_bar + 8u;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -265,41 +289,41 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
 
     // the producer's first loads are in flight while the barriers are being set up
     int4 rec = make_int4(0, 0, 0, 0), first_a = rec, first_b = rec;
-    if (tid == kConsumerThreads) {
+    if (tid == kProducerWarp * 32) {
         const int4* r = p.cta + 3 * cta;
         rec = __ldg(r);
         first_a = __ldg(r + 1);
         first_b = __ldg(r + 2);
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_big)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_small)) : "memory");
+    } else if (warp >= kFinisherWarp0 && lane == 0) {
+        rec = __ldg(p.cta + 3 * cta);
     }
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (uint32_t s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), kConsumerWarps);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (uint32_t s = 0; s < QSLOTS; ++s) {
             mbar_init(qfull_bar(s), 1);
             mbar_init(qempty_bar(s), kConsumerWarps);
         }
-        mbar_init(mready_bar, kConsumerWarps);
-        mbar_init(mdone_bar, kConsumerWarps);
-        mbar_init(cfence_bar, kConsumerWarps);
-        mbar_init(cflag_bar, kConsumerWarps);
-        flags[0] = 0;
-        flags[1] = 0;
+        for (uint32_t s = 0; s < kMergeBufs; ++s) {
+            mbar_init(mready_bar(s), kConsumerWarps);
+            mbar_init(mdone_bar(s), p.fin_warps);
+        }
+        mbar_init(fstored_bar, p.fin_warps);
+        mbar_init(fcounted_bar, p.fin_warps);
+        *abort_flag = 0;
+        *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // query rows >= group stay zero for the whole kernel; the bulk copy only writes rows < group
-    for (int i = tid; i < 2 * Cfg::kQBytes / 16; i += kTcThreads)
-        reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0, 0, 0, 0);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
 
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             const int it_begin = rec.x, it_end = rec.y;
@@ -308,10 +332,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             bool ok = true;
             const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
             const int64_t v_array = k_array + p.rows_per_array;
-            uint32_t k_item = 0;
-            for (int it = it_begin; ok; ++it, ++k_item) {
-                const uint32_t qs = k_item & 1u;
-                ok = mbar_wait(qempty_bar(qs), ((k_item >> 1) & 1u) ^ 1u, abort_flag, p.status, limit);
+            uint32_t qs = 0, qphase = 0;
+            for (int it = it_begin; ok; ++it) {
+                ok = mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit);
                 if (!ok) break;
                 int* dsc = desc + qs * 8;
                 if (it >= it_end) {                      // end marker
@@ -337,6 +360,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                           static_cast<const uint8_t*>(p.q) +
                               (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
                           q_bytes, qfull_bar(qs));
+                if (++qs == QSLOTS) {
+                    qs = 0;
+                    qphase ^= 1u;
+                }
                 const int64_t row = b.z;
                 const int32_t* pages = nullptr;
                 if (MODE == kModePaged)
@@ -382,7 +409,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                     }
                     issued_any |= 1u << stage;
                     issued_odd ^= 1u << stage;
-                    if (++stage == static_cast<uint32_t>(STAGES)) {
+                    if (++stage == STAGES) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -391,13 +418,156 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             if (!ok) {
                 // Something timed out.  Before the CTA's shared memory can be handed to another
                 // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
-                for (int s = 0; s < STAGES; ++s)
+                for (uint32_t s = 0; s < STAGES; ++s)
                     if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
                         mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
                                        limit / 4 + 1);
             }
         }
         __syncwarp();
+        return;
+    }
+
+    if (warp >= kFinisherWarp0) {
+        // ------------------------------------------------------------------ finishers
+        if (MODE == kModeProbe) return;
+        const int ftid = tid - kFinisherWarp0 * 32;
+        const int fthreads = p.fin_warps * 32;
+        const int n_items = __shfl_sync(0xFFFFFFFFu, rec.y - rec.x, 0);
+        const int group = p.group;
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+        constexpr int PER_ROW = D / 4;                   // float4 chunks per head
+        const int total = group * PER_ROW;
+        // CH = chunks of four output elements per thread; every thread computes CH chunks
+        // (indices past the end are clamped, their results dropped) so the code is branch-free
+        auto run = [&](auto ch_tag) {
+            constexpr int CH = decltype(ch_tag)::value;
+            uint32_t n_split = 0;
+            for (int k = 0; k < n_items; ++k) {
+                const uint32_t mb = static_cast<uint32_t>(k) & 1u;
+                if (!mbar_wait(mready_bar(mb), (static_cast<uint32_t>(k) >> 1) & 1u, abort_flag, p.status, limit))
+                    return;
+                const int* hdr = mrg_hdr + mb * 8;
+                const int req = hdr[0], head = hdr[1], direct = hdr[2], slot = hdr[3], comb = hdr[4];
+                const bool count_in = !direct && p.counters != nullptr;
+                int4 cr = make_int4(0, 0, 0, 0);         // {request, head, first slot, pieces}
+                if (count_in) cr = __ldg(p.combine + comb);
+                const float* bo = mrg_o + mb * Cfg::kMergeFloats;
+                const float* bml = mrg_ml + mb * Cfg::kMlFloats;
+                float4 acc[CH];
+                float acc_m[CH], acc_l[CH];
+                int rr[CH], dd[CH];
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const int idx = min(ftid + i * fthreads, total - 1);
+                    const int r = idx / PER_ROW, d0 = (idx - r * PER_ROW) * 4;
+                    rr[i] = r;
+                    dd[i] = d0;
+                    float mw[kConsumerWarps], lw[kConsumerWarps], M = -INFINITY;
+                    float4 x[kConsumerWarps];
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float2 ml = *reinterpret_cast<const float2*>(bml + (w * ROWS + r) * 2);
+                        mw[w] = ml.x;
+                        lw[w] = ml.y;
+                        x[w] = *reinterpret_cast<const float4*>(bo + (w * ROWS + r) * MO + d0);
+                        M = fmaxf(M, ml.x);
+                    }
+                    float L = 0.f;
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float e = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);   // warps without keys
+                        L = fmaf(lw[w], e, L);
+                        a.x = fmaf(x[w].x, e, a.x);
+                        a.y = fmaf(x[w].y, e, a.y);
+                        a.z = fmaf(x[w].z, e, a.z);
+                        a.w = fmaf(x[w].w, e, a.w);
+                    }
+                    acc[i] = a;
+                    acc_m[i] = M;
+                    acc_l[i] = L;
+                }
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    if (ftid + i * fthreads >= total) continue;
+                    const int r = rr[i], d0 = dd[i];
+                    if (direct) {
+                        const float inv = 1.f / acc_l[i];
+                        const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
+                        store4(out + row * D + d0, acc[i].x * inv, acc[i].y * inv, acc[i].z * inv, acc[i].w * inv);
+                        if (d0 == 0 && p.lse) p.lse[row] = (acc_m[i] + log2f(acc_l[i])) * 0.6931471805599453f;
+                    } else {
+                        const size_t prow = static_cast<size_t>(slot) * group + r;
+                        *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = acc[i];
+                        if (d0 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(acc_m[i], acc_l[i]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(mdone_bar(mb));          // the buffer may be refilled
+                    if (count_in) mbar_arrive(fstored_bar);
+                }
+                if (!count_in) continue;
+                // The CTA that delivers a split stream's last piece merges all of them.  Once
+                // every finisher thread has issued its partial stores, one thread fences them,
+                // counts this piece in and tells the rest whether the count is complete; if so
+                // each thread folds all pieces in slot order, its own from the registers it
+                // still holds, the others read back through L2.
+                if (!mbar_wait(fstored_bar, n_split & 1u, abort_flag, p.status, limit)) return;
+                if (ftid == 0) {
+                    __threadfence();
+                    const uint32_t seen = atomicAdd(p.counters + comb, 1u);
+                    const int last = seen + 1u == static_cast<uint32_t>(cr.w);
+                    if (last) p.counters[comb] = 0u;      // ready for the next launch
+                    *last_flag = last;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(fcounted_bar);
+                if (!mbar_wait(fcounted_bar, n_split & 1u, abort_flag, p.status, limit)) return;
+                ++n_split;
+                if (!*last_flag) continue;
+                __threadfence();
+                const size_t orow0 = static_cast<size_t>(cr.x) * p.q_heads + static_cast<size_t>(cr.y) * group;
+                float fm[CH], fl[CH];
+                float4 fa[CH];
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    fm[i] = -INFINITY;
+                    fl[i] = 0.f;
+                    fa[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                for (int s = 0; s < cr.w; ++s) {
+                    if (cr.z + s == slot) {               // this CTA's own piece
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], acc_m[i], acc_l[i], acc[i]);
+                        continue;
+                    }
+                    float2 ml[CH];
+                    float4 x[CH];
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) {        // all loads of the piece first
+                        const size_t prow = static_cast<size_t>(cr.z + s) * group + rr[i];
+                        ml[i] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
+                        x[i] = ldcg4(p.part_o + prow * D + dd[i]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], ml[i].x, ml[i].y, x[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    if (ftid + i * fthreads >= total) continue;
+                    const float inv = 1.f / fl[i];
+                    store4(out + (orow0 + rr[i]) * D + dd[i], fa[i].x * inv, fa[i].y * inv, fa[i].z * inv, fa[i].w * inv);
+                    if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + log2f(fl[i])) * 0.6931471805599453f;
+                }
+            }
+        };
+        constexpr int CHUNKS4 = (ROWS * PER_ROW + 127) / 128;   // with four finisher warps
+        if (p.fin_warps == 4)
+            run(std::integral_constant<int, CHUNKS4>{});
+        else
+            run(std::integral_constant<int, 2 * CHUNKS4>{});
         return;
     }
 
@@ -415,13 +585,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     const int key_lo = warp * 16 + qd;                // the thread's two key rows: key_lo, key_lo + 8
     const int vkey0 = warp * 16 + qt * 2;             // keys of its value fragments: vkey0, +1, +8, +9
     const float scale = p.scale_log2;
-    const int group = p.group;
 
-    uint32_t stage = 0, phase = 0, n_split = 0;
+    uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
     bool ok = true;
     for (uint32_t k_item = 0; ok; ++k_item) {
-        const uint32_t qs = k_item & 1u;
-        ok = mbar_wait(qfull_bar(qs), (k_item >> 1) & 1u, abort_flag, p.status, limit);
+        ok = mbar_wait(qfull_bar(qs), qphase, abort_flag, p.status, limit);
         if (!ok) break;
         const int* dsc = desc + qs * 8;
         const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3], slot = dsc[4], comb = dsc[5];
@@ -443,6 +611,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(qempty_bar(qs));
+        if (++qs == QSLOTS) {
+            qs = 0;
+            qphase ^= 1u;
+        }
 
         float o[NT][D / 16][4];
         float m_run[NT][2], l_run[NT][2];
@@ -542,7 +714,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar(stage));
-            if (++stage == static_cast<uint32_t>(STAGES)) {
+            if (++stage == STAGES) {
                 stage = 0;
                 phase ^= 1u;
             }
@@ -550,7 +722,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         if (!ok) break;
         if (MODE == kModeProbe) continue;
 
-        // ---- merge the four warps' partial results and write the item's result
+        // ---- hand the warp's partial result to the finishers and move on
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -558,12 +730,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 l_run[nt][0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][0], off);
                 l_run[nt][1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][1], off);
             }
-        if (k_item > 0) {
-            ok = mbar_wait(mdone_bar, (k_item - 1u) & 1u, abort_flag, p.status, limit);
+        const uint32_t mb = k_item & 1u;
+        if (k_item >= 2) {                            // the finishers are done with item k_item - 2
+            ok = mbar_wait(mdone_bar(mb), ((k_item >> 1) - 1u) & 1u, abort_flag, p.status, limit);
             if (!ok) break;
         }
-        float* mo = mrg_o + warp * ROWS * MO;
-        float* mml = mrg_ml + warp * ROWS * 2;
+        float* mo = mrg_o + mb * Cfg::kMergeFloats + warp * ROWS * MO;
+        float* mml = mrg_ml + mb * Cfg::kMlFloats + warp * ROWS * 2;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int h0 = nt * 8 + qt * 2;
@@ -582,74 +755,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 mml[h0 * 2 + 3] = l_run[nt][1];
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(mready_bar);
-        ok = mbar_wait(mready_bar, k_item & 1u, abort_flag, p.status, limit);
-        if (!ok) break;
-        constexpr int PER_ROW = D / 8;
-        for (int idx = tid; idx < group * PER_ROW; idx += kConsumerThreads) {
-            const int r = idx / PER_ROW, c = idx - r * PER_ROW;
-            const int d0 = c * 4, d1 = D / 2 + c * 4;
-            float mw[kConsumerWarps], M = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
-                mw[w] = mrg_ml[(w * ROWS + r) * 2];
-                M = fmaxf(M, mw[w]);
-            }
-            float L = 0.f;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
-                const float e = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);   // warps without keys
-                const float4 x = *reinterpret_cast<const float4*>(mrg_o + (w * ROWS + r) * MO + d0);
-                const float4 y = *reinterpret_cast<const float4*>(mrg_o + (w * ROWS + r) * MO + d1);
-                L = fmaf(mrg_ml[(w * ROWS + r) * 2 + 1], e, L);
-                a.x = fmaf(x.x, e, a.x); a.y = fmaf(x.y, e, a.y); a.z = fmaf(x.z, e, a.z); a.w = fmaf(x.w, e, a.w);
-                b.x = fmaf(y.x, e, b.x); b.y = fmaf(y.y, e, b.y); b.z = fmaf(y.z, e, b.z); b.w = fmaf(y.w, e, b.w);
-            }
-            if (direct) {
-                const float inv = 1.f / L;
-                const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
-                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-                store4(out + row * D + d0, a.x * inv, a.y * inv, a.z * inv, a.w * inv);
-                store4(out + row * D + d1, b.x * inv, b.y * inv, b.z * inv, b.w * inv);
-                if (c == 0 && p.lse) p.lse[row] = (M + log2f(L)) * 0.6931471805599453f;
-            } else {
-                const size_t prow = static_cast<size_t>(slot) * group + r;
-                *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = a;
-                *reinterpret_cast<float4*>(p.part_o + prow * D + d1) = b;
-                if (c == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(M, L);
-            }
-        }
-        if (!direct && p.counters != nullptr) {
-            // ---- the CTA that delivers a split stream's last piece merges all of them: every
-            //      thread's partial stores are fenced, one thread counts this piece in, and the
-            //      CTA that sees the count complete reads the pieces back through L2
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(cfence_bar);
-            ok = mbar_wait(cfence_bar, n_split & 1u, abort_flag, p.status, limit);
-            if (!ok) break;
-            const int4 cr = __ldg(p.combine + comb);         // {request, head, first slot, pieces}
-            if (tid == 0) {
-                const uint32_t seen = atomicAdd(p.counters + comb, 1u);
-                const int last = seen + 1u == static_cast<uint32_t>(cr.w);
-                if (last) p.counters[comb] = 0u;              // ready for the next launch
-                *last_flag = last;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(cflag_bar);
-            ok = mbar_wait(cflag_bar, n_split & 1u, abort_flag, p.status, limit);
-            if (!ok) break;
-            ++n_split;
-            if (*last_flag) {
-                __threadfence();
-                combine_stream(p.part_o, p.part_ml, cr.z, cr.w, cr.x, cr.y, group, D, p.q_heads,
-                               reinterpret_cast<__nv_bfloat16*>(p.out), p.lse, tid, kConsumerThreads);
-            }
+        if (tid == 0) {
+            int* hdr = mrg_hdr + mb * 8;
+            hdr[0] = req;
+            hdr[1] = head;
+            hdr[2] = direct;
+            hdr[3] = slot;
+            hdr[4] = comb;
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(mdone_bar);
+        if (lane == 0) mbar_arrive(mready_bar(mb));
     }
 }
 
@@ -938,14 +1053,16 @@ cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_
     using Cfg = TcConfig<D, NT>;
     static bool configured = false;
     auto kern = decode_tc_kernel<D, NT, MODE>;
-    const int smem = Cfg::smem_bytes(p.stages);
-    if (p.stages < 2 || p.stages > kMaxStages || smem > kSmemPerCtaMax) return cudaErrorInvalidValue;
+    const int smem = Cfg::smem_bytes(p.stages, p.q_slots);
+    if (p.stages < 2 || p.stages > kMaxStages || p.q_slots < kMinQSlots || p.q_slots > kMaxQSlots ||
+        smem > kSmemPerCtaMax || (p.fin_warps != 2 && p.fin_warps != kMaxFinisherWarps))
+        return cudaErrorInvalidValue;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p);
+    kern<<<n_ctas, kConsumerThreads + 32 + p.fin_warps * 32, smem, stream>>>(maps.big, maps.small, p);
     return cudaGetLastError();
 }
 
@@ -959,12 +1076,22 @@ cudaError_t launch_tc_mode(const TensorMaps& maps, const DecodeParams& p, int mo
     return cudaErrorInvalidValue;
 }
 
+// Pipeline depth and query-ring depth that fit when `ctas_per_sm` CTAs share an SM: as many
+// stages as possible on top of the smallest ring, then the ring grows into what is left.
 template <int D, int NT>
-int32_t tc_stages_inst(int32_t ctas_per_sm) {
+void tc_shape_inst(int32_t ctas_per_sm, int32_t* stages, int32_t* q_slots) {
     using Cfg = TcConfig<D, NT>;
     const int budget = std::min(kSmemPerSm / ctas_per_sm - kSmemCtaReserve, kSmemPerCtaMax);
-    const int n = (budget - Cfg::kFixedBytes - Cfg::kAlignSlack) / Cfg::kStageBytes;
-    return n < 2 ? 0 : (n > kMaxStages ? kMaxStages : n);
+    const int room = budget - Cfg::kFixedBytes - Cfg::kAlignSlack - kMinQSlots * Cfg::kQBytes;
+    int n = room / Cfg::kStageBytes;
+    n = n > kMaxStages ? kMaxStages : n;
+    if (n < 2) {
+        *stages = *q_slots = 0;
+        return;
+    }
+    const int extra = (room - n * Cfg::kStageBytes) / Cfg::kQBytes;
+    *stages = n;
+    *q_slots = std::min(kMaxQSlots, kMinQSlots + extra);
 }
 
 template <typename T>
@@ -986,11 +1113,14 @@ bool tc_supported(int32_t head_dim, int32_t group) {
 
 bool generic_supported(int32_t head_dim) { return head_dim == 32 || head_dim == 64 || head_dim == 128; }
 
-int32_t tc_stages(int32_t head_dim, int32_t group, int32_t ctas_per_sm) {
-    if (!tc_supported(head_dim, group) || ctas_per_sm < 1) return 0;
+void tc_shape(int32_t head_dim, int32_t group, int32_t ctas_per_sm, int32_t* stages, int32_t* q_slots) {
+    *stages = *q_slots = 0;
+    if (!tc_supported(head_dim, group) || ctas_per_sm < 1) return;
     const bool two = group > 8;
-    if (head_dim == 128) return two ? tc_stages_inst<128, 2>(ctas_per_sm) : tc_stages_inst<128, 1>(ctas_per_sm);
-    return two ? tc_stages_inst<64, 2>(ctas_per_sm) : tc_stages_inst<64, 1>(ctas_per_sm);
+    if (head_dim == 128)
+        two ? tc_shape_inst<128, 2>(ctas_per_sm, stages, q_slots) : tc_shape_inst<128, 1>(ctas_per_sm, stages, q_slots);
+    else
+        two ? tc_shape_inst<64, 2>(ctas_per_sm, stages, q_slots) : tc_shape_inst<64, 1>(ctas_per_sm, stages, q_slots);
 }
 
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
