@@ -116,6 +116,31 @@ def kv_rows(seed: int, layer: int, req: int, kind: int, t0: int, t1: int,
     return x.view(t1 - t0, kv_heads, head_dim)
 
 
+def kv_rows_batch(seed: int, layer: int, reqs: Sequence[int], kind: int, t0: Sequence[int],
+                  t1: Sequence[int], kv_heads: int, head_dim: int, dtype: torch.dtype,
+                  device="cpu") -> torch.Tensor:
+    """kv_rows of several requests at once, concatenated in request order:
+    [sum(t1 - t0), kv_heads, head_dim].  Element for element equal to calling kv_rows per
+    request; one pass of the hash over all of them (many short runs cost one launch each
+    otherwise)."""
+    device = torch.device(device)
+    per_tok = kv_heads * head_dim
+    counts = [(int(b) - int(a)) * per_tok for a, b in zip(t0, t1)]
+    total = sum(counts)
+    if total == 0:
+        return torch.empty(0, kv_heads, head_dim, dtype=dtype, device=device)
+    seeds = torch.tensor([fold_key((seed, layer, int(r), kind)) for r in reqs], dtype=torch.int64)
+    cnt = torch.tensor(counts, dtype=torch.int64)
+    first = torch.tensor([int(a) * per_tok for a in t0], dtype=torch.int64)
+    run_start = torch.cumsum(cnt, 0) - cnt
+    s = torch.repeat_interleave(seeds, cnt).to(device)
+    idx = torch.arange(total, dtype=torch.int64, device=device) + torch.repeat_interleave(first - run_start, cnt).to(device)
+    lo = idx & _M32
+    hi = idx >> 32
+    h = _mix32(lo ^ _mix32(hi ^ s))
+    return _normal_table(dtype, device)[h & ((1 << _TABLE_BITS) - 1)].view(-1, kv_heads, head_dim)
+
+
 def q_rows(seed: int, layer: int, req: int, step: int, q_heads: int, head_dim: int,
            dtype: torch.dtype, device="cpu") -> torch.Tensor:
     """The query of one request at decode step `step`: [q_heads, head_dim]."""
