@@ -431,6 +431,38 @@ def run_ours(args):
         kernels_us = {"append": app_ms / max(app_n, 1) * 1e3, "decode": dec_ms / dec_n * 1e3,
                       "combine": cmb_ms / cmb_n * 1e3 if cmb_n else 0.0}
 
+    # ---- contiguity ablation: the same requests re-laid in 16-token pages (shuffled), same kernel
+    paged_line = None
+    if "paged" in phases:
+        host_len = [int(c) + 1 for c in w.context]
+        max_pages = max(-(-L // 16) for L in host_len)
+        n_pages = sum(-(-L // 16) for L in host_len) + 16
+        page_bytes = w.layers * 2 * w.kv_heads * 16 * row_bytes
+        pages = torch.empty(n_pages * page_bytes, dtype=torch.uint8, device=dev)
+        ptab = torch.zeros(n * max_pages, dtype=torch.int32, device=dev)
+        paged = odma.Paged(sd.pool, pages.data_ptr(), pages.numel())
+        paged.build(tables, host_len, 950900, ptab.data_ptr(), max_pages, sd.stream)
+        reps = max(3, min(K, 200)) if step_layers == 1 else 3
+        res = {}
+        for kind in ("slab", "paged"):
+            for timed in (False, True):
+                if timed:
+                    sd.pool.profile_enable(True)
+                for i in range(reps * step_layers):
+                    l = i % w.layers
+                    if kind == "slab":
+                        sd.pool.decode_attention(l, q[l].data_ptr(), w.q_heads, tables, out[l].data_ptr(), 0, sd.stream)
+                    else:
+                        paged.decode_attention(l, q[l].data_ptr(), w.q_heads, tables, ptab.data_ptr(), max_pages,
+                                               out[l].data_ptr(), 0, sd.stream)
+                torch.cuda.synchronize()
+            t_ms, cnt = sd.pool.profile_read(odma.K_DECODE)
+            sd.pool.profile_enable(False)
+            res[kind] = {"us_per_launch": t_ms / cnt * 1e3, "GBs": kv_bytes_per_launch / (t_ms / cnt * 1e-3) / 1e9}
+        assert sd.pool.check_status(sd.stream) == odma.OK
+        paged_line = {"pages": "16 tokens, ids shuffled", **res}
+        del pages, paged
+
     # ---- end to end from pinned host buffers ---------------------------------------------------
     e2e = None
     if "e2e" in phases:
@@ -486,6 +518,8 @@ def run_ours(args):
                        "ms_per_step": e2e_ms / e2e_steps}
     if roofline:
         line["roofline"], line["kernels_us"] = roofline, kernels_us
+    if paged_line:
+        line["page16_ablation"] = paged_line
     if clk:
         line["clocks"] = clk
     if rank == 0 and world == 1 and "cpu" in phases:
@@ -524,7 +558,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--phases", default="timed,kernels,e2e,clocks,cpu",
                     help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
-                         "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline)")
+                         "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
+                         "paged (page-16 ablation of the decode kernel on the same inputs)")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
     args = ap.parse_args()
     if args.warmup < 3:
