@@ -325,15 +325,36 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            const int it_begin = rec.x, it_end = rec.y;
-            uint32_t stage = 0, phase = 0;
-            uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
-            bool ok = true;
-            const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
-            const int64_t v_array = k_array + p.rows_per_array;
-            uint32_t qs = 0, qphase = 0;
-            for (int it = it_begin; ok; ++it) {
+        // Lane 0 issues every copy.  The other lanes only fetch item descriptors: 32 at a
+        // time, one per lane, handed to lane 0 by shuffles, so that the table reads of short
+        // items are off the issuing lane's critical path.
+        const int it_begin = __shfl_sync(0xFFFFFFFFu, rec.x, 0), it_end = __shfl_sync(0xFFFFFFFFu, rec.y, 0);
+        uint32_t stage = 0, phase = 0;
+        uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
+        bool ok = true;
+        const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
+        const int64_t v_array = k_array + p.rows_per_array;
+        uint32_t qs = 0, qphase = 0;
+        int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
+        for (int it = it_begin;; ++it) {
+            const int j = (it - it_begin) & 31;
+            if (j == 0 && it + lane < it_end) {
+                mine_a = __ldg(p.items + 2 * (it + lane));
+                mine_b = __ldg(p.items + 2 * (it + lane) + 1);
+            }
+            int4 a = first_a, b = first_b;               // the first item came with the CTA record
+            if (it != it_begin) {
+                a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
+                a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
+                a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
+                a.w = __shfl_sync(0xFFFFFFFFu, mine_a.w, j);
+                b.x = __shfl_sync(0xFFFFFFFFu, mine_b.x, j);
+                b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
+                b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
+                b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
+            }
+            int more = 0;
+            if (lane == 0) do {
                 ok = mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit);
                 if (!ok) break;
                 int* dsc = desc + qs * 8;
@@ -341,11 +362,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                     dsc[2] = 0;
                     mbar_arrive(qfull_bar(qs));
                     break;
-                }
-                int4 a = first_a, b = first_b;
-                if (it != it_begin) {
-                    a = __ldg(p.items + 2 * it);
-                    b = __ldg(p.items + 2 * it + 1);
                 }
                 const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
                 dsc[0] = req;
@@ -414,17 +430,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                         phase ^= 1u;
                     }
                 }
-            }
-            if (!ok) {
-                // Something timed out.  Before the CTA's shared memory can be handed to another
-                // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
-                for (uint32_t s = 0; s < STAGES; ++s)
-                    if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
-                        mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
-                                       limit / 4 + 1);
-            }
+                more = ok ? 1 : 0;
+            } while (false);
+            if (!__shfl_sync(0xFFFFFFFFu, more, 0)) break;
         }
-        __syncwarp();
+        if (lane == 0 && !ok) {
+            // Something timed out.  Before the CTA's shared memory can be handed to another
+            // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
+            for (uint32_t s = 0; s < STAGES; ++s)
+                if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
+                    mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
+                                   limit / 4 + 1);
+        }
         return;
     }
 
