@@ -78,7 +78,7 @@ class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
     def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0,
-                 per_sm: int = 1, fused: int = 1):
+                 fused: int = 1):
         from paper_2512_09427_b200 import odma
         self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
         self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
@@ -92,7 +92,7 @@ class SlabDecode:
         cfg.p_den = pd
         cfg.max_batch = max(1024, w.batch)
         cfg.plan_ctas = plan_ctas
-        cfg.ctas_per_sm, cfg.fused_combine = per_sm, fused
+        cfg.fused_combine = fused
         self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
         self.stream = torch.cuda.current_stream().cuda_stream
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
@@ -372,7 +372,7 @@ def run_ours(args):
     phases = set(args.phases.split(","))
     K, W = args.steps, args.warmup
     w, step_layers, copies = pick_workload(args.workload, rank, args.copies)
-    sd = SlabDecode(w, step_layers, dev)
+    sd = SlabDecode(w, step_layers, dev, fused=args.fused_combine)
     bounds, epoch = sd.learn_boundaries()
     sd.admit_and_fill()
     q, kn, vn, out = sd.make_inputs()
@@ -560,6 +560,7 @@ def main():
                     help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
                          "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
                          "paged (page-16 ablation of the decode kernel on the same inputs)")
+    ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -84,10 +84,8 @@ typedef struct odma_config {
     int32_t large_fixed;     /* 1: every Large Bucket slab has max_len tokens (0) */
     int32_t max_batch;       /* most requests per odma_build_tables call; sizes scratch (1024) */
     int32_t max_group;       /* most query heads per KV head; sizes scratch (8) */
-    int32_t plan_ctas;       /* persistent CTAs the split plan targets; 0 = ctas_per_sm per SM of
-                                the current device (148 SMs when the pool has no device memory) */
-    int32_t ctas_per_sm;     /* CTAs of the decode kernel resident on one SM: 1 or 2; sets the
-                                depth of each CTA's staging pipeline (1) */
+    int32_t plan_ctas;       /* persistent CTAs the split plan targets; 0 = one per SM of the
+                                current device (148 when the pool has no device memory) */
     int32_t fused_combine;   /* 1: the CTA that delivers the last piece of a split stream merges
                                 the pieces inside the decode kernel; 0: a separate combine kernel
                                 is launched after it (1) */

@@ -217,8 +217,7 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->q_heads = q_heads;
     p->kv_heads = pool->kv_heads;
     p->group = q_heads / pool->kv_heads;
-    tc_shape(pool->head_dim, p->group, pool->alloc.config().ctas_per_sm, &p->stages, &p->q_slots);
-    p->fin_warps = pool->alloc.config().ctas_per_sm == 1 ? 4 : 2;   // two CTAs share the register file
+    tc_shape(pool->head_dim, p->group, &p->stages, &p->q_slots);
     p->head_dim = pool->head_dim;
     p->scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(pool->head_dim)));
     p->status = pool->d_status;
@@ -259,7 +258,6 @@ void odma_config_default(odma_config* cfg) {
     cfg->max_batch = 1024;
     cfg->max_group = 8;
     cfg->plan_ctas = 0;
-    cfg->ctas_per_sm = 1;
     cfg->fused_combine = 1;
 }
 
@@ -289,7 +287,6 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
     if (layers < 1 || kv_heads < 1 || head_dim < 1 || (static_cast<int64_t>(head_dim) * esz) % 16 != 0)
         return ODMA_ERR_INVALID;
     if (cfg.max_batch < 1 || cfg.max_group < 1 || cfg.plan_ctas < 0) return ODMA_ERR_INVALID;
-    if (cfg.ctas_per_sm < 1 || cfg.ctas_per_sm > 2) return ODMA_ERR_INVALID;
     if (dev_base && (reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0) return ODMA_ERR_INVALID;
 
     odma_pool* p = new (std::nothrow) odma_pool();
@@ -311,7 +308,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
         delete p;
         return ODMA_ERR_INVALID;
     }
-    p->plan_ctas = cfg.plan_ctas > 0 ? cfg.plan_ctas : 148 * cfg.ctas_per_sm;
+    p->plan_ctas = cfg.plan_ctas > 0 ? cfg.plan_ctas : 148;
     if (dev_base) {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -319,7 +316,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
             delete p;
             return ODMA_ERR_CUDA;
         }
-        if (cfg.plan_ctas == 0) p->plan_ctas = sms * cfg.ctas_per_sm;
+        if (cfg.plan_ctas == 0) p->plan_ctas = sms;
     }
     p->slots_max = static_cast<int64_t>(cfg.max_batch) * kv_heads + p->plan_ctas;
     p->table_words_max = plan_table_words(cfg.max_batch, kv_heads, p->plan_ctas);

@@ -15,7 +15,6 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
-#include <type_traits>
 
 #include "odma.h"
 
@@ -140,12 +139,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // decode attention, tensor-core path (bf16, head_dim 64 or 128, group <= 16)
 // =============================================================================================
 //
-// Roles: warps 0..3 consume, warp 4 (one lane) produces, warps 5.. finish.  A pipeline stage
-// holds one tile of 64 keys and 64 values of one stream, written by TMA with the 128-byte
-// swizzle so that ldmatrix reads are conflict-free.  Consumer warp w owns keys [16w, 16w+16) of
-// every tile and keeps its own running (max, sum, output).  When an item ends the four warps
-// drop their partial results into one of two merge buffers and go straight on to the next
-// item; the finisher warps merge the four, write the item's result (or partial result) to
+// Roles: warps 0..7 consume (two groups of four), warp 8 produces, warps 9.. finish.  A
+// pipeline stage holds one tile of 64 keys and 64 values of one stream, written by TMA with the
+// 128-byte swizzle so that ldmatrix reads are conflict-free.  The CTA's items go to the two
+// consumer groups in turn (short items are latency chains; two in flight hide each other).
+// Warp w of a group owns keys [16w, 16w+16) of every tile of the group's item and keeps its own
+// running (max, sum, output).  When an item ends the four warps drop their partial results
+// into the group's merge buffer and go straight on to the group's next item; the finisher warps merge the four, write the item's result (or partial result) to
 // global memory and, for a split stream, count the piece in and merge all pieces if it was
 // the last one.  Queries and item descriptors travel through a ring of 4..8 slots so the
 // producer can run several short items ahead of the consumers.
@@ -160,12 +160,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // softmax weights go from the first product's accumulator to the second product's B operand
 // with one 8x8 register transpose (movmatrix) per eight keys.
 
-constexpr int kConsumerWarps = 4;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kFinisherWarp0 = kConsumerWarps + 1;
-constexpr int kMaxFinisherWarps = 4;              // 2 when two CTAs share an SM (register file)
-constexpr int kTcThreads = kConsumerThreads + 32 + kMaxFinisherWarps * 32;
+constexpr int kConsumerWarps = 4;                 // per consumer group: one tile is shared by four warps
+constexpr int kConsumerGroups = 2;                // items go to the groups in turn
+constexpr int kConsumerThreads = kConsumerGroups * kConsumerWarps * 32;
+constexpr int kProducerWarp = kConsumerGroups * kConsumerWarps;
+constexpr int kFinisherWarp0 = kProducerWarp + 1;
+constexpr int kFinisherWarps = 3;                 // 12 warps in all: three per scheduler, 168 registers each
+constexpr int kFinisherThreads = kFinisherWarps * 32;
+constexpr int kTcThreads = kConsumerThreads + 32 + kFinisherThreads;
 constexpr int kTile = 64;
 constexpr int kMaxStages = 8;
 constexpr int kMinQSlots = 4, kMaxQSlots = 8;
@@ -302,18 +304,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     if (tid == 0) {
         for (uint32_t s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
-            mbar_init(empty_bar(s), kConsumerWarps);
+            mbar_init(empty_bar(s), kConsumerGroups * kConsumerWarps);
         }
         for (uint32_t s = 0; s < QSLOTS; ++s) {
             mbar_init(qfull_bar(s), 1);
-            mbar_init(qempty_bar(s), kConsumerWarps);
+            mbar_init(qempty_bar(s), kConsumerGroups * kConsumerWarps);
         }
         for (uint32_t s = 0; s < kMergeBufs; ++s) {
             mbar_init(mready_bar(s), kConsumerWarps);
-            mbar_init(mdone_bar(s), p.fin_warps);
+            mbar_init(mdone_bar(s), kFinisherWarps);
         }
-        mbar_init(fstored_bar, p.fin_warps);
-        mbar_init(fcounted_bar, p.fin_warps);
+        mbar_init(fstored_bar, kFinisherWarps);
+        mbar_init(fcounted_bar, kFinisherWarps);
         *abort_flag = 0;
         *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -449,7 +451,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         // ------------------------------------------------------------------ finishers
         if (MODE == kModeProbe) return;
         const int ftid = tid - kFinisherWarp0 * 32;
-        const int fthreads = p.fin_warps * 32;
+        constexpr int fthreads = kFinisherThreads;
         const int n_items = __shfl_sync(0xFFFFFFFFu, rec.y - rec.x, 0);
         const int group = p.group;
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
@@ -457,8 +459,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         const int total = group * PER_ROW;
         // CH = chunks of four output elements per thread; every thread computes CH chunks
         // (indices past the end are clamped, their results dropped) so the code is branch-free
-        auto run = [&](auto ch_tag) {
-            constexpr int CH = decltype(ch_tag)::value;
+        constexpr int CH = (ROWS * PER_ROW + kFinisherThreads - 1) / kFinisherThreads;
+        {
             uint32_t n_split = 0;
             for (int k = 0; k < n_items; ++k) {
                 const uint32_t mb = static_cast<uint32_t>(k) & 1u;
@@ -579,12 +581,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                     if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + log2f(fl[i])) * 0.6931471805599453f;
                 }
             }
-        };
-        constexpr int CHUNKS4 = (ROWS * PER_ROW + 127) / 128;   // with four finisher warps
-        if (p.fin_warps == 4)
-            run(std::integral_constant<int, CHUNKS4>{});
-        else
-            run(std::integral_constant<int, 2 * CHUNKS4>{});
+        }
         return;
     }
 
@@ -592,15 +589,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     const int qd = lane >> 2, qt = lane & 3;          // row within 8, position within the quad
     const int mi = lane >> 3, r8 = lane & 7;          // ldmatrix: matrix id, row within it
     // K tile as the A operand: matrices (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15)
-    const uint32_t k_lane_off = (warp * 16 + (mi & 1) * 8 + r8) * 128;
+    const int cw = warp & (kConsumerWarps - 1);       // warp within its group
+    const uint32_t grp = static_cast<uint32_t>(warp) / kConsumerWarps;
+    const uint32_t k_lane_off = (cw * 16 + (mi & 1) * 8 + r8) * 128;
     const uint32_t xk = (mi >> 1) ^ r8;
     // V tile, transposed on load, as the A operand: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
-    const uint32_t v_lane_off = (warp * 16 + (mi >> 1) * 8 + r8) * 128;
+    const uint32_t v_lane_off = (cw * 16 + (mi >> 1) * 8 + r8) * 128;
     const uint32_t xv = (mi & 1) ^ r8;
     // Q as the B operand: four consecutive 16-byte chunks of head r8
     const uint32_t q_lane_off = r8 * (D * 2) + mi * 16;
-    const int key_lo = warp * 16 + qd;                // the thread's two key rows: key_lo, key_lo + 8
-    const int vkey0 = warp * 16 + qt * 2;             // keys of its value fragments: vkey0, +1, +8, +9
+    const int key_lo = cw * 16 + qd;                // the thread's two key rows: key_lo, key_lo + 8
+    const int vkey0 = cw * 16 + qt * 2;             // keys of its value fragments: vkey0, +1, +8, +9
     const float scale = p.scale_log2;
 
     uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
@@ -611,6 +610,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         const int* dsc = desc + qs * 8;
         const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3], slot = dsc[4], comb = dsc[5];
         if (ntok == 0) break;
+        const int ntiles = (ntok + kTile - 1) / kTile;
+        if ((k_item & 1u) != grp) {
+            // The other group's item: let go of the slot and walk over its tiles in step with
+            // the ring.  A barrier's parity tells apart only two consecutive phases, so neither
+            // group may fall a whole phase behind or run one ahead of any stage: every warp of
+            // both groups waits for each tile to land and signs the stage off, the owners after
+            // using it, the others at once.
+            __syncwarp();
+            if (lane == 0) mbar_arrive(qempty_bar(qs));
+            if (++qs == QSLOTS) {
+                qs = 0;
+                qphase ^= 1u;
+            }
+            for (int t = 0; t < ntiles; ++t) {
+                ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, limit);
+                if (!ok) break;
+                if (lane == 0) mbar_arrive(empty_bar(stage));
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            continue;
+        }
 
         uint32_t qb[NT][D / 16][2];
         if (MODE != kModeProbe) {
@@ -643,12 +666,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             l_run[nt][0] = l_run[nt][1] = 0.f;
         }
 
-        const int ntiles = (ntok + kTile - 1) / kTile;
         for (int t = 0; t < ntiles; ++t) {
             ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, limit);
             if (!ok) break;
             const int valid = min(kTile, ntok - t * kTile);
-            if (MODE != kModeProbe && warp * 16 < valid) {
+            if (MODE != kModeProbe && cw * 16 < valid) {
                 const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
                 const uint32_t vbase = kbase + Cfg::kKvTileBytes;
                 // ---- S^T = K Q^T for this warp's 16 keys; two accumulators shorten the chain
@@ -747,13 +769,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 l_run[nt][0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][0], off);
                 l_run[nt][1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][1], off);
             }
-        const uint32_t mb = k_item & 1u;
+        const uint32_t mb = k_item & 1u;              // = grp: each group has its own buffer
         if (k_item >= 2) {                            // the finishers are done with item k_item - 2
             ok = mbar_wait(mdone_bar(mb), ((k_item >> 1) - 1u) & 1u, abort_flag, p.status, limit);
             if (!ok) break;
         }
-        float* mo = mrg_o + mb * Cfg::kMergeFloats + warp * ROWS * MO;
-        float* mml = mrg_ml + mb * Cfg::kMlFloats + warp * ROWS * 2;
+        float* mo = mrg_o + mb * Cfg::kMergeFloats + cw * ROWS * MO;
+        float* mml = mrg_ml + mb * Cfg::kMlFloats + cw * ROWS * 2;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int h0 = nt * 8 + qt * 2;
@@ -772,7 +794,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 mml[h0 * 2 + 3] = l_run[nt][1];
             }
         }
-        if (tid == 0) {
+        if (cw == 0 && lane == 0) {
             int* hdr = mrg_hdr + mb * 8;
             hdr[0] = req;
             hdr[1] = head;
@@ -1072,14 +1094,14 @@ cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_
     auto kern = decode_tc_kernel<D, NT, MODE>;
     const int smem = Cfg::smem_bytes(p.stages, p.q_slots);
     if (p.stages < 2 || p.stages > kMaxStages || p.q_slots < kMinQSlots || p.q_slots > kMaxQSlots ||
-        smem > kSmemPerCtaMax || (p.fin_warps != 2 && p.fin_warps != kMaxFinisherWarps))
+        smem > kSmemPerCtaMax)
         return cudaErrorInvalidValue;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<n_ctas, kConsumerThreads + 32 + p.fin_warps * 32, smem, stream>>>(maps.big, maps.small, p);
+    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p);
     return cudaGetLastError();
 }
 
@@ -1130,9 +1152,10 @@ bool tc_supported(int32_t head_dim, int32_t group) {
 
 bool generic_supported(int32_t head_dim) { return head_dim == 32 || head_dim == 64 || head_dim == 128; }
 
-void tc_shape(int32_t head_dim, int32_t group, int32_t ctas_per_sm, int32_t* stages, int32_t* q_slots) {
+void tc_shape(int32_t head_dim, int32_t group, int32_t* stages, int32_t* q_slots) {
+    const int32_t ctas_per_sm = 1;
     *stages = *q_slots = 0;
-    if (!tc_supported(head_dim, group) || ctas_per_sm < 1) return;
+    if (!tc_supported(head_dim, group)) return;
     const bool two = group > 8;
     if (head_dim == 128)
         two ? tc_shape_inst<128, 2>(ctas_per_sm, stages, q_slots) : tc_shape_inst<128, 1>(ctas_per_sm, stages, q_slots);

@@ -39,7 +39,6 @@ struct DecodeParams {
     int64_t wait_limit_ns;
     int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
-    int32_t fin_warps;          // its finisher warps: 4, or 2 when two CTAs share an SM
 };
 
 struct TensorMaps {
@@ -51,9 +50,9 @@ enum DecodeMode { kModeSlab = 0, kModePaged = 1, kModeProbe = 2 };
 
 // Returns false when (head_dim, group) has no tensor-core instantiation.
 bool tc_supported(int32_t head_dim, int32_t group);
-// Pipeline stages and query-ring slots that fit when `ctas_per_sm` CTAs share one SM's shared
-// memory (both 0 when nothing fits).
-void tc_shape(int32_t head_dim, int32_t group, int32_t ctas_per_sm, int32_t* stages, int32_t* q_slots);
+// Pipeline stages and query-ring slots that fit into one SM's shared memory (one CTA per SM;
+// both 0 when nothing fits).
+void tc_shape(int32_t head_dim, int32_t group, int32_t* stages, int32_t* q_slots);
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
                              cudaStream_t stream);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);

@@ -65,100 +65,202 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     }
     table[t.off_cu_new + n] = cu;
 
-    // Cut points.  Shares are equal in COST, not in tiles: starting a stream (its query, its
-    // first rows in a new part of memory, its merge at the end) costs about as much as
-    // streaming kStreamCostTiles more tiles, so a stream of `per` tiles weighs per +
-    // kStreamCostTiles.  A cut that falls into a stream's start-up part moves to the stream's
-    // start, one that falls inside a short stream moves to its nearer end.
-    std::vector<int64_t> first_cost(static_cast<size_t>(n) + 1, 0);
-    for (int32_t i = 0; i < n; ++i)
-        first_cost[i + 1] = first_cost[i] + ((first_tile[i + 1] - first_tile[i]) / hkv + kStreamCostTiles) * hkv;
-    const int64_t total_cost = first_cost[n];
-    std::vector<int64_t> cut(static_cast<size_t>(ctas) + 1);
-    cut[0] = 0;
-    cut[ctas] = total;
-    int32_t req = 0;
-    for (int32_t c = 1; c < ctas; ++c) {
-        const int64_t xc = total_cost * c / ctas;
-        while (first_cost[req + 1] <= xc) ++req;                    // request holding cost unit xc
-        const int64_t per = (first_tile[req + 1] - first_tile[req]) / hkv;   // tiles per stream
-        const int64_t per_cost = per + kStreamCostTiles;
-        const int64_t sh = (xc - first_cost[req]) / per_cost;       // stream of that request
-        const int64_t off = (xc - first_cost[req]) - sh * per_cost - kStreamCostTiles;
-        const int64_t s0 = first_tile[req] + sh * per, s1 = s0 + per;
-        int64_t x = s0 + std::max<int64_t>(off, 0);
-        if (per <= kSnapTiles) x = (x - s0 <= s1 - x) ? s0 : s1;
-        cut[c] = std::max(x, cut[c - 1]);
-    }
+    // Shares.  The streams are dealt into at most `ctas` shares of (nearly) equal COST:
+    //   * a tile of 64 tokens costs 1;
+    //   * starting a stream (its query, its first rows in a new part of memory, handing its
+    //     result over) costs kStreamCostTiles;
+    //   * a piece of a split stream costs kSplitCostTiles on top: its partial result goes
+    //     through global memory and the CTA that delivers the last piece merges them all, a
+    //     chain of dependent round trips that a CTA ending on such a piece cannot hide.
+    // With capacity C = the average cost per share: "long" streams fill one share after the
+    // other, whole where they fit, cut where they do not (no piece shorter than
+    // kMinPieceTiles); every other stream goes whole, longest first, to the share with the
+    // least load so far (small streams level the shares out).  Long means longer than a share;
+    // if that leaves shares overfilled (many streams of between half a share and a share, which
+    // do not pack), the plan is redone with long = longer than half a share.
+    std::vector<int32_t> order(static_cast<size_t>(n));
+    for (int32_t i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return in.len[x] > in.len[y]; });
 
-    // walk the tile sequence once, emitting one piece per (share, stream) overlap, in stream
-    // order; a piece's slot (where its partial result goes) is its index in that order
-    struct Piece { int32_t w[8]; };
+    struct Piece { int32_t w[8]; int32_t share; };
     std::vector<Piece> pieces;
-    std::vector<int32_t> share_begin(static_cast<size_t>(ctas) + 1, 0);
     std::vector<int32_t> comb;      // {req, head, first_slot, n_slots}
-    int32_t r = 0, head = 0;
-    int64_t stream_lo = 0;          // first tile of the current stream
-    int64_t pos = 0;
-    int32_t stream_first = 0;
-    for (int32_t c = 0; c < ctas; ++c) {
-        share_begin[c] = static_cast<int32_t>(pieces.size());
-        while (pos < cut[c + 1]) {
-            const int64_t per = (in.len[r] + kTileTokens - 1) / kTileTokens;
-            const int64_t stream_hi = stream_lo + per;
-            const int64_t end = std::min(stream_hi, cut[c + 1]);
-            const int64_t tok0 = (pos - stream_lo) * kTileTokens;
-            const int64_t tok1 = std::min<int64_t>((end - stream_lo) * kTileTokens, in.len[r]);
-            const int32_t k = static_cast<int32_t>(pieces.size());
+    std::vector<int64_t> load;
+    // deal(C, false) cuts the long streams only and returns the number of pieces (-1: more
+    // than `ctas` shares needed); deal(C, true) emits the whole plan.
+    auto deal = [&](int64_t C, bool emit, int64_t long_div) -> int64_t {
+        int64_t n_cut = 0;
+        load.assign(static_cast<size_t>(ctas), 0);
+        int32_t fresh = 0;          // the share that pieces of long streams are filling
+        if (emit) {
+            pieces.clear();
+            comb.clear();
+        }
+        auto put = [&](int32_t r, int32_t head, int64_t tile0, int64_t ntiles, bool whole, int32_t share) {
+            if (!emit) return;
+            const int64_t tok0 = tile0 * kTileTokens;
+            const int64_t tok1 = std::min<int64_t>((tile0 + ntiles) * kTileTokens, in.len[r]);
             Piece pc;
             pc.w[0] = r;
             pc.w[1] = head;
             pc.w[2] = static_cast<int32_t>(tok0);
             pc.w[3] = static_cast<int32_t>(tok1 - tok0);
-            pc.w[4] = (pos == stream_lo && end == stream_hi) ? 1 : 0;    // whole stream: direct
-            pc.w[5] = k;                                                 // slot
+            pc.w[4] = whole ? 1 : 0;
+            pc.w[5] = static_cast<int32_t>(pieces.size());       // slot
             // first row of the piece inside one K (or V) array of the pool
             pc.w[6] = static_cast<int32_t>(static_cast<int64_t>(in.base[r]) * hkv +
                                            static_cast<int64_t>(head) * in.cap[r] + tok0);
-            pc.w[7] = -1;                                                // combine record, set below
-            if (pos == stream_lo) stream_first = k;
+            pc.w[7] = -1;                                          // combine record, set below
+            pc.share = share;
             pieces.push_back(pc);
-            pos = end;
-            if (end == stream_hi) {                                      // stream finished
-                const int32_t n_pieces = static_cast<int32_t>(pieces.size()) - stream_first;
-                if (n_pieces > 1) {
-                    const int32_t ci = static_cast<int32_t>(comb.size() / 4);
-                    for (int32_t j = stream_first; j < stream_first + n_pieces; ++j) pieces[j].w[7] = ci;
-                    comb.push_back(r);
-                    comb.push_back(head);
-                    comb.push_back(stream_first);
-                    comb.push_back(n_pieces);
+        };
+        auto record_split = [&](int32_t r, int32_t head, int32_t first_slot) {
+            const int32_t n_pieces = static_cast<int32_t>(pieces.size()) - first_slot;
+            const int32_t ci = static_cast<int32_t>(comb.size() / 4);
+            for (int32_t j = first_slot; j < first_slot + n_pieces; ++j) pieces[j].w[7] = ci;
+            comb.push_back(r);
+            comb.push_back(head);
+            comb.push_back(first_slot);
+            comb.push_back(n_pieces);
+        };
+        // long streams first (the order is by length), filling one share after the other; a
+        // stream's last piece leaves room that the next stream, or short streams later, take
+        int32_t oi = 0;
+        for (; oi < n; ++oi) {
+            const int32_t r = order[oi];
+            const int64_t per = (in.len[r] + kTileTokens - 1) / kTileTokens;
+            if (long_div * (per + kStreamCostTiles) <= C || per < 2 * kMinPieceTiles) break;
+            for (int32_t head = 0; head < hkv; ++head) {
+                if (fresh < ctas && load[fresh] + per + kStreamCostTiles <= C) {     // fits whole
+                    put(r, head, 0, per, true, fresh);
+                    load[fresh] += per + kStreamCostTiles;
+                    continue;
                 }
-                stream_lo = stream_hi;
-                if (++head == hkv) {
-                    head = 0;
-                    ++r;
+                const int32_t first_slot = static_cast<int32_t>(pieces.size());
+                int64_t done = 0;
+                while (done < per) {
+                    if (fresh >= ctas) return -1;
+                    const int64_t extra = kSplitCostTiles + (done == 0 ? kStreamCostTiles : 0);
+                    int64_t room = C - load[fresh] - extra;
+                    if (room < kMinPieceTiles && load[fresh] > 0) {          // this share is full
+                        ++fresh;
+                        continue;
+                    }
+                    int64_t take = std::min(std::max<int64_t>(room, 1), per - done);
+                    if (per - done - take > 0 && per - done - take < kMinPieceTiles)
+                        take = std::max<int64_t>(1, per - done - kMinPieceTiles);   // no crumbs
+                    put(r, head, done, take, false, fresh);
+                    ++n_cut;
+                    load[fresh] += take + extra;
+                    done += take;
+                    if (done < per) ++fresh;
+                }
+                if (emit) {
+                    if (static_cast<int32_t>(pieces.size()) - first_slot > 1)
+                        record_split(r, head, first_slot);
+                    else
+                        pieces[first_slot].w[4] = 1;       // moved to a fresh share and fitted whole
                 }
             }
         }
+        if (!emit) return n_cut;
+        // every other stream whole, longest first, to the least loaded share: shares are kept
+        // in buckets by load (loads are small integers), the least loaded bucket is found by
+        // a pointer that only moves up
+        int64_t top = 0;
+        for (int32_t c = 0; c < ctas; ++c) top = std::max(top, load[c]);
+        std::vector<std::vector<int32_t>> bucket(static_cast<size_t>(top) + 2);
+        for (int32_t c = ctas - 1; c >= 0; --c) bucket[static_cast<size_t>(load[c])].push_back(c);
+        size_t lo = 0;
+        auto least = [&]() {
+            while (bucket[lo].empty()) ++lo;
+            const int32_t c = bucket[lo].back();
+            bucket[lo].pop_back();
+            return c;
+        };
+        auto back = [&](int32_t c) {
+            if (static_cast<size_t>(load[c]) >= bucket.size()) bucket.resize(static_cast<size_t>(load[c]) + 1);
+            bucket[static_cast<size_t>(load[c])].push_back(c);
+        };
+        for (; oi < n; ++oi) {
+            const int32_t r = order[oi];
+            const int64_t per = (in.len[r] + kTileTokens - 1) / kTileTokens;
+            for (int32_t head = 0; head < hkv; ++head) {
+                int32_t c = least();
+                if (load[c] == 0 || load[c] + per + kStreamCostTiles <= C + kSlackTiles || per < 2 * kMinPieceTiles) {
+                    put(r, head, 0, per, true, c);
+                    load[c] += per + kStreamCostTiles;
+                    back(c);
+                    continue;
+                }
+                // it would overfill even the least loaded share: cut it over the least loaded ones
+                const int32_t first_slot = static_cast<int32_t>(pieces.size());
+                int64_t done = 0;
+                while (done < per) {
+                    const int64_t extra = kSplitCostTiles + (done == 0 ? kStreamCostTiles : 0);
+                    const int64_t room = C - load[c] - extra;
+                    int64_t take = per - done;
+                    if (room >= std::max<int64_t>(kMinPieceTiles, per / 2) && room < take) {   // two pieces at most
+                        take = room;
+                        if (per - done - take < kMinPieceTiles) take = std::max<int64_t>(1, per - done - kMinPieceTiles);
+                    }
+                    put(r, head, done, take, false, c);
+                    load[c] += take + extra;
+                    back(c);
+                    done += take;
+                    if (done < per) c = least();
+                }
+                if (static_cast<int32_t>(pieces.size()) - first_slot > 1)
+                    record_split(r, head, first_slot);
+                else
+                    pieces[first_slot].w[4] = 1;       // no share had room for a piece: whole after all
+            }
+        }
+        return n_cut;
+    };
+    int64_t cost = 0;
+    for (int32_t i = 0; i < n; ++i)
+        cost += ((in.len[i] + kTileTokens - 1) / kTileTokens + kStreamCostTiles) * hkv;
+    // the capacity is the average cost per share, split costs included (a few rounds: the
+    // number of pieces depends on the capacity)
+    for (int64_t long_div = 1; long_div <= 2; ++long_div) {
+        // the capacity is the average cost per share, split costs included (a few rounds: the
+        // number of pieces depends on the capacity)
+        int64_t C = std::max<int64_t>((cost + ctas - 1) / ctas, 1 + kStreamCostTiles);
+        for (int round = 0; round < 64; ++round) {
+            const int64_t n_cut = deal(C, false, long_div);
+            const int64_t want = n_cut < 0 ? C + C / 128 + 1 : (cost + n_cut * kSplitCostTiles + ctas - 1) / ctas;
+            if (n_cut >= 0 && want <= C) break;
+            C = std::max(want, C + 1);
+        }
+        if (deal(C, true, long_div) < 0) return ODMA_ERR_INVALID;
+        int64_t worst = 0;
+        for (int32_t c = 0; c < ctas; ++c) worst = std::max(worst, load[c]);
+        if (worst <= C + kSlackTiles + C / 16) break;
     }
-    share_begin[ctas] = static_cast<int32_t>(pieces.size());
     const int32_t n_items = static_cast<int32_t>(pieces.size());
 
-    // Each CTA works through the pieces of split streams first (at most its first and its last
-    // piece), then through the whole streams: partial results are delivered early, so the
-    // merge of a split stream overlaps with streaming instead of trailing the kernel.
-    int32_t out_i = 0;
-    for (int32_t c = 0; c < ctas; ++c) {
+    // Group the pieces by share.  Each CTA works through its pieces of split streams first,
+    // then through the whole streams: partial results are delivered early, so the merge of a
+    // split stream overlaps with streaming instead of trailing the kernel.
+    std::vector<int32_t> count(static_cast<size_t>(ctas) + 1, 0);
+    for (const Piece& pc : pieces) ++count[pc.share + 1];
+    int32_t used = 0;
+    for (int32_t c = 0; c < ctas; ++c)
+        if (count[c + 1] > 0) used = c + 1;
+    std::vector<int32_t> at(static_cast<size_t>(ctas) + 1, 0);
+    for (int32_t c = 0; c < ctas; ++c) at[c + 1] = at[c] + count[c + 1];
+    std::vector<int32_t> fill(at.begin(), at.end() - 1);
+    for (int pass = 0; pass < 2; ++pass)
+        for (const Piece& pc : pieces)
+            if ((pc.w[4] == 0) == (pass == 0)) {
+                std::copy(pc.w, pc.w + 8, items + 8 * fill[pc.share]);
+                ++fill[pc.share];
+            }
+    for (int32_t c = 0; c < used; ++c) {
         int32_t* rec = table + t.off_cta + kCtaWords * c;
-        rec[0] = out_i;
-        for (int pass = 0; pass < 2; ++pass)
-            for (int32_t k = share_begin[c]; k < share_begin[c + 1]; ++k)
-                if ((pieces[k].w[4] == 0) == (pass == 0)) {
-                    std::copy(pieces[k].w, pieces[k].w + 8, items + 8 * out_i);
-                    ++out_i;
-                }
-        rec[1] = out_i;
+        rec[0] = at[c];
+        rec[1] = at[c + 1];
         rec[2] = rec[3] = 0;
         // a copy of the CTA's first item rides in its record: one load starts its stream
         for (int k = 0; k < 8; ++k) rec[4 + k] = rec[0] < rec[1] ? items[8 * rec[0] + k] : 0;
@@ -172,7 +274,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     t.n = n;
     t.n_new_total = cu;
     t.n_items = n_items;
-    t.n_ctas = ctas;
+    t.n_ctas = used;
     t.n_combine = static_cast<int32_t>(comb.size() / 4);
     t.words = w;
     t.tile_tokens = kTileTokens;
