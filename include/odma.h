@@ -89,6 +89,10 @@ typedef struct odma_config {
     int32_t fused_combine;   /* 1: the CTA that delivers the last piece of a split stream merges
                                 the pieces inside the decode kernel; 0: a separate combine kernel
                                 is launched after it (1) */
+    int32_t fused_append;    /* 1: odma_decode_step / odma_decode_step_host let the bf16 decode
+                                kernel take the step's new token from k_new / v_new and write
+                                it into the slab itself (one launch per layer); 0: they launch
+                                the append kernel first (1) */
 } odma_config;
 
 typedef struct odma_slab {
@@ -115,7 +119,8 @@ typedef struct odma_stats {
  *   the tokens appended this step), cta[n_ctas][12], items[n_items][8], combine[n_combine][4].
  *   cta     = {item_begin, item_end, 0, 0, copy of items[item_begin]}: CTA c works through
  *             items [item_begin, item_end), pieces of split streams first
- *   item    = {request, kv_head, first_token, n_tokens, direct(1)|partial(0), slot,
+ *   item    = {request, kv_head, first_token, n_tokens, flags (bit 0: the piece is the whole
+ *              stream, written out directly; bit 1: the piece ends its stream), slot,
  *              first row of the piece inside one K/V array, combine record (-1 if direct)};
  *             slots number all pieces in (request, head, token) order
  *   combine = {request, kv_head, first_slot, n_slots}

@@ -221,6 +221,8 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->head_dim = pool->head_dim;
     p->scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(pool->head_dim)));
     p->status = pool->d_status;
+    p->k_new = nullptr;
+    p->v_new = nullptr;
     p->page_table = nullptr;
     p->max_pages = 0;
     p->wait_limit_ns = kDefaultWaitLimitNs;
@@ -259,6 +261,7 @@ void odma_config_default(odma_config* cfg) {
     cfg->max_group = 8;
     cfg->plan_ctas = 0;
     cfg->fused_combine = 1;
+    cfg->fused_append = 1;
 }
 
 const char* odma_strerror(int32_t code) {
@@ -482,12 +485,30 @@ int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables
     return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
 
-int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
-                              const odma_tables* tables, void* out, float* lse, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// True when the bf16 tensor-core kernel serves this pool and group size (the kernel that can
+// take the step's append along).
+bool uses_tc(const odma_pool* pool, int32_t q_heads) {
+    return pool->has_maps && tc_supported(pool->head_dim, q_heads / pool->kv_heads);
+}
+
+// odma_decode_attention; with k_new / v_new the tensor-core kernel also appends the step's
+// token (one per request) instead of finding it in the slab.
+int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                              const odma_tables* tables, void* out, float* lse, void* stream,
+                              const void* k_new, const void* v_new) {
     int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
     if (rc != ODMA_OK) return rc;
     DecodeParams p;
     fill_decode_params(pool, layer, q, q_heads, tables, out, lse, &p);
+    if (k_new) {
+        if (!uses_tc(pool, q_heads) || !tables->one_new_each || !v_new) return ODMA_ERR_INVALID;
+        p.k_new = k_new;
+        p.v_new = v_new;
+    }
     cudaError_t e;
     bool fused = false;
     {
@@ -515,6 +536,15 @@ int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int
     return ODMA_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
+                              const odma_tables* tables, void* out, float* lse, void* stream) {
+    return decode_attention_impl(pool, layer, q, q_heads, tables, out, lse, stream, nullptr, nullptr);
+}
+
 int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
                               int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
                               void* h_out, void* stream) {
@@ -533,9 +563,13 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
         cudaMemcpyAsync(pool->d_k_new, h_k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
         cudaMemcpyAsync(pool->d_v_new, h_v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return ODMA_ERR_CUDA;
-    rc = odma_append_kv(pool, layer, &t, pool->d_k_new, pool->d_v_new, stream);
-    if (rc != ODMA_OK) return rc;
-    rc = odma_decode_attention(pool, layer, pool->d_q, q_heads, &t, pool->d_out, nullptr, stream);
+    const bool fuse = pool->alloc.config().fused_append && uses_tc(pool, q_heads);
+    if (!fuse) {
+        rc = odma_append_kv(pool, layer, &t, pool->d_k_new, pool->d_v_new, stream);
+        if (rc != ODMA_OK) return rc;
+    }
+    rc = decode_attention_impl(pool, layer, pool->d_q, q_heads, &t, pool->d_out, nullptr, stream,
+                               fuse ? pool->d_k_new : nullptr, fuse ? pool->d_v_new : nullptr);
     if (rc != ODMA_OK) return rc;
     if (cudaMemcpyAsync(h_out, pool->d_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return ODMA_ERR_CUDA;
@@ -554,13 +588,20 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
     if (rc != ODMA_OK) return rc;
     const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
     const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    // on the tensor-core path the append rides in the decode kernel: one launch per layer
+    const bool fuse = pool->alloc.config().fused_append && q_heads >= pool->kv_heads &&
+                      q_heads % pool->kv_heads == 0 && uses_tc(pool, q_heads) && aligned16(d_k_new) && aligned16(d_v_new);
     for (int32_t l = 0; l < n_layers; ++l) {
-        rc = odma_append_kv(pool, layer + l, &t, static_cast<const uint8_t*>(d_k_new) + l * kb,
-                            static_cast<const uint8_t*>(d_v_new) + l * kb, stream);
-        if (rc != ODMA_OK) return rc;
-        rc = odma_decode_attention(pool, layer + l, static_cast<const uint8_t*>(d_q) + l * qb, q_heads, &t,
+        const uint8_t* kn = static_cast<const uint8_t*>(d_k_new) + l * kb;
+        const uint8_t* vn = static_cast<const uint8_t*>(d_v_new) + l * kb;
+        if (!fuse) {
+            rc = odma_append_kv(pool, layer + l, &t, kn, vn, stream);
+            if (rc != ODMA_OK) return rc;
+        }
+        rc = decode_attention_impl(pool, layer + l, static_cast<const uint8_t*>(d_q) + l * qb, q_heads, &t,
                                    static_cast<uint8_t*>(d_out) + l * qb,
-                                   lse ? lse + static_cast<size_t>(l) * n * q_heads : nullptr, stream);
+                                   lse ? lse + static_cast<size_t>(l) * n * q_heads : nullptr, stream,
+                                   fuse ? kn : nullptr, fuse ? vn : nullptr);
         if (rc != ODMA_OK) return rc;
     }
     if (tables_out) *tables_out = t;

@@ -361,17 +361,23 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 if (!ok) break;
                 int* dsc = desc + qs * 8;
                 if (it >= it_end) {                      // end marker
-                    dsc[2] = 0;
+                    dsc[6] = 0;
                     mbar_arrive(qfull_bar(qs));
                     break;
                 }
-                const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
+                const int req = a.x, head = a.y, tok0 = a.z;
                 dsc[0] = req;
                 dsc[1] = head;
+                // With the append fused in, the stream's last token is not in the slab yet: it
+                // is not streamed; the finishers take it from k_new / v_new and write it there.
+                const bool has_new = p.k_new != nullptr && (b.x & 2);
+                const int ntok = a.w - (has_new ? 1 : 0);
                 dsc[2] = ntok;
-                dsc[3] = b.x;     // direct
-                dsc[4] = b.y;     // slot
-                dsc[5] = b.w;     // combine record
+                dsc[3] = b.x & 1;                        // direct
+                dsc[4] = b.y;                            // slot
+                dsc[5] = b.w;                            // combine record
+                dsc[6] = 1;                              // a real item
+                dsc[7] = has_new ? b.z + ntok : -1;      // pool row of the new token
                 const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
                 mbar_expect_tx(qfull_bar(qs), q_bytes);
                 bulk_load(q_u32 + qs * Cfg::kQBytes,
@@ -507,6 +513,40 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                     acc_m[i] = M;
                     acc_l[i] = L;
                 }
+                const int new_row = hdr[5];
+                if (new_row >= 0) {
+                    // the token appended this step: its score against each head from k_new
+                    // (lanes that share a head add their parts up), its value from v_new; then
+                    // its K and V rows go into the slab for the steps to come
+                    const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(p.q) +
+                                                (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group) * D;
+                    const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D;
+                    const __nv_bfloat16* krow = reinterpret_cast<const __nv_bfloat16*>(p.k_new) + nrow;
+                    const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(p.v_new) + nrow;
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) {
+                        const uint2 qv = __ldg(reinterpret_cast<const uint2*>(qrow + rr[i] * D + dd[i]));
+                        const uint2 kv2 = __ldg(reinterpret_cast<const uint2*>(krow + dd[i]));
+                        const uint2 vv = __ldg(reinterpret_cast<const uint2*>(vrow + dd[i]));
+                        float dot = __uint_as_float(qv.x << 16) * __uint_as_float(kv2.x << 16);
+                        dot = fmaf(__uint_as_float(qv.x & 0xFFFF0000u), __uint_as_float(kv2.x & 0xFFFF0000u), dot);
+                        dot = fmaf(__uint_as_float(qv.y << 16), __uint_as_float(kv2.y << 16), dot);
+                        dot = fmaf(__uint_as_float(qv.y & 0xFFFF0000u), __uint_as_float(kv2.y & 0xFFFF0000u), dot);
+#pragma unroll
+                        for (int off = PER_ROW / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
+                        const float4 x = make_float4(__uint_as_float(vv.x << 16), __uint_as_float(vv.x & 0xFFFF0000u),
+                                                     __uint_as_float(vv.y << 16), __uint_as_float(vv.y & 0xFFFF0000u));
+                        lse_fold(acc_m[i], acc_l[i], acc[i], dot * p.scale_log2, 1.f, x);
+                    }
+                    constexpr int ROW_VECS = D * 2 / 16;
+                    if (ftid < 2 * ROW_VECS) {
+                        const int kv = ftid / ROW_VECS, vec = ftid - kv * ROW_VECS;
+                        const uint4* src = reinterpret_cast<const uint4*>((kv ? vrow : krow)) + vec;
+                        uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
+                                     ((static_cast<int64_t>(p.layer) * 2 + kv) * p.rows_per_array + new_row) * ROW_VECS + vec;
+                        *dst = __ldg(src);
+                    }
+                }
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
                     if (ftid + i * fthreads >= total) continue;
@@ -609,7 +649,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         if (!ok) break;
         const int* dsc = desc + qs * 8;
         const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3], slot = dsc[4], comb = dsc[5];
-        if (ntok == 0) break;
+        const int new_row = dsc[7];
+        if (dsc[6] == 0) break;
         const int ntiles = (ntok + kTile - 1) / kTile;
         if ((k_item & 1u) != grp) {
             // The other group's item: let go of the slot and walk over its tiles in step with
@@ -801,6 +842,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
             hdr[2] = direct;
             hdr[3] = slot;
             hdr[4] = comb;
+            hdr[5] = new_row;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(mready_bar(mb));
@@ -865,7 +907,7 @@ decode_generic_kernel(const DecodeParams p) {
     const int4 rec = __ldg(p.cta + 3 * cta);
     for (int it = rec.x; it < rec.y; ++it) {
         const int4 a = p.items[2 * it], b = p.items[2 * it + 1];
-        const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w, direct = b.x, slot = b.y;
+        const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w, direct = b.x & 1, slot = b.y;
         const int64_t row0 = static_cast<int64_t>(p.base[req]) * p.kv_heads +
                              static_cast<int64_t>(head) * p.cap[req] + tok0;
         const T* K = pool + (static_cast<int64_t>(p.layer) * 2 * p.rows_per_array + row0) * D;

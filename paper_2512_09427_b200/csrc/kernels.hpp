@@ -28,6 +28,8 @@ struct DecodeParams {
     float* part_o;              // [slots, group, head_dim] unnormalised partial outputs
     float* part_ml;             // [slots, group, 2] running max (log2 domain) and sum
     const void* pool;           // base of the slab pool (or of the paged copy)
+    const void* k_new;          // append fused into the decode kernel: the step's new rows,
+    const void* v_new;          // [n, kv_heads, head_dim], one token per request; nullptr = not fused
     int64_t rows_per_array;     // T * kv_heads   (paged: n_pages * kv_heads * 16)
     int32_t layer;
     int32_t q_heads, kv_heads, group, head_dim;

@@ -105,7 +105,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
             pc.w[1] = head;
             pc.w[2] = static_cast<int32_t>(tok0);
             pc.w[3] = static_cast<int32_t>(tok1 - tok0);
-            pc.w[4] = whole ? 1 : 0;
+            pc.w[4] = (whole ? 1 : 0) | (tok1 == in.len[r] ? 2 : 0);   // bit 0 direct, bit 1 ends its stream
             pc.w[5] = static_cast<int32_t>(pieces.size());       // slot
             // first row of the piece inside one K (or V) array of the pool
             pc.w[6] = static_cast<int32_t>(static_cast<int64_t>(in.base[r]) * hkv +
@@ -159,7 +159,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
                     if (static_cast<int32_t>(pieces.size()) - first_slot > 1)
                         record_split(r, head, first_slot);
                     else
-                        pieces[first_slot].w[4] = 1;       // moved to a fresh share and fitted whole
+                        pieces[first_slot].w[4] |= 1;      // moved to a fresh share and fitted whole
                 }
             }
         }
@@ -213,7 +213,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
                 if (static_cast<int32_t>(pieces.size()) - first_slot > 1)
                     record_split(r, head, first_slot);
                 else
-                    pieces[first_slot].w[4] = 1;       // no share had room for a piece: whole after all
+                    pieces[first_slot].w[4] |= 1;      // no share had room for a piece: whole after all
             }
         }
         return n_cut;
@@ -253,7 +253,7 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
     std::vector<int32_t> fill(at.begin(), at.end() - 1);
     for (int pass = 0; pass < 2; ++pass)
         for (const Piece& pc : pieces)
-            if ((pc.w[4] == 0) == (pass == 0)) {
+            if (((pc.w[4] & 1) == 0) == (pass == 0)) {
                 std::copy(pc.w, pc.w + 8, items + 8 * fill[pc.share]);
                 ++fill[pc.share];
             }

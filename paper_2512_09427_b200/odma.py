@@ -31,7 +31,7 @@ class Config(C.Structure):
                 ("p_num", C.c_int32 * MAX_BUCKETS), ("p_den", C.c_int32),
                 ("gamma_permille", C.c_int32), ("tau_permille", C.c_int32), ("growth", C.c_int32),
                 ("large_fixed", C.c_int32), ("max_batch", C.c_int32), ("max_group", C.c_int32),
-                ("plan_ctas", C.c_int32), ("fused_combine", C.c_int32)]
+                ("plan_ctas", C.c_int32), ("fused_combine", C.c_int32), ("fused_append", C.c_int32)]
 
 
 class Slab(C.Structure):

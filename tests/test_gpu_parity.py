@@ -239,6 +239,55 @@ def test_decode_step_from_host_buffers_matches_the_device_path():
     assert_close(out, ref, w.dtype, "host step")
 
 
+@pytest.mark.parametrize("fused_append", [1, 0])
+def test_decode_step_with_the_append_inside_the_decode_kernel(fused_append):
+    """odma_decode_step: the new token is taken from k_new / v_new by the decode kernel itself
+    (never read from the slab) and written into the slab for later steps.  Lengths chosen so
+    that some streams consist of the new token alone, some end a tile exactly, some are split."""
+    odma = lib()
+    lens = [0, 1, 63, 64, 127, 128, 500, 2771]
+    w = qwen_small(lens, layers=2)
+    s = Session(w, fill=0x7FC0, plan_ctas=19, fused_append=fused_append)     # untouched rows are NaN
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    pre = [r for r in reqs if w.context[r] > 0]
+    s.append(pre, [int(w.context[r]) for r in pre])
+    for step in range(2):
+        for r in reqs:
+            s.ls.ensure(r, s.lens[r] + 1)
+        q = torch.stack([s.queries(l, reqs, w.q_heads, step) for l in range(w.layers)]).contiguous()
+        kn = torch.stack([torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]) for l in range(w.layers)]).contiguous()
+        vn = torch.stack([torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]) for l in range(w.layers)]).contiguous()
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((w.layers, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev)
+        t = odma.Tables()
+        s.pool.profile_enable(True)
+        s.pool.decode_step(0, w.layers, w.q_heads, reqs, q.data_ptr(), kn.data_ptr(), vn.data_ptr(), out.data_ptr(),
+                           lse.data_ptr(), s.stream, t)
+        torch.cuda.synchronize()
+        assert s.pool.check_status(s.stream) == odma.OK
+        assert s.pool.profile_read(odma.K_APPEND)[1] == (0 if fused_append else w.layers)
+        assert s.pool.profile_read(odma.K_DECODE)[1] == w.layers
+        s.pool.profile_enable(False)
+        assert t.n_combine > 0
+        s.ls.commit(reqs, 1)
+        for l in range(w.layers):
+            for i, r in enumerate(reqs):
+                s.kv.append(r, l, kn[l, i:i + 1], vn[l, i:i + 1])
+        for r in reqs:
+            s.lens[r] += 1
+        for l in range(w.layers):
+            ref, ref_lse, _ = s.oracle_out(l, reqs, q[l], w.q_heads)
+            assert torch.isfinite(out[l].float()).all() and torch.isfinite(lse[l]).all()
+            assert_close(out[l], ref, w.dtype, f"fused step {step} layer {l}")
+            assert np.abs(lse[l].double().cpu().numpy() - ref_lse).max() <= 2e-2
+            for r in reqs:                      # the slab now holds the new rows, bit for bit
+                k_ref, v_ref = s.kv.gathered(r, l)
+                assert np.array_equal(s.pool_rows(l, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+                assert np.array_equal(s.pool_rows(l, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
 @pytest.mark.parametrize("fused", [1, 0])
 def test_profile_counts_launches(fused):
     odma = lib()

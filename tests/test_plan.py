@@ -51,7 +51,7 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
     assert t.n_ctas <= ctas
     # within a CTA's share the pieces of split streams come first
     for c in range(t.n_ctas):
-        d = items[cta_begin[c]:cta_begin[c + 1], 4]
+        d = items[cta_begin[c]:cta_begin[c + 1], 4] & 1
         assert list(d) == sorted(d)
     # slots number the pieces in (request, head, token) order; per stream they tile [0, len)
     # in order with no gap or overlap
@@ -59,7 +59,9 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
     assert list(by_slot[:, 5]) == list(range(t.n_items))
     cover = {}
     slabs = {r: pool.get_slab(r)[1] for r in range(n)}
-    for req, head, tok0, ntok, direct, slot, row, ci in by_slot:
+    for req, head, tok0, ntok, flags, slot, row, ci in by_slot:
+        direct = flags & 1
+        assert ((flags >> 1) & 1) == (tok0 + ntok == lens[req])      # bit 1: the piece ends its stream
         assert ntok >= 1 and tok0 % 64 == 0
         base, cap = slabs[req][0], slabs[req][1]
         assert row == base * hkv + head * cap + tok0        # the documented row(head, t) formula
@@ -97,7 +99,7 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
                       for c in range(t.n_ctas)])
     starts = np.array([sum(1 for k in range(cta_begin[c], cta_begin[c + 1]) if items[k, 2] == 0)
                        for c in range(t.n_ctas)])
-    parts = np.array([sum(1 for k in range(cta_begin[c], cta_begin[c + 1]) if items[k, 4] == 0)
+    parts = np.array([sum(1 for k in range(cta_begin[c], cta_begin[c + 1]) if items[k, 4] & 1 == 0)
                       for c in range(t.n_ctas)])
     total = sum(-(-L // 64) for L in lens) * hkv
     assert tiles.sum() == total and starts.sum() == n * hkv
@@ -105,8 +107,8 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
     if t.n_ctas > 1 and max(lens) > 128:
         assert cost.max() <= 1.25 * cost.sum() / ctas + 6, (cost.max(), cost.sum() / ctas)   # 6: a stream too short to split
     # pieces of split streams are never crumbs
-    for req, head, tok0, ntok, direct, *_ in by_slot:
-        if not direct and lens[req] > 6 * 64:
+    for req, head, tok0, ntok, flags, *_ in by_slot:
+        if not (flags & 1) and lens[req] > 6 * 64:
             assert ntok >= 2 * 64 or tok0 + ntok == lens[req]
     assert t.words * 4 <= pool.tables_bytes(n)
 
