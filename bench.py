@@ -93,6 +93,7 @@ class SlabDecode:
         cfg.max_batch = max(1024, w.batch)
         cfg.plan_ctas = plan_ctas
         cfg.fused_combine = fused
+        self.pool_cfg = cfg
         self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
         self.stream = torch.cuda.current_stream().cuda_stream
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
@@ -101,6 +102,7 @@ class SlabDecode:
         self.reqs_c = (C.c_uint64 * w.batch)(*self.reqs)
         self.zeros_c = (C.c_int32 * w.batch)()
         self.migrations_at_fill = 0
+        self._ptrs = {}
 
     def learn_boundaries(self):
         """Static ladder, or boundaries learned from the warm-up window of realised lengths."""
@@ -163,8 +165,12 @@ class SlabDecode:
         """Step i from device buffers: the layers it touches, one C call, then the length commit."""
         L = self.step_layers
         l0 = (i * L) % self.w.layers
-        self.pool.decode_step(l0, L, self.w.q_heads, self.reqs_c, q[l0].data_ptr(), kn[l0].data_ptr(),
-                              vn[l0].data_ptr(), out[l0].data_ptr(), 0, self.stream, tables)
+        key = (q.data_ptr(), l0)
+        ptrs = self._ptrs.get(key)
+        if ptrs is None:                         # tensor indexing costs microseconds: do it once
+            ptrs = self._ptrs[key] = (q[l0].data_ptr(), kn[l0].data_ptr(), vn[l0].data_ptr(), out[l0].data_ptr())
+        self.pool.decode_step(l0, L, self.w.q_heads, self.reqs_c, ptrs[0], ptrs[1], ptrs[2], ptrs[3], 0,
+                              self.stream, tables)
         self.commit_none()
 
     def commit_none(self):
@@ -403,7 +409,9 @@ def run_ours(args):
         clocks.mark(t_wall0, time.time())
     ms = ev0.elapsed_time(ev1)
     assert sd.pool.check_status(sd.stream) == odma.OK
-    launches_per_step = step_layers * (2 + (1 if tables.n_combine > 0 else 0))
+    fused_append = bool(sd.pool_cfg.fused_append) and w.dtype == torch.bfloat16
+    launches_per_step = step_layers * (1 + (0 if fused_append else 1) +
+                                       (1 if tables.n_combine > 0 and not args.fused_combine else 0))
     kv_bytes_per_launch = tables.kv_tokens * 2 * w.kv_heads * row_bytes
     step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes)
 
@@ -441,7 +449,10 @@ def run_ours(args):
         pages = torch.empty(n_pages * page_bytes, dtype=torch.uint8, device=dev)
         ptab = torch.zeros(n * max_pages, dtype=torch.int32, device=dev)
         paged = odma.Paged(sd.pool, pages.data_ptr(), pages.numel())
-        paged.build(tables, host_len, 950900, ptab.data_ptr(), max_pages, sd.stream)
+        own = torch.empty(sd.pool.tables_bytes(n), dtype=torch.uint8, device=dev)
+        # tables of the ablation's own: context+1 tokens, the last one written by the steps above
+        tables_a = sd.pool.build_tables(sd.reqs, own.data_ptr(), own.numel(), sd.stream)
+        paged.build(tables_a, host_len, 950900, ptab.data_ptr(), max_pages, sd.stream)
         reps = max(3, min(K, 200)) if step_layers == 1 else 3
         res = {}
         for kind in ("slab", "paged"):
@@ -451,9 +462,9 @@ def run_ours(args):
                 for i in range(reps * step_layers):
                     l = i % w.layers
                     if kind == "slab":
-                        sd.pool.decode_attention(l, q[l].data_ptr(), w.q_heads, tables, out[l].data_ptr(), 0, sd.stream)
+                        sd.pool.decode_attention(l, q[l].data_ptr(), w.q_heads, tables_a, out[l].data_ptr(), 0, sd.stream)
                     else:
-                        paged.decode_attention(l, q[l].data_ptr(), w.q_heads, tables, ptab.data_ptr(), max_pages,
+                        paged.decode_attention(l, q[l].data_ptr(), w.q_heads, tables_a, ptab.data_ptr(), max_pages,
                                                out[l].data_ptr(), 0, sd.stream)
                 torch.cuda.synchronize()
             t_ms, cnt = sd.pool.profile_read(odma.K_DECODE)

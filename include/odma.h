@@ -235,7 +235,13 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
  * d_q, d_out [n_layers, n, q_heads, head_dim]; d_k_new, d_v_new [n_layers, n, kv_heads,
  * head_dim]; lse device fp32 [n_layers, n, q_heads] or NULL.  tables_out (host, nullable)
  * receives the description of the built batch; its d_table stays valid until the next
- * odma_decode_step / odma_decode_step_host on this pool.  Does not commit lengths. */
+ * odma_decode_step / odma_decode_step_host on this pool.  Does not commit lengths.
+ * On a bf16 pool with fused_append the decode kernel appends the token itself (one launch per
+ * layer, no append kernel).  Consecutive steps of the same batch (same requests, no slab
+ * moved, grown by at most 32 tokens per request since the last full plan) reuse that plan: a
+ * stream's last piece takes the growth, and for batches of up to 256 requests the lengths
+ * travel with the kernel's arguments, so such a step copies no table; the length words of
+ * d_table in device memory are then those of the last full plan. */
 int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32_t q_heads,
                          const uint64_t* reqs, int32_t n, const void* d_q, const void* d_k_new,
                          const void* d_v_new, void* d_out, float* lse, void* stream,

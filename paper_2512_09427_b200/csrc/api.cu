@@ -18,6 +18,7 @@ using namespace odma;
 namespace {
 
 constexpr int kStagingSlots = 4;
+constexpr int kPlanReuseTokens = 32;   // a plan is reused until the batch grew this much per request
 constexpr int64_t kDefaultWaitLimitNs = 2000000000ll;   // 2 s: far above any kernel here
 
 struct ProfRecord {
@@ -61,6 +62,22 @@ struct odma_pool {
     std::vector<ProfRecord> prof;
     // reusable host vectors
     std::vector<int32_t> v_base, v_cap, v_len;
+    // The last full plan of a decode step (one new token per request).  While the same
+    // requests sit in the same slabs and have only grown a little, the next step reuses its
+    // dealing of streams to CTAs and only rewrites the lengths: a stream's last piece takes the
+    // growth.  A full plan is made again once the batch has grown by kPlanReuseTokens tokens per
+    // request on average, and whenever the batch or a slab changes.
+    struct PlanCache {
+        bool valid = false;
+        std::vector<uint64_t> reqs;
+        std::vector<int32_t> base, cap, len0, table;
+        std::vector<int32_t> end_word;   // table words holding n_tokens of pieces that end a stream ...
+        std::vector<int32_t> end_req;    // ... their request (index in the batch) ...
+        std::vector<int32_t> end_tok0;   // ... and first token
+        odma_tables desc{};
+        uint64_t gen = 0;                // counts full plans
+    } plan_cache;
+    uint64_t step_table_gen = 0;         // the full plan whose table sits in d_step_table (0: none)
 };
 
 struct odma_paged {
@@ -168,6 +185,23 @@ int32_t gather_batch(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new
     return ODMA_OK;
 }
 
+// After gather_batch: may the cached plan of an earlier decode step serve this batch?  Same
+// requests in the same slabs, grown only, and by no more than kPlanReuseTokens per request.
+bool plan_reusable(const odma_pool* pool, const uint64_t* reqs, int32_t n, int64_t* kv_tokens) {
+    const odma_pool::PlanCache& pc = pool->plan_cache;
+    if (!pc.valid || static_cast<int32_t>(pc.reqs.size()) != n || !std::equal(reqs, reqs + n, pc.reqs.begin()) ||
+        pool->v_base != pc.base || pool->v_cap != pc.cap)
+        return false;
+    int64_t growth = 0, total = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        if (pool->v_len[i] < pc.len0[i]) return false;
+        growth += pool->v_len[i] - pc.len0[i];
+        total += pool->v_len[i];
+    }
+    *kv_tokens = total;
+    return growth <= static_cast<int64_t>(kPlanReuseTokens) * n;
+}
+
 int32_t plan_into(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
                   int32_t* host_table, uint64_t table_bytes, odma_tables* out) {
     if (!pool || !reqs || !host_table || !out || n < 1) return ODMA_ERR_INVALID;
@@ -182,9 +216,49 @@ int32_t plan_into(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, i
     in.cap = pool->v_cap.data();
     in.len = pool->v_len.data();
     in.n_new = n_new;
+    odma_pool::PlanCache& pc = pool->plan_cache;
+    if (!n_new && static_cast<uint64_t>(pc.desc.words) * 4 <= table_bytes) {
+        int64_t kv_tokens = 0;
+        if (plan_reusable(pool, reqs, n, &kv_tokens)) {
+            std::copy(pc.table.begin(), pc.table.begin() + pc.desc.words, host_table);
+            std::copy(pool->v_len.begin(), pool->v_len.end(), host_table + pc.desc.off_len);
+            for (size_t k = 0; k < pc.end_word.size(); ++k)
+                host_table[pc.end_word[k]] = pool->v_len[pc.end_req[k]] - pc.end_tok0[k];
+            *out = pc.desc;
+            out->kv_tokens = kv_tokens;
+            out->epoch = pool->alloc.epoch();
+            return ODMA_OK;
+        }
+    }
     rc = plan_batch(in, host_table, static_cast<int64_t>(table_bytes / 4), out);
     if (rc != ODMA_OK) return rc;
     out->epoch = pool->alloc.epoch();
+    pc.valid = false;
+    if (!n_new) {
+        pc.reqs.assign(reqs, reqs + n);
+        pc.base = pool->v_base;
+        pc.cap = pool->v_cap;
+        pc.len0 = pool->v_len;
+        pc.table.assign(host_table, host_table + out->words);
+        pc.desc = *out;
+        pc.end_word.clear();
+        pc.end_req.clear();
+        pc.end_tok0.clear();
+        auto note = [&](int32_t word0) {             // word0: first word of an item (or of its copy)
+            if (host_table[word0 + 4] & 2) {
+                pc.end_word.push_back(word0 + 3);
+                pc.end_req.push_back(host_table[word0]);
+                pc.end_tok0.push_back(host_table[word0 + 2]);
+            }
+        };
+        for (int32_t k = 0; k < out->n_items; ++k) note(out->off_items + 8 * k);
+        for (int32_t c = 0; c < out->n_ctas; ++c) {  // the first item's copy in each CTA record
+            const int32_t* rec = host_table + out->off_cta + 12 * c;
+            if (rec[0] < rec[1]) note(out->off_cta + 12 * c + 4);
+        }
+        pc.valid = true;
+        pc.gen += 1;
+    }
     return ODMA_OK;
 }
 
@@ -499,7 +573,7 @@ bool uses_tc(const odma_pool* pool, int32_t q_heads) {
 // token (one per request) instead of finding it in the slab.
 int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
                               const odma_tables* tables, void* out, float* lse, void* stream,
-                              const void* k_new, const void* v_new) {
+                              const void* k_new, const void* v_new, const InlineLens* lens = nullptr) {
     int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
     if (rc != ODMA_OK) return rc;
     DecodeParams p;
@@ -516,7 +590,7 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
             if (p.stages < 2) return ODMA_ERR_INVALID;
             fused = p.counters != nullptr;
-            e = launch_decode_tc(pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream));
+            e = launch_decode_tc(pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens);
         } else if (generic_supported(pool->head_dim)) {
             p.counters = nullptr;
             e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
@@ -556,6 +630,7 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
     int32_t rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
                                    static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
     if (rc != ODMA_OK) return rc;
+    pool->step_table_gen = pool->plan_cache.valid ? pool->plan_cache.gen : 0;
     const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
     const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
     cudaStream_t s = as_stream(stream);
@@ -582,15 +657,44 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
                          odma_tables* tables_out) {
     if (!pool || !pool->dev_base || !d_q || !d_k_new || !d_v_new || !d_out) return ODMA_ERR_INVALID;
     if (n_layers < 1 || layer < 0 || layer + n_layers > pool->layers) return ODMA_ERR_INVALID;
-    odma_tables t;
-    int32_t rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
-                                   static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
-    if (rc != ODMA_OK) return rc;
+    if (!reqs || n < 1 || n > pool->alloc.config().max_batch) return ODMA_ERR_INVALID;
     const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
     const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
     // on the tensor-core path the append rides in the decode kernel: one launch per layer
     const bool fuse = pool->alloc.config().fused_append && q_heads >= pool->kv_heads &&
                       q_heads % pool->kv_heads == 0 && uses_tc(pool, q_heads) && aligned16(d_k_new) && aligned16(d_v_new);
+    // With the append fused, nothing but that kernel reads the step's lengths, and it can take
+    // them with its arguments: when the plan of an earlier step still serves (same requests,
+    // same slabs, grown a little) and its table is the one in device memory, this step needs
+    // no table copy at all.
+    odma_tables t;
+    static thread_local InlineLens lens;
+    const bool inline_lens = fuse && n <= kInlineLens;
+    bool reused = false;
+    int32_t rc;
+    if (inline_lens) {
+        rc = gather_batch(pool, reqs, nullptr, n);
+        if (rc != ODMA_OK) return rc;
+        int64_t kv_tokens = 0;
+        if (pool->step_table_gen != 0 && pool->step_table_gen == pool->plan_cache.gen &&
+            plan_reusable(pool, reqs, n, &kv_tokens)) {
+            t = pool->plan_cache.desc;
+            t.d_table = pool->d_step_table;
+            t.kv_tokens = kv_tokens;
+            t.epoch = pool->alloc.epoch();
+            reused = true;
+        }
+    }
+    if (!reused) {
+        rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
+                               static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
+        if (rc != ODMA_OK) return rc;
+        pool->step_table_gen = pool->plan_cache.valid ? pool->plan_cache.gen : 0;
+    }
+    if (inline_lens) {
+        lens.n = n;
+        std::copy(pool->v_len.begin(), pool->v_len.begin() + n, lens.len);
+    }
     for (int32_t l = 0; l < n_layers; ++l) {
         const uint8_t* kn = static_cast<const uint8_t*>(d_k_new) + l * kb;
         const uint8_t* vn = static_cast<const uint8_t*>(d_v_new) + l * kb;
@@ -601,7 +705,7 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
         rc = decode_attention_impl(pool, layer + l, static_cast<const uint8_t*>(d_q) + l * qb, q_heads, &t,
                                    static_cast<uint8_t*>(d_out) + l * qb,
                                    lse ? lse + static_cast<size_t>(l) * n * q_heads : nullptr, stream,
-                                   fuse ? kn : nullptr, fuse ? vn : nullptr);
+                                   fuse ? kn : nullptr, fuse ? vn : nullptr, inline_lens ? &lens : nullptr);
         if (rc != ODMA_OK) return rc;
     }
     if (tables_out) *tables_out = t;

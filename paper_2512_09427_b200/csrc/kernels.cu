@@ -252,7 +252,8 @@ __device__ __forceinline__ void combine_stream(const float* part_o, const float*
 template <int D, int NT, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
-                 const __grid_constant__ CUtensorMap tm_small, const DecodeParams p) {
+                 const __grid_constant__ CUtensorMap tm_small, const DecodeParams p,
+                 const __grid_constant__ InlineLens lens) {
     using Cfg = TcConfig<D, NT>;
     constexpr int ROWS = Cfg::kRows;
     constexpr int HALVES = D / 64;                 // 128-byte column blocks per row
@@ -371,7 +372,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 // With the append fused in, the stream's last token is not in the slab yet: it
                 // is not streamed; the finishers take it from k_new / v_new and write it there.
                 const bool has_new = p.k_new != nullptr && (b.x & 2);
-                const int ntok = a.w - (has_new ? 1 : 0);
+                // a piece that ends its stream ends where the stream ends NOW (the plan may be
+                // an earlier step's, made when the stream was a little shorter)
+                const int ntok_now = (lens.n > 0 && (b.x & 2)) ? lens.len[req] - tok0 : a.w;
+                const int ntok = ntok_now - (has_new ? 1 : 0);
                 dsc[2] = ntok;
                 dsc[3] = b.x & 1;                        // direct
                 dsc[4] = b.y;                            // slot
@@ -1130,7 +1134,8 @@ constexpr int kSmemPerCtaMax = 232448;    // most one CTA may ask for
 constexpr int kSmemCtaReserve = 1024;     // what the system keeps per resident CTA
 
 template <int D, int NT, int MODE>
-cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_ctas, cudaStream_t stream) {
+cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_ctas, cudaStream_t stream,
+                           const InlineLens& lens) {
     using Cfg = TcConfig<D, NT>;
     static bool configured = false;
     auto kern = decode_tc_kernel<D, NT, MODE>;
@@ -1143,16 +1148,17 @@ cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p);
+    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p, lens);
     return cudaGetLastError();
 }
 
 template <int D, int NT>
-cudaError_t launch_tc_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s) {
+cudaError_t launch_tc_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s,
+                           const InlineLens& lens) {
     switch (mode) {
-        case kModeSlab: return launch_tc_inst<D, NT, kModeSlab>(maps, p, n_ctas, s);
-        case kModePaged: return launch_tc_inst<D, NT, kModePaged>(maps, p, n_ctas, s);
-        case kModeProbe: return launch_tc_inst<D, NT, kModeProbe>(maps, p, n_ctas, s);
+        case kModeSlab: return launch_tc_inst<D, NT, kModeSlab>(maps, p, n_ctas, s, lens);
+        case kModePaged: return launch_tc_inst<D, NT, kModePaged>(maps, p, n_ctas, s, lens);
+        case kModeProbe: return launch_tc_inst<D, NT, kModeProbe>(maps, p, n_ctas, s, lens);
     }
     return cudaErrorInvalidValue;
 }
@@ -1206,14 +1212,16 @@ void tc_shape(int32_t head_dim, int32_t group, int32_t* stages, int32_t* q_slots
 }
 
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, const InlineLens* lens_in) {
+    static const InlineLens no_lens{};                 // n = 0: lengths as planned
+    const InlineLens& lens = lens_in ? *lens_in : no_lens;
     const bool two = p.group > 8;
     if (p.head_dim == 128)
-        return two ? launch_tc_mode<128, 2>(maps, p, mode, n_ctas, stream)
-                   : launch_tc_mode<128, 1>(maps, p, mode, n_ctas, stream);
+        return two ? launch_tc_mode<128, 2>(maps, p, mode, n_ctas, stream, lens)
+                   : launch_tc_mode<128, 1>(maps, p, mode, n_ctas, stream, lens);
     if (p.head_dim == 64)
-        return two ? launch_tc_mode<64, 2>(maps, p, mode, n_ctas, stream)
-                   : launch_tc_mode<64, 1>(maps, p, mode, n_ctas, stream);
+        return two ? launch_tc_mode<64, 2>(maps, p, mode, n_ctas, stream, lens)
+                   : launch_tc_mode<64, 1>(maps, p, mode, n_ctas, stream, lens);
     return cudaErrorInvalidValue;
 }
 

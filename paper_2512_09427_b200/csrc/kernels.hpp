@@ -43,6 +43,14 @@ struct DecodeParams {
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
 };
 
+// Lengths handed to the tensor-core kernel with its arguments instead of through the table in
+// device memory (a step that reuses the previous step's plan then needs no copy at all).
+constexpr int kInlineLens = 256;
+struct InlineLens {
+    int32_t n;                  // 0: take the lengths the plan was made with (items' n_tokens)
+    int32_t len[kInlineLens];   // length after this step's append, per request of the batch
+};
+
 struct TensorMaps {
     CUtensorMap big;    // box 64 rows x 64 elements
     CUtensorMap small;  // box 16 rows x 64 elements
@@ -56,7 +64,7 @@ bool tc_supported(int32_t head_dim, int32_t group);
 // both 0 when nothing fits).
 void tc_shape(int32_t head_dim, int32_t group, int32_t* stages, int32_t* q_slots);
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                             cudaStream_t stream);
+                             cudaStream_t stream, const InlineLens* lens = nullptr);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
 bool generic_supported(int32_t head_dim);
 

@@ -288,6 +288,45 @@ def test_decode_step_with_the_append_inside_the_decode_kernel(fused_append):
                 assert np.array_equal(s.pool_rows(l, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
 
 
+def test_many_fused_steps_reuse_the_plan_and_then_replan():
+    """36 consecutive decode steps of one batch through odma_decode_step: the plan of step 0
+    serves until the batch has grown by 32 tokens per request (lengths ride in the kernel
+    arguments, streams cross tile boundaries on the way), then a fresh plan is made."""
+    odma = lib()
+    lens = [30, 62, 63, 100, 127, 500, 1000]
+    w = qwen_small(lens)
+    w = wl.scaled(w, predicted=w.context + 64)
+    s = Session(w, plan_ctas=11)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    s.append(reqs, [int(c) for c in w.context])
+    t = odma.Tables()
+    plans = []
+    for step in range(36):
+        q = s.queries(0, reqs, w.q_heads, step).contiguous()
+        kn = torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+        vn = torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+        out = torch.full_like(q, float("nan"))
+        s.pool.decode_step(0, 1, w.q_heads, reqs, q.data_ptr(), kn.data_ptr(), vn.data_ptr(), out.data_ptr(), 0,
+                           s.stream, t)
+        torch.cuda.synchronize()
+        assert s.pool.check_status(s.stream) == odma.OK
+        plans.append((t.n_items, t.kv_tokens))
+        s.ls.commit(reqs, 1)
+        for i, r in enumerate(reqs):
+            s.kv.append(r, 0, kn[i:i + 1], vn[i:i + 1])
+            s.lens[r] += 1
+        if step in (0, 1, 17, 31, 32, 33, 35):
+            ref, _, _ = s.oracle_out(0, reqs, q, w.q_heads)
+            assert_close(out, ref, w.dtype, f"step {step}")
+    assert [kv for _, kv in plans] == [sum(lens) + w.batch * (k + 1) for k in range(36)]
+    for r in reqs:                                  # every appended row reached the slab
+        k_ref, v_ref = s.kv.gathered(r, 0)
+        assert np.array_equal(s.pool_rows(0, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+        assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
 @pytest.mark.parametrize("fused", [1, 0])
 def test_profile_counts_launches(fused):
     odma = lib()

@@ -6,16 +6,16 @@ from helpers import host_pool, lib
 from paper_2512_09427_b200 import workloads as wl
 
 
-def _plan(lens, kv_heads=4, ctas=148, max_len=32768 + 4096):
+def _plan(lens, kv_heads=4, ctas=148, max_len=32768 + 4096, headroom=0):
     buckets = [64, 256, 1024, 4096, 16384, max_len]
-    tokens = sum(min(b for b in buckets if b >= L) for L in lens)
+    tokens = sum(min(b for b in buckets if b >= L + headroom) for L in lens)
     w = wl.scaled(wl.config5(batch=1), pool_bytes=int(tokens * 1.3 + 64) * 2 * kv_heads * 128 * 2,
                   layers=1, kv_heads=kv_heads, max_len=max_len)
     pool = host_pool(w, plan_ctas=ctas, max_batch=max(1024, len(lens)))
     assert pool.set_buckets(buckets) == 0
     reqs = list(range(len(lens)))
     for r, L in zip(reqs, lens):
-        rc, slab = pool.alloc(r, int(L))
+        rc, slab = pool.alloc(r, int(L) + headroom)
         assert rc == 0, rc
         if L > 1:
             assert pool.commit_step([r], [int(L) - 1]) == 0
@@ -122,3 +122,50 @@ def test_plan_rejects_bad_batches():
     assert pool.commit_step([0], [slab[1] - ln]) == 0
     assert pool.plan_host([0, 1])[0] == odma.ERR_OVERFLOW
     assert pool.plan_host([0, 1], [0, 1])[0] == odma.OK
+
+
+def test_a_decode_step_plan_is_reused_while_the_batch_only_grows_a_little():
+    """Consecutive decode steps of the same batch keep the dealing of streams to CTAs; only the
+    lengths (and with them the last piece of each stream) move.  After enough growth, or when a
+    slab changes, the plan is made afresh."""
+    lens = list(wl.config2().context + 1)
+    hkv = 4
+    pool, t0, w0 = _plan(lens, hkv, 148, headroom=64)   # _plan has committed len-1 tokens and planned +1
+    reqs = list(range(len(lens)))
+
+    def cover(t, w, cur):
+        items = w[t.off_items:t.off_items + 8 * t.n_items].reshape(-1, 8)
+        got = {}
+        for req, head, tok0, ntok, flags, *_ in items[np.argsort(items[:, 5])]:
+            assert got.get((req, head), 0) == tok0
+            got[(req, head)] = tok0 + ntok
+        assert got == {(r, h): cur[r] for r in reqs for h in range(hkv)}
+        assert list(w[t.off_len:t.off_len + len(cur)]) == cur and t.kv_tokens == sum(cur)
+        recs = w[t.off_cta:t.off_cta + 12 * t.n_ctas].reshape(-1, 12)
+        for c in range(t.n_ctas):
+            if recs[c, 0] < recs[c, 1]:
+                assert list(recs[c, 4:]) == list(items[recs[c, 0]])
+        return items
+
+    base = cover(t0, w0, lens)
+    cur = list(lens)
+    for step in range(1, 40):
+        assert pool.commit_step(reqs) == 0
+        cur = [L + 1 for L in cur]
+        rc, t, words = pool.plan_host(reqs)
+        assert rc == 0
+        items = cover(t, np.array(words, dtype=np.int64), cur)
+        same = items.shape == base.shape and np.array_equal(items[:, [0, 1, 2, 4, 5, 6, 7]], base[:, [0, 1, 2, 4, 5, 6, 7]])
+        if step <= 32:
+            assert same, step                      # same pieces on the same CTAs, longer ends
+        else:
+            base = items if not same else base     # a fresh plan may cut elsewhere
+    # a request that moved to another slab invalidates the cached plan at once
+    rc, slab, ln = pool.get_slab(0)
+    rc, slab2, mig = pool.ensure_capacity(0, slab[1] + 1)        # beyond its slab: moves to the Large Bucket
+    assert rc == 0 and mig == 1
+    rc, t, words = pool.plan_host(reqs)
+    assert rc == 0
+    items = cover(t, np.array(words, dtype=np.int64), cur)
+    row0 = items[(items[:, 0] == 0) & (items[:, 1] == 0) & (items[:, 2] == 0)][0, 6]
+    assert row0 == slab2[0] * hkv
