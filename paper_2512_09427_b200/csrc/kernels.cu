@@ -322,6 +322,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Programmatic dependent launch: everything above (barrier set-up, the CTA's record from the
+    // step's table, which no kernel writes) may run while the previous kernel of the stream is
+    // still draining; nothing below may.  The next kernel of the stream is let go at once: its
+    // CTAs only find room as these exit, and they wait at this same point for the whole grid.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
@@ -1148,8 +1154,17 @@ cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<n_ctas, kTcThreads, smem, stream>>>(maps.big, maps.small, p, lens);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas));
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, maps.big, maps.small, p, lens);
 }
 
 template <int D, int NT>
