@@ -11,7 +11,7 @@ namespace odma {
 constexpr int32_t kTileTokens = 64;   // tokens staged per pipeline stage
 constexpr int32_t kSnapTiles = 2;     // streams this short are never cut in two
 constexpr int32_t kStreamCostTiles = 1;  // a stream's start-up weighs as much as this many tiles
-constexpr int32_t kSplitCostTiles = 2;   // so does, on top, every piece of a split stream
+constexpr int32_t kSplitCostTiles = 6;   // so does, on top, every piece of a split stream
 constexpr int32_t kMinPieceTiles = 3;    // no piece of a split stream is shorter than this
 constexpr int32_t kSlackTiles = 2;       // a whole stream may overfill a share by this much rather than be cut
 constexpr int32_t kCtaWords = 12;     // per-CTA record: {item_begin, item_end, 0, 0, first item[8]}

@@ -93,7 +93,7 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
     assert [tuple(int(x) for x in c) for c in comb] == want
     for ci, (req, head, first, pieces) in enumerate(want):
         assert (by_slot[first:first + pieces, 7] == ci).all()
-    # balance: shares are equal in cost: a tile costs 1, a stream start 1, a piece of a split
+    # balance: shares are equal in cost: a tile costs 1, a stream start 1, a piece of a split (6 on top)
     # stream 2 on top; no share exceeds the average by more than a quarter (+ rounding)
     tiles = np.array([sum(-(-int(items[k, 3]) // 64) for k in range(cta_begin[c], cta_begin[c + 1]))
                       for c in range(t.n_ctas)])
@@ -103,7 +103,7 @@ def test_plan_covers_every_tile_exactly_once_and_is_balanced(lens, ctas):
                       for c in range(t.n_ctas)])
     total = sum(-(-L // 64) for L in lens) * hkv
     assert tiles.sum() == total and starts.sum() == n * hkv
-    cost = tiles + starts + 2 * parts
+    cost = tiles + starts + 6 * parts
     if t.n_ctas > 1 and max(lens) > 128:
         assert cost.max() <= 1.25 * cost.sum() / ctas + 6, (cost.max(), cost.sum() / ctas)   # 6: a stream too short to split
     # pieces of split streams are never crumbs
