@@ -619,38 +619,6 @@ int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int
     return decode_attention_impl(pool, layer, q, q_heads, tables, out, lse, stream, nullptr, nullptr);
 }
 
-int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
-                              int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
-                              void* h_out, void* stream) {
-    if (!pool || !pool->dev_base || !h_q || !h_k_new || !h_v_new || !h_out) return ODMA_ERR_INVALID;
-    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0 ||
-        q_heads / pool->kv_heads > pool->alloc.config().max_group)
-        return ODMA_ERR_INVALID;
-    odma_tables t;
-    int32_t rc = odma_build_tables(pool, reqs, nullptr, n, pool->d_step_table,
-                                   static_cast<uint64_t>(pool->table_words_max) * 4, stream, &t);
-    if (rc != ODMA_OK) return rc;
-    pool->step_table_gen = pool->plan_cache.valid ? pool->plan_cache.gen : 0;
-    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
-    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
-    cudaStream_t s = as_stream(stream);
-    if (cudaMemcpyAsync(pool->d_q, h_q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(pool->d_k_new, h_k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(pool->d_v_new, h_v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return ODMA_ERR_CUDA;
-    const bool fuse = pool->alloc.config().fused_append && uses_tc(pool, q_heads);
-    if (!fuse) {
-        rc = odma_append_kv(pool, layer, &t, pool->d_k_new, pool->d_v_new, stream);
-        if (rc != ODMA_OK) return rc;
-    }
-    rc = decode_attention_impl(pool, layer, pool->d_q, q_heads, &t, pool->d_out, nullptr, stream,
-                               fuse ? pool->d_k_new : nullptr, fuse ? pool->d_v_new : nullptr);
-    if (rc != ODMA_OK) return rc;
-    if (cudaMemcpyAsync(h_out, pool->d_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return ODMA_ERR_CUDA;
-    return ODMA_OK;
-}
-
 int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32_t q_heads,
                          const uint64_t* reqs, int32_t n, const void* d_q, const void* d_k_new,
                          const void* d_v_new, void* d_out, float* lse, void* stream,
@@ -711,6 +679,31 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
     if (tables_out) *tables_out = t;
     return ODMA_OK;
 }
+
+int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
+                              int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
+                              void* h_out, void* stream) {
+    if (!pool || !pool->dev_base || !h_q || !h_k_new || !h_v_new || !h_out) return ODMA_ERR_INVALID;
+    if (!reqs || n < 1 || n > pool->alloc.config().max_batch) return ODMA_ERR_INVALID;
+    if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0 ||
+        q_heads / pool->kv_heads > pool->alloc.config().max_group)
+        return ODMA_ERR_INVALID;
+    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
+    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(pool->d_q, h_q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(pool->d_k_new, h_k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(pool->d_v_new, h_v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    // the step itself is the device-buffer one (same plan reuse, same fused append)
+    int32_t rc = odma_decode_step(pool, layer, 1, q_heads, reqs, n, pool->d_q, pool->d_k_new, pool->d_v_new,
+                                  pool->d_out, nullptr, stream, nullptr);
+    if (rc != ODMA_OK) return rc;
+    if (cudaMemcpyAsync(h_out, pool->d_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    return ODMA_OK;
+}
+
 
 int32_t odma_decode_attention_static(const odma_pool* pool, const void* dev_base, int32_t layer,
                                      const void* q, int32_t q_heads, const odma_tables* tables,
