@@ -495,9 +495,29 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
                     const int idx = min(ftid + i * fthreads, total - 1);
-                    const int r = idx / PER_ROW, d0 = (idx - r * PER_ROW) * 4;
-                    rr[i] = r;
-                    dd[i] = d0;
+                    rr[i] = idx / PER_ROW;
+                    dd[i] = (idx - rr[i] * PER_ROW) * 4;
+                }
+                // the token appended this step (if this piece ends its stream): its query, key
+                // and value parts are fetched now so that the loads fly during the merge below
+                const int new_row = hdr[5];
+                const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(p.q) +
+                                            (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group) * D;
+                const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D;
+                const __nv_bfloat16* krow = reinterpret_cast<const __nv_bfloat16*>(p.k_new) + nrow;
+                const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(p.v_new) + nrow;
+                uint2 nq[CH], nk[CH], nv[CH];
+                if (new_row >= 0) {
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) {
+                        nq[i] = __ldg(reinterpret_cast<const uint2*>(qrow + rr[i] * D + dd[i]));
+                        nk[i] = __ldg(reinterpret_cast<const uint2*>(krow + dd[i]));
+                        nv[i] = __ldg(reinterpret_cast<const uint2*>(vrow + dd[i]));
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const int r = rr[i], d0 = dd[i];
                     float mw[kConsumerWarps], lw[kConsumerWarps], M = -INFINITY;
                     float4 x[kConsumerWarps];
 #pragma unroll
@@ -523,21 +543,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                     acc_m[i] = M;
                     acc_l[i] = L;
                 }
-                const int new_row = hdr[5];
                 if (new_row >= 0) {
-                    // the token appended this step: its score against each head from k_new
-                    // (lanes that share a head add their parts up), its value from v_new; then
-                    // its K and V rows go into the slab for the steps to come
-                    const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(p.q) +
-                                                (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group) * D;
-                    const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D;
-                    const __nv_bfloat16* krow = reinterpret_cast<const __nv_bfloat16*>(p.k_new) + nrow;
-                    const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(p.v_new) + nrow;
+                    // its score against each head (lanes that share a head add their parts up),
+                    // its value; then its K and V rows go into the slab for the steps to come
 #pragma unroll
                     for (int i = 0; i < CH; ++i) {
-                        const uint2 qv = __ldg(reinterpret_cast<const uint2*>(qrow + rr[i] * D + dd[i]));
-                        const uint2 kv2 = __ldg(reinterpret_cast<const uint2*>(krow + dd[i]));
-                        const uint2 vv = __ldg(reinterpret_cast<const uint2*>(vrow + dd[i]));
+                        const uint2 qv = nq[i], kv2 = nk[i], vv = nv[i];
                         float dot = __uint_as_float(qv.x << 16) * __uint_as_float(kv2.x << 16);
                         dot = fmaf(__uint_as_float(qv.x & 0xFFFF0000u), __uint_as_float(kv2.x & 0xFFFF0000u), dot);
                         dot = fmaf(__uint_as_float(qv.y << 16), __uint_as_float(kv2.y << 16), dot);
