@@ -326,8 +326,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
     // step's table, which no kernel writes) may run while the previous kernel of the stream is
     // still draining; nothing below may.  The next kernel of the stream is let go at once: its
     // CTAs only find room as these exit, and they wait at this same point for the whole grid.
+    // One exception, below: the producer starts the CTA's first tiles before it waits, those
+    // that hold no row a decode kernel just ahead in the stream could still be writing.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (warp != kProducerWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
@@ -344,6 +346,36 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
         const int64_t v_array = k_array + p.rows_per_array;
         uint32_t qs = 0, qphase = 0;
+        // Early start.  The only pool rows the previous kernel of the stream may still be
+        // writing (when it is this kernel, one step or one layer earlier) are the last two of a
+        // stream: the token it appended, and this step's position if the step is a repeat.
+        // Full tiles of the CTA's first item that end before those rows are requested now, so
+        // that HBM is already streaming when the previous grid finishes; everything else
+        // (queries, other items, ragged tiles) comes after the wait.
+        int early = 0;
+        if (lane == 0 && MODE != kModePaged && it_begin < it_end) {
+            const int tok0 = first_a.z;
+            const int ntok_now = (lens.n > 0 && (first_b.x & 2)) ? lens.len[first_a.x] - tok0 : first_a.w;
+            const int safe_tok = (first_b.x & 2) ? ntok_now - 2 : ntok_now;
+            early = min(static_cast<int>(STAGES), max(safe_tok, 0) / kTile);
+            for (int t = 0; t < early; ++t) {
+                const uint32_t kdst = kv_u32 + t * Cfg::kStageBytes;
+                const uint32_t vdst = kdst + Cfg::kKvTileBytes;
+                mbar_expect_tx(full_bar(t), Cfg::kStageBytes);
+                const int32_t ky = static_cast<int32_t>(k_array + first_b.z + t * kTile);
+                const int32_t vy = static_cast<int32_t>(v_array + first_b.z + t * kTile);
+#pragma unroll
+                for (int h = 0; h < HALVES; ++h) {
+                    tma_load_2d(kdst + h * HALF_BYTES, &tm_big, h * 64, ky, full_bar(t));
+                    tma_load_2d(vdst + h * HALF_BYTES, &tm_big, h * 64, vy, full_bar(t));
+                }
+                issued_any |= 1u << t;
+                issued_odd ^= 1u << t;
+            }
+            stage = static_cast<uint32_t>(early) % STAGES;
+            phase = static_cast<uint32_t>(early) == STAGES ? 1u : 0u;
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
         for (int it = it_begin;; ++it) {
             const int j = (it - it_begin) & 31;
@@ -403,7 +435,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 if (MODE == kModePaged)
                     pages = p.page_table + static_cast<size_t>(req) * p.max_pages + tok0 / 16;
                 const int ntiles = (ntok + kTile - 1) / kTile;
-                for (int t = 0; t < ntiles; ++t) {
+                for (int t = (it == it_begin ? early : 0); t < ntiles; ++t) {   // the early tiles are under way
                     ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit);
                     if (!ok) break;
                     const int valid = min(kTile, ntok - t * kTile);
