@@ -327,6 +327,43 @@ def test_many_fused_steps_reuse_the_plan_and_then_replan():
         assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
 
 
+def test_back_to_back_steps_on_one_layer_without_host_syncs():
+    """Steps enqueued back to back on the same layer: each kernel starts (and requests its first
+    tiles) while its predecessor, which is still appending a row to every stream, drains.  All
+    outputs and every appended row must come out as if the steps had run one at a time."""
+    odma = lib()
+    lens = [70, 129, 200, 640, 1500, 3000]
+    w = qwen_small(lens)
+    w = wl.scaled(w, predicted=w.context + 48)
+    s = Session(w, plan_ctas=13)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    s.append(reqs, [int(c) for c in w.context])
+    steps = 24
+    qs = [s.queries(0, reqs, w.q_heads, k).contiguous() for k in range(steps)]
+    kns = [torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]).contiguous() for k in range(steps)]
+    vns = [torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]).contiguous() for k in range(steps)]
+    outs = [torch.full_like(qs[0], float("nan")) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for k in range(steps):                       # no synchronisation inside this loop
+        s.pool.decode_step(0, 1, w.q_heads, reqs, qs[k].data_ptr(), kns[k].data_ptr(), vns[k].data_ptr(),
+                           outs[k].data_ptr(), 0, s.stream)
+        s.ls.commit(reqs, 1)
+    torch.cuda.synchronize()
+    assert s.pool.check_status(s.stream) == odma.OK
+    for k in range(steps):
+        for i, r in enumerate(reqs):
+            s.kv.append(r, 0, kns[k][i:i + 1], vns[k][i:i + 1])
+        ref, _, _ = s.oracle_out(0, reqs, qs[k], w.q_heads)
+        assert_close(outs[k], ref, w.dtype, f"step {k}")
+    for r in reqs:
+        s.lens[r] += steps
+        k_ref, v_ref = s.kv.gathered(r, 0)
+        assert np.array_equal(s.pool_rows(0, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+        assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
 @pytest.mark.parametrize("fused", [1, 0])
 def test_profile_counts_launches(fused):
     odma = lib()
