@@ -174,3 +174,40 @@ def test_config4_drift_stream_attention_at_boundary_epochs():
     assert st["completed"] == 1600 and st["migrations"] > 0
     print("config4:", seen, "migrations", st["migrations"],
           "utilisation %.3f" % (st["sum_len_completed"] / st["sum_cap_completed"]))
+
+
+def test_config2_in_the_benchmarks_own_launch_configuration():
+    """bench.py's set-up and step for config 2 (rotating KV copies, odma_decode_step with the
+    append and the merge inside the decode kernel, plan reused from step to step): outputs of
+    sampled requests on two of the copies against the checker, and the appended rows in place."""
+    import bench
+    odma = lib()
+    w, step_layers, copies = bench.pick_workload("config2")
+    sd = bench.SlabDecode(w, step_layers, torch.device("cuda:0"))
+    bounds, epoch = sd.learn_boundaries()
+    assert len(bounds) == 4 and epoch == 10
+    sd.admit_and_fill()
+    q, kn, vn, out = sd.make_inputs()
+    t = odma.Tables()
+    for i in range(2 * copies):                    # every copy twice: second round reuses the plan
+        sd.step(i, q, kn, vn, out, t)
+    torch.cuda.synchronize()
+    assert sd.pool.check_status(sd.stream) == odma.OK
+    assert t.n_ctas == 148 and t.kv_tokens == int((w.context + 1).sum())
+    order = np.argsort(w.context)
+    sample = sorted({int(order[0]), int(order[len(order) // 2]), int(order[-1]), 0, w.batch - 1})
+    idx = torch.tensor(sample, device=sd.dev)
+    for layer in (0, copies - 1):
+        ref, _ = checker_out(w, layer, sample, [int(w.context[r]) + 1 for r in sample], q[layer][idx])
+        err = assert_close(out[layer][idx], ref, w.dtype, f"bench configuration, copy {layer}")
+        print("config2 as benchmarked, copy", layer, "max_abs %.2e rel_l2 %.2e" % err)
+        # the step's token sits behind each sampled request's context in the slab
+        T = sd.pool.get_stats()["total_tokens"]
+        arr = sd.mem.view(w.dtype)[: w.layers * 2 * T * w.kv_heads * w.head_dim].view(w.layers * 2, T * w.kv_heads, w.head_dim)
+        for r in sample:
+            rc, slab, ln = sd.pool.get_slab(r)
+            base, cap = slab[0], slab[1]
+            for kv, new in ((0, kn), (1, vn)):
+                for h in range(w.kv_heads):
+                    row = base * w.kv_heads + h * cap + int(w.context[r])
+                    assert torch.equal(arr[layer * 2 + kv][row], new[layer][r, h])
