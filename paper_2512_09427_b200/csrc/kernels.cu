@@ -2,14 +2,16 @@
 //
 //  append_kv_kernel        writes the step's new K/V rows behind each request's tokens
 //  migrate_copy_kernel     slab -> slab copy of one request (allocate-and-copy migration)
-//  decode_tc_kernel        split decode attention, bf16: TMA-staged slab streams, GQA heads
-//                          packed into the M dimension of mma.sync tiles, fp32 online softmax
+//  decode_tc_kernel        split decode attention, bf16: TMA-staged slab streams, keys on the M
+//                          side and the GQA group's heads on the N side of mma.sync tiles, fp32
+//                          online softmax; can take the step's append and the merge of split
+//                          streams along
 //  decode_generic_kernel   same result for any dtype / group size on the plain ALUs (fp32 path)
 //  combine_kernel          log-sum-exp merge of the partial results of split streams
 //  scatter_pages_kernel    re-lays slabs into 16-token pages (ablation input)
 //
-// The decode kernels are persistent: CTA c works through items [cta_begin[c], cta_begin[c+1])
-// of the host-built plan; an item is a run of tokens of one (request, KV head) stream.
+// The decode kernels are persistent: CTA c works through the items of its record in the
+// host-built plan; an item is a run of tokens of one (request, KV head) stream.
 #include "kernels.hpp"
 
 #include <cuda_bf16.h>
