@@ -74,6 +74,74 @@ def pick_workload(name: str, rank: int = 0, copies_override: int = 0):
     return w, step_layers, copies
 
 
+class _HostLoop:
+    """The library's allocator (a bookkeeping-only pool: no device memory) behind the face
+    workloads.run_closed_loop drives."""
+
+    def __init__(self, pool, odma):
+        self.pool, self.odma = pool, odma
+
+    def alloc(self, req, predicted):
+        rc, slab = self.pool.alloc(req, predicted)
+        return slab[:4] if rc == self.odma.OK else None
+
+    def ensure(self, req, need):
+        rc, slab, mig = self.pool.ensure_capacity(req, need)
+        if rc == self.odma.ERR_NOMEM:
+            return None
+        assert rc == self.odma.OK, rc
+        return slab[:4], mig
+
+    def commit(self, reqs, n_new):
+        reqs = list(reqs)
+        assert self.pool.commit_step(reqs, [n_new] * len(reqs)) == 0
+
+    def free(self, req):
+        assert self.pool.free(req) == 0
+
+    def buckets(self):
+        return self.pool.get_buckets()
+
+
+def config4_drift(rank: int = 0):
+    """Config 4 on the host: the whole 10,000-request drift stream through the library's
+    allocator (closed loop of 128 live requests).  Returns the allocator's statistics and two
+    snapshots of the live batch, one from each half of the stream, as workloads for the GPU."""
+    from paper_2512_09427_b200 import odma
+    w = wl.config4(seed=950904 + 1000 * rank)
+    cfg = odma.config_default()
+    cfg.safety_pct, cfg.max_len, cfg.granule, cfg.window, cfg.refresh = w.safety_pct, w.max_len, w.granule, w.window, w.refresh
+    pool = odma.Pool(0, w.pool_bytes, w.layers, w.kv_heads, w.head_dim, odma.DTYPE_BF16, cfg)
+    assert pool.set_buckets(list(w.static_buckets)) == 0
+    snaps = {}
+
+    def on_epoch(epoch, live, lens):
+        snaps[epoch] = ([int(r) for r in live], np.asarray(lens, dtype=np.int64).copy(), pool.get_buckets()[0])
+
+    res = wl.run_closed_loop(_HostLoop(pool, odma), w.context, w.predicted, w.extra["concurrency"], on_epoch=on_epoch)
+    st = pool.get_stats()
+    n_req = int(w.context.shape[0])
+    stats = {"requests": n_req, "completed": st["completed"], "utilisation": st["sum_len_completed"] / max(st["sum_cap_completed"], 1),
+             "static_utilisation": float(w.context.sum()) / (n_req * w.max_len), "migrations": st["migrations"],
+             "migration_rate": st["migrations"] / n_req, "deferred_admissions": res.deferred, "preempted": res.preempted,
+             "large_bucket_peak_tokens": st["safety_peak"], "recalibrations": len(res.boundary_log),
+             "boundaries_first_half": list(res.boundary_log[len(res.boundary_log) // 4][1]),
+             "boundaries_second_half": list(res.boundary_log[-2][1])}
+    epochs = sorted(snaps)
+    halves = []
+    for name, e in (("first half (lognormal, median 256)", epochs[len(epochs) // 4]),
+                    ("second half (70% median 128 / 30% median 4096)", epochs[-2])):
+        live, lens, bounds = snaps[e]
+        total = w.context[np.asarray(live)]
+        ctx = np.maximum(lens - 1, 1)
+        tokens = int(sum(min(b for b in bounds if b >= t) if t <= bounds[-1] else -(-int(t) // 16) * 16 for t in total) / 0.85) + 4096
+        halves.append((name, e, wl.Workload(
+            name="config4", seed=w.seed + e, layers=1, q_heads=w.q_heads, kv_heads=w.kv_heads, head_dim=w.head_dim,
+            dtype=w.dtype, pool_bytes=tokens * 2 * w.kv_heads * w.head_dim * 2, safety_pct=15, max_len=w.max_len,
+            context=ctx, predicted=np.maximum(total, ctx + 1), static_buckets=tuple(sorted(set(int(b) for b in bounds))))))
+    return stats, halves
+
+
 class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
@@ -185,8 +253,11 @@ class SlabDecode:
         L = self.step_layers
         l0 = (i * L) % self.w.layers
         for l in range(l0, l0 + L):
-            self.pool.decode_step_host(l, self.w.q_heads, self.reqs_c, hq[l].data_ptr(), hkn[l].data_ptr(),
-                                       hvn[l].data_ptr(), hout[l].data_ptr(), self.stream)
+            key = (hq.data_ptr(), l)
+            ptrs = self._ptrs.get(key)
+            if ptrs is None:                     # tensor indexing costs microseconds: do it once
+                ptrs = self._ptrs[key] = (hq[l].data_ptr(), hkn[l].data_ptr(), hvn[l].data_ptr(), hout[l].data_ptr())
+            self.pool.decode_step_host(l, self.w.q_heads, self.reqs_c, ptrs[0], ptrs[1], ptrs[2], ptrs[3], self.stream)
         torch.cuda.current_stream().synchronize()
         self.commit_none()
 
@@ -559,6 +630,55 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_config4(args):
+    """`--workload config4`: the drift stream through the allocator on the host (utilisation,
+    migrations, boundaries), then the decode step of the live batch of each half on the GPU."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    stats, halves = config4_drift()
+    peak, peak_kind = measured_peak()
+    K, W = args.steps, args.warmup
+    out_halves = []
+    for name, epoch, w in halves:
+        kv_bytes = int((w.context + 1).sum()) * 2 * w.kv_heads * w.head_dim * w.elem_bytes
+        copies = max(2, -(-3 * L2_BYTES // kv_bytes))               # rotate over copies: cold L2
+        wc = wl.scaled(w, layers=copies, pool_bytes=w.pool_bytes * copies)
+        sd = SlabDecode(wc, 1, dev, fused=args.fused_combine)
+        sd.learn_boundaries()
+        sd.admit_and_fill()
+        q, kn, vn, out = sd.make_inputs()
+        tables = sd.odma.Tables()
+        for i in range(W):
+            sd.step(i, q, kn, vn, out, tables)
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for i in range(K):
+            sd.step(W + i, q, kn, vn, out, tables)
+        ev1.record()
+        torch.cuda.synchronize()
+        assert sd.pool.check_status(sd.stream) == sd.odma.OK
+        ms = ev0.elapsed_time(ev1) / K
+        st = sd.pool.get_stats()
+        out_halves.append({"half": name, "epoch": epoch, "batch": wc.batch, "kv_tokens": int(tables.kv_tokens),
+                           "ms_per_step": ms, "tokens_per_s": wc.batch / (ms * 1e-3),
+                           "decode_gbs": kv_bytes / (ms * 1e-3) / 1e9, "frac_of_peak": kv_bytes / (ms * 1e-3) / 1e9 / peak,
+                           "batch_utilisation": st["used_live"] / max(st["reserved_live"], 1),
+                           "plan": {"ctas": tables.n_ctas, "items": tables.n_items, "combine": tables.n_combine},
+                           "kv_copies": copies})
+        del sd, q, kn, vn, out
+        torch.cuda.empty_cache()
+    line = {"metric": METRIC, "value": out_halves[0]["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+            "ms_per_step": out_halves[0]["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "configs[3]: drift stream, 10,000 requests, rebucketing every 500, 28q/4kv/128 bf16 single "
+                                   "layer, steady-state batch 128; `value` is the first half's batch, both halves below"},
+            "allocator": stats, "halves": out_halves, "peak": peak, "peak_kind": peak_kind}
+    print(json.dumps(line), flush=True)
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
     if dist is None:
@@ -574,7 +694,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config5"])
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--phases", default="timed,kernels,e2e,clocks,cpu",
                     help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
@@ -587,6 +707,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "config4":
+        run_config4(args)
     else:
         run_ours(args)
 
