@@ -99,8 +99,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
-// Two views of a [rows x head_dim] bf16 row array: 64-row and 16-row boxes of 64 elements
-// (128 bytes, the widest inner extent the 128-byte swizzle allows).
+// Four views of a [rows x head_dim] bf16 row array: boxes of 16, 32, 48 and 64 rows by 64
+// elements (128 bytes, the widest inner extent the 128-byte swizzle allows).
 int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, TensorMaps* out) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
@@ -111,15 +111,13 @@ int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, TensorMaps*
     const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(rows)};
     const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(head_dim) * 2};
     const cuuint32_t estride[2] = {1, 1};
-    const cuuint32_t box_big[2] = {64, 64}, box_small[2] = {64, 16};
-    if (encode(&out->big, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box_big, estride,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return ODMA_ERR_CUDA;
-    if (encode(&out->small, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box_small, estride,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return ODMA_ERR_CUDA;
+    for (int k = 0; k < 4; ++k) {
+        const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(16 * (k + 1))};
+        if (encode(&out->box[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estride,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return ODMA_ERR_CUDA;
+    }
     return ODMA_OK;
 }
 

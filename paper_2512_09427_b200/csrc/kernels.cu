@@ -253,8 +253,7 @@ __device__ __forceinline__ void combine_stream(const float* part_o, const float*
 
 template <int D, int NT, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
-decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
-                 const __grid_constant__ CUtensorMap tm_small, const DecodeParams p,
+decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                  const __grid_constant__ InlineLens lens) {
     using Cfg = TcConfig<D, NT>;
     constexpr int ROWS = Cfg::kRows;
@@ -299,8 +298,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
         rec = __ldg(r);
         first_a = __ldg(r + 1);
         first_b = __ldg(r + 2);
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_big)) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_small)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[3])) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[0])) : "memory");
     } else if (warp >= kFinisherWarp0 && lane == 0) {
         rec = __ldg(p.cta + 3 * cta);
     }
@@ -368,8 +367,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                 const int32_t vy = static_cast<int32_t>(v_array + first_b.z + t * kTile);
 #pragma unroll
                 for (int h = 0; h < HALVES; ++h) {
-                    tma_load_2d(kdst + h * HALF_BYTES, &tm_big, h * 64, ky, full_bar(t));
-                    tma_load_2d(vdst + h * HALF_BYTES, &tm_big, h * 64, vy, full_bar(t));
+                    tma_load_2d(kdst + h * HALF_BYTES, &tm.box[3], h * 64, ky, full_bar(t));
+                    tma_load_2d(vdst + h * HALF_BYTES, &tm.box[3], h * 64, vy, full_bar(t));
                 }
                 issued_any |= 1u << t;
                 issued_odd ^= 1u << t;
@@ -449,29 +448,34 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tm_big,
                         const int32_t vy = static_cast<int32_t>(v_array + row + t * kTile);
 #pragma unroll
                         for (int h = 0; h < HALVES; ++h) {
-                            tma_load_2d(kdst + h * HALF_BYTES, &tm_big, h * 64, ky, full_bar(stage));
-                            tma_load_2d(vdst + h * HALF_BYTES, &tm_big, h * 64, vy, full_bar(stage));
+                            tma_load_2d(kdst + h * HALF_BYTES, &tm.box[3], h * 64, ky, full_bar(stage));
+                            tma_load_2d(vdst + h * HALF_BYTES, &tm.box[3], h * 64, vy, full_bar(stage));
                         }
                     } else {
-                        const int nb = (valid + 15) >> 4;     // 16-row boxes; never past ceil16(len)
+                        const int nb = (valid + 15) >> 4;     // 16-row units; never past ceil16(len)
                         mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
-                        for (int bx = 0; bx < nb; ++bx) {
-                            int32_t ky, vy;
-                            if (MODE == kModePaged) {
+                        if (MODE == kModePaged) {             // one 16-row box per page
+                            for (int bx = 0; bx < nb; ++bx) {
                                 const int64_t prow =
                                     (static_cast<int64_t>(pages[t * 4 + bx]) * p.kv_heads + head) * 16;
-                                ky = static_cast<int32_t>(k_array + prow);
-                                vy = static_cast<int32_t>(v_array + prow);
-                            } else {
-                                ky = static_cast<int32_t>(k_array + row + t * kTile + bx * 16);
-                                vy = static_cast<int32_t>(v_array + row + t * kTile + bx * 16);
+                                const int32_t ky = static_cast<int32_t>(k_array + prow);
+                                const int32_t vy = static_cast<int32_t>(v_array + prow);
+#pragma unroll
+                                for (int h = 0; h < HALVES; ++h) {
+                                    tma_load_2d(kdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, ky,
+                                                full_bar(stage));
+                                    tma_load_2d(vdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, vy,
+                                                full_bar(stage));
+                                }
                             }
+                        } else {                              // a ragged tail: one box of 16, 32 or 48 rows
+                            const CUtensorMap* box = &tm.box[nb - 1];
+                            const int32_t ky = static_cast<int32_t>(k_array + row + t * kTile);
+                            const int32_t vy = static_cast<int32_t>(v_array + row + t * kTile);
 #pragma unroll
                             for (int h = 0; h < HALVES; ++h) {
-                                tma_load_2d(kdst + h * HALF_BYTES + bx * 2048, &tm_small, h * 64, ky,
-                                            full_bar(stage));
-                                tma_load_2d(vdst + h * HALF_BYTES + bx * 2048, &tm_small, h * 64, vy,
-                                            full_bar(stage));
+                                tma_load_2d(kdst + h * HALF_BYTES, box, h * 64, ky, full_bar(stage));
+                                tma_load_2d(vdst + h * HALF_BYTES, box, h * 64, vy, full_bar(stage));
                             }
                         }
                     }
@@ -1209,7 +1213,7 @@ cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, maps.big, maps.small, p, lens);
+    return cudaLaunchKernelEx(&cfg, kern, maps, p, lens);
 }
 
 template <int D, int NT>

@@ -52,8 +52,7 @@ struct InlineLens {
 };
 
 struct TensorMaps {
-    CUtensorMap big;    // box 64 rows x 64 elements
-    CUtensorMap small;  // box 16 rows x 64 elements
+    CUtensorMap box[4];   // boxes of 16, 32, 48 and 64 rows x 64 elements (box[k]: 16 (k+1) rows)
 };
 
 enum DecodeMode { kModeSlab = 0, kModePaged = 1, kModeProbe = 2 };
