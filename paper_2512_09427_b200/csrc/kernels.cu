@@ -182,6 +182,8 @@ struct TcConfig {
     static constexpr int kKvTileBytes = kTile * D * 2;
     static constexpr int kStageBytes = 2 * kKvTileBytes;
     static constexpr int kQBytes = kRows * D * 2;
+    static constexpr int kNewBytes = 2 * D * 2;            // the step's new K row and V row of the item's stream
+    static constexpr int kQSlotBytes = kQBytes + kNewBytes;
     static constexpr int kMoStride = D + 4;
     static constexpr int kMergeFloats = kConsumerWarps * kRows * kMoStride;
     static constexpr int kMlFloats = kConsumerWarps * kRows * 2;
@@ -190,7 +192,7 @@ struct TcConfig {
                                        kMaxQSlots * 32 + kNumBars * 8 + 64;
     static constexpr int kAlignSlack = 1024;
     static int smem_bytes(int stages, int q_slots) {
-        return stages * kStageBytes + q_slots * kQBytes + kFixedBytes + kAlignSlack;
+        return stages * kStageBytes + q_slots * kQSlotBytes + kFixedBytes + kAlignSlack;
     }
 };
 
@@ -268,7 +270,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* kv = smem;
     uint8_t* qbuf = kv + STAGES * Cfg::kStageBytes;
-    float* mrg_o = reinterpret_cast<float*>(qbuf + QSLOTS * Cfg::kQBytes);
+    float* mrg_o = reinterpret_cast<float*>(qbuf + QSLOTS * Cfg::kQSlotBytes);
     float* mrg_ml = mrg_o + kMergeBufs * Cfg::kMergeFloats;
     int* mrg_hdr = reinterpret_cast<int*>(mrg_ml + kMergeBufs * Cfg::kMlFloats);   // 8 ints per buffer
     int* desc = mrg_hdr + kMergeBufs * 8;                                           // 8 ints per slot
@@ -422,11 +424,17 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 dsc[6] = 1;                              // a real item
                 dsc[7] = has_new ? b.z + ntok : -1;      // pool row of the new token
                 const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
-                mbar_expect_tx(qfull_bar(qs), q_bytes);
-                bulk_load(q_u32 + qs * Cfg::kQBytes,
+                mbar_expect_tx(qfull_bar(qs), q_bytes + (has_new ? Cfg::kNewBytes : 0));
+                bulk_load(q_u32 + qs * Cfg::kQSlotBytes,
                           static_cast<const uint8_t*>(p.q) +
                               (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
                           q_bytes, qfull_bar(qs));
+                if (has_new) {                           // the new token's K and V rows ride behind the queries
+                    const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
+                    const uint32_t ndst = q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes;
+                    bulk_load(ndst, static_cast<const uint8_t*>(p.k_new) + nrow, D * 2, qfull_bar(qs));
+                    bulk_load(ndst + D * 2, static_cast<const uint8_t*>(p.v_new) + nrow, D * 2, qfull_bar(qs));
+                }
                 if (++qs == QSLOTS) {
                     qs = 0;
                     qphase ^= 1u;
@@ -536,23 +544,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     rr[i] = idx / PER_ROW;
                     dd[i] = (idx - rr[i] * PER_ROW) * 4;
                 }
-                // the token appended this step (if this piece ends its stream): its query, key
-                // and value parts are fetched now so that the loads fly during the merge below
-                const int new_row = hdr[5];
-                const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(p.q) +
-                                            (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group) * D;
-                const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D;
-                const __nv_bfloat16* krow = reinterpret_cast<const __nv_bfloat16*>(p.k_new) + nrow;
-                const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(p.v_new) + nrow;
-                uint2 nq[CH], nk[CH], nv[CH];
-                if (new_row >= 0) {
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) {
-                        nq[i] = __ldg(reinterpret_cast<const uint2*>(qrow + rr[i] * D + dd[i]));
-                        nk[i] = __ldg(reinterpret_cast<const uint2*>(krow + dd[i]));
-                        nv[i] = __ldg(reinterpret_cast<const uint2*>(vrow + dd[i]));
-                    }
-                }
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
                     const int r = rr[i], d0 = dd[i];
@@ -580,31 +571,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     acc[i] = a;
                     acc_m[i] = M;
                     acc_l[i] = L;
-                }
-                if (new_row >= 0) {
-                    // its score against each head (lanes that share a head add their parts up),
-                    // its value; then its K and V rows go into the slab for the steps to come
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) {
-                        const uint2 qv = nq[i], kv2 = nk[i], vv = nv[i];
-                        float dot = __uint_as_float(qv.x << 16) * __uint_as_float(kv2.x << 16);
-                        dot = fmaf(__uint_as_float(qv.x & 0xFFFF0000u), __uint_as_float(kv2.x & 0xFFFF0000u), dot);
-                        dot = fmaf(__uint_as_float(qv.y << 16), __uint_as_float(kv2.y << 16), dot);
-                        dot = fmaf(__uint_as_float(qv.y & 0xFFFF0000u), __uint_as_float(kv2.y & 0xFFFF0000u), dot);
-#pragma unroll
-                        for (int off = PER_ROW / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
-                        const float4 x = make_float4(__uint_as_float(vv.x << 16), __uint_as_float(vv.x & 0xFFFF0000u),
-                                                     __uint_as_float(vv.y << 16), __uint_as_float(vv.y & 0xFFFF0000u));
-                        lse_fold(acc_m[i], acc_l[i], acc[i], dot * p.scale_log2, 1.f, x);
-                    }
-                    constexpr int ROW_VECS = D * 2 / 16;
-                    if (ftid < 2 * ROW_VECS) {
-                        const int kv = ftid / ROW_VECS, vec = ftid - kv * ROW_VECS;
-                        const uint4* src = reinterpret_cast<const uint4*>((kv ? vrow : krow)) + vec;
-                        uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
-                                     ((static_cast<int64_t>(p.layer) * 2 + kv) * p.rows_per_array + new_row) * ROW_VECS + vec;
-                        *dst = __ldg(src);
-                    }
                 }
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
@@ -742,20 +708,13 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 #pragma unroll
                 for (int j = 0; j < D / 32; ++j) {
                     uint32_t r[4];
-                    ldmatrix_x4(r, q_u32 + qs * Cfg::kQBytes + nt * 8 * (D * 2) + q_lane_off + j * 64);
+                    ldmatrix_x4(r, q_u32 + qs * Cfg::kQSlotBytes + nt * 8 * (D * 2) + q_lane_off + j * 64);
                     qb[nt][2 * j][0] = r[0];
                     qb[nt][2 * j][1] = r[1];
                     qb[nt][2 * j + 1][0] = r[2];
                     qb[nt][2 * j + 1][1] = r[3];
                 }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(qempty_bar(qs));
-        if (++qs == QSLOTS) {
-            qs = 0;
-            qphase ^= 1u;
-        }
-
         float o[NT][D / 16][4];
         float m_run[NT][2], l_run[NT][2];
 #pragma unroll
@@ -764,6 +723,61 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             for (int i = 0; i < D / 16; ++i) o[nt][i][0] = o[nt][i][1] = o[nt][i][2] = o[nt][i][3] = 0.f;
             m_run[nt][0] = m_run[nt][1] = -INFINITY;
             l_run[nt][0] = l_run[nt][1] = 0.f;
+        }
+        if (MODE == kModeSlab && new_row >= 0 && cw == 0) {
+            // The token appended this step (the piece ends its stream and the append is fused
+            // in): its K and V rows sit behind the queries in the slot.  The group's first warp
+            // starts from it instead of from nothing: running maximum = its score, sum = 1,
+            // output = its value row; and it writes the two rows into the slab for the steps
+            // to come.  Each lane holds, of head qd, elements kk*16 + 2qt + {0, 1, 8, 9} of the
+            // query: it adds up its part of the score, the quad completes it.
+            const uint8_t* nk = qbuf + qs * Cfg::kQSlotBytes + Cfg::kQBytes;
+            const uint8_t* nv = nk + D * 2;
+            float dot[NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) dot[nt] = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t k0 = *reinterpret_cast<const uint32_t*>(nk + (kk * 16 + qt * 2) * 2);
+                const uint32_t k1 = *reinterpret_cast<const uint32_t*>(nk + (kk * 16 + qt * 2 + 8) * 2);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint32_t q0 = qb[nt][kk][0], q1 = qb[nt][kk][1];
+                    dot[nt] = fmaf(__uint_as_float(q0 << 16), __uint_as_float(k0 << 16), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q0 & 0xFFFF0000u), __uint_as_float(k0 & 0xFFFF0000u), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q1 << 16), __uint_as_float(k1 << 16), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q1 & 0xFFFF0000u), __uint_as_float(k1 & 0xFFFF0000u), dot[nt]);
+                }
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                dot[nt] += __shfl_xor_sync(0xFFFFFFFFu, dot[nt], 1);
+                dot[nt] += __shfl_xor_sync(0xFFFFFFFFu, dot[nt], 2);
+                // the accumulator columns of this lane are heads 2qt and 2qt + 1
+                m_run[nt][0] = __shfl_sync(0xFFFFFFFFu, dot[nt], qt * 8) * scale;
+                m_run[nt][1] = __shfl_sync(0xFFFFFFFFu, dot[nt], qt * 8 + 4) * scale;
+                l_run[nt][0] = l_run[nt][1] = qd == 0 ? 1.f : 0.f;      // summed over qd when the item ends
+#pragma unroll
+                for (int dt = 0; dt < D / 16; ++dt) {
+                    const uint32_t lo = *reinterpret_cast<const uint16_t*>(nv + (dt * 16 + qd) * 2);
+                    const uint32_t hi = *reinterpret_cast<const uint16_t*>(nv + (dt * 16 + qd + 8) * 2);
+                    o[nt][dt][0] = o[nt][dt][1] = __uint_as_float(lo << 16);
+                    o[nt][dt][2] = o[nt][dt][3] = __uint_as_float(hi << 16);
+                }
+            }
+            constexpr int ROW_VECS = D * 2 / 16;
+            if (lane < 2 * ROW_VECS) {                   // K row, then V row, 16 bytes per lane
+                const int kv = lane / ROW_VECS, vec = lane - kv * ROW_VECS;
+                uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
+                             ((static_cast<int64_t>(p.layer) * 2 + kv) * p.rows_per_array + new_row) * ROW_VECS + vec;
+                *dst = *reinterpret_cast<const uint4*>(nk + lane * 16);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(qempty_bar(qs));
+        if (++qs == QSLOTS) {
+            qs = 0;
+            qphase ^= 1u;
         }
 
         for (int t = 0; t < ntiles; ++t) {
@@ -901,7 +915,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             hdr[2] = direct;
             hdr[3] = slot;
             hdr[4] = comb;
-            hdr[5] = new_row;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(mready_bar(mb));
@@ -1233,14 +1246,14 @@ template <int D, int NT>
 void tc_shape_inst(int32_t ctas_per_sm, int32_t* stages, int32_t* q_slots) {
     using Cfg = TcConfig<D, NT>;
     const int budget = std::min(kSmemPerSm / ctas_per_sm - kSmemCtaReserve, kSmemPerCtaMax);
-    const int room = budget - Cfg::kFixedBytes - Cfg::kAlignSlack - kMinQSlots * Cfg::kQBytes;
+    const int room = budget - Cfg::kFixedBytes - Cfg::kAlignSlack - kMinQSlots * Cfg::kQSlotBytes;
     int n = room / Cfg::kStageBytes;
     n = n > kMaxStages ? kMaxStages : n;
     if (n < 2) {
         *stages = *q_slots = 0;
         return;
     }
-    const int extra = (room - n * Cfg::kStageBytes) / Cfg::kQBytes;
+    const int extra = (room - n * Cfg::kStageBytes) / Cfg::kQSlotBytes;
     *stages = n;
     *q_slots = std::min(kMaxQSlots, kMinQSlots + extra);
 }
