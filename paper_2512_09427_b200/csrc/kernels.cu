@@ -132,6 +132,25 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 2^x, log2 x and 1/x straight from the special-function unit (relative error about 2^-22;
+// 2^-inf = 0, which the softmax relies on).  Used where a result is rounded to bf16 or only
+// rescales one, and in the merges, whose inputs are rescaled the same way on every path.
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_log2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_rcp(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -216,8 +235,8 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float
 // depend on which CTA happens to do the merge.
 __device__ __forceinline__ void lse_fold(float& M, float& L, float4& a, float m, float l, const float4& x) {
     const float mn = fmaxf(M, m);
-    const float e0 = M == -INFINITY ? 0.f : exp2f(M - mn);
-    const float e1 = m == -INFINITY ? 0.f : exp2f(m - mn);
+    const float e0 = M == -INFINITY ? 0.f : fast_exp2(M - mn);
+    const float e1 = m == -INFINITY ? 0.f : fast_exp2(m - mn);
     L = fmaf(L, e0, l * e1);
     a.x = fmaf(a.x, e0, x.x * e1);
     a.y = fmaf(a.y, e0, x.y * e1);
@@ -246,10 +265,10 @@ __device__ __forceinline__ void combine_stream(const float* part_o, const float*
             const float4 x = ldcg4(part_o + prow * D + d0);
             lse_fold(M, L, a, ml.x, ml.y, x);
         }
-        const float inv = 1.f / L;
+        const float inv = fast_rcp(L);
         const size_t row = static_cast<size_t>(req) * q_heads + static_cast<size_t>(head) * group + r;
         store4(out + row * D + d0, a.x * inv, a.y * inv, a.z * inv, a.w * inv);
-        if (d0 == 0 && lse) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+        if (d0 == 0 && lse) lse[row] = (M + fast_log2(L)) * 0.6931471805599453f;
     }
 }
 
@@ -295,13 +314,13 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
     // the producer's first loads are in flight while the barriers are being set up
     int4 rec = make_int4(0, 0, 0, 0), first_a = rec, first_b = rec;
-    if (tid == kProducerWarp * 32) {
+    if (warp == kProducerWarp) {
         const int4* r = p.cta + 3 * cta;
         rec = __ldg(r);
         first_a = __ldg(r + 1);
         first_b = __ldg(r + 2);
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[3])) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[0])) : "memory");
+        if (lane < 4)
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[lane])) : "memory");
     } else if (warp >= kFinisherWarp0 && lane == 0) {
         rec = __ldg(p.cta + 3 * cta);
     }
@@ -325,14 +344,16 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // Programmatic dependent launch: everything above (barrier set-up, the CTA's record from the
-    // step's table, which no kernel writes) may run while the previous kernel of the stream is
-    // still draining; nothing below may.  The next kernel of the stream is let go at once: its
-    // CTAs only find room as these exit, and they wait at this same point for the whole grid.
-    // One exception, below: the producer starts the CTA's first tiles before it waits, those
-    // that hold no row a decode kernel just ahead in the stream could still be writing.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (warp != kProducerWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Programmatic dependent launch.  Everything above (barrier set-up, the CTA's record from
+    // the step's table, which no kernel writes) may run while the previous kernel of the stream
+    // is still draining; so may the producer's early loads below.  Everything else comes after
+    // the dependency wait.  The next kernel of the stream is let go only AFTER this wait: when
+    // its CTAs run their own early part, the kernel before this one is then known to be
+    // complete, so the only kernel a CTA can overlap with is its immediate predecessor.
+    if (warp != kProducerWarp) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
 
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
@@ -342,61 +363,104 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // Lane 0 issues every copy.  The other lanes only fetch item descriptors: 32 at a
         // time, one per lane, handed to lane 0 by shuffles, so that the table reads of short
         // items are off the issuing lane's critical path.
-        const int it_begin = __shfl_sync(0xFFFFFFFFu, rec.x, 0), it_end = __shfl_sync(0xFFFFFFFFu, rec.y, 0);
-        uint32_t stage = 0, phase = 0;
+        const int it_begin = rec.x, it_end = rec.y;       // every lane read the record
         uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
         bool ok = true;
         const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
         const int64_t v_array = k_array + p.rows_per_array;
-        uint32_t qs = 0, qphase = 0;
-        // Early start.  The only pool rows the previous kernel of the stream may still be
-        // writing (when it is this kernel, one step or one layer earlier) are the last two of a
-        // stream: the token it appended, and this step's position if the step is a repeat.
-        // Full tiles of the CTA's first item that end before those rows are requested now, so
-        // that HBM is already streaming when the previous grid finishes; everything else
-        // (queries, other items, ragged tiles) comes after the wait.
-        int early = 0;
-        if (lane == 0 && MODE != kModePaged && it_begin < it_end) {
-            const int tok0 = first_a.z;
-            const int ntok_now = (lens.n > 0 && (first_b.x & 2)) ? lens.len[first_a.x] - tok0 : first_a.w;
-            const int safe_tok = (first_b.x & 2) ? ntok_now - 2 : ntok_now;
-            early = min(static_cast<int>(STAGES), max(safe_tok, 0) / kTile);
-            for (int t = 0; t < early; ++t) {
-                const uint32_t kdst = kv_u32 + t * Cfg::kStageBytes;
-                const uint32_t vdst = kdst + Cfg::kKvTileBytes;
-                mbar_expect_tx(full_bar(t), Cfg::kStageBytes);
-                const int32_t ky = static_cast<int32_t>(k_array + first_b.z + t * kTile);
-                const int32_t vy = static_cast<int32_t>(v_array + first_b.z + t * kTile);
-#pragma unroll
-                for (int h = 0; h < HALVES; ++h) {
-                    tma_load_2d(kdst + h * HALF_BYTES, &tm.box[3], h * 64, ky, full_bar(t));
-                    tma_load_2d(vdst + h * HALF_BYTES, &tm.box[3], h * 64, vy, full_bar(t));
-                }
-                issued_any |= 1u << t;
-                issued_odd ^= 1u << t;
+
+        // An item's rows as this step sees them.  A piece that ends its stream ends where the
+        // stream ends NOW (the plan may be an earlier step's, made when the stream was a little
+        // shorter).  With the append fused in, the stream's last token is not in the slab yet:
+        // it is not streamed (a consumer warp takes it from k_new / v_new and writes it there).
+        // `safe` = rows that no kernel still running can be writing: the previous kernel of the
+        // stream (the only one that can overlap with this one) may be this kernel one step
+        // earlier, whose new token is the stream's last row but one; the last row is this
+        // step's own.
+        struct Rows {
+            int ntok, safe;
+            bool has_new;
+        };
+        auto rows_of = [&](const int4& a, const int4& b) {
+            Rows r;
+            const bool ends = (b.x & 2) != 0;
+            const int ntok_now = (lens.n > 0 && ends) ? lens.len[a.x] - a.z : a.w;
+            r.has_new = p.k_new != nullptr && ends;
+            r.ntok = ntok_now - (r.has_new ? 1 : 0);
+            r.safe = ends ? ntok_now - 2 : ntok_now;
+            return r;
+        };
+        // One tile of a slab stream = up to four groups of 16 rows, fetched with one copy per
+        // 128-byte column block of K and of V (a box of 16, 32, 48 or 64 rows; never past
+        // ceil16 of the stream's length).  part 0: the whole tile; part 1: only the groups that
+        // lie wholly in the safe rows, with the barrier told to expect the whole tile; part 2:
+        // the rest of a tile whose part 1 is under way.
+        auto issue_slab_tile = [&](uint32_t stage, int64_t row, int t, const Rows& r, int part) {
+            const int r0 = t * kTile;
+            const int nb = (min(kTile, r.ntok - r0) + 15) >> 4;
+            const int ge = min(nb, max(r.safe - r0, 0) >> 4);
+            const int g0 = part == 2 ? ge : 0, g1 = part == 1 ? ge : nb;
+            if (part != 2) {
+                mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                issued_any |= 1u << stage;
+                issued_odd ^= 1u << stage;
             }
-            stage = static_cast<uint32_t>(early) % STAGES;
-            phase = static_cast<uint32_t>(early) == STAGES ? 1u : 0u;
+            if (g1 <= g0) return;
+            const CUtensorMap* box = &tm.box[g1 - g0 - 1];
+            const uint32_t kdst = kv_u32 + stage * Cfg::kStageBytes + g0 * 2048;
+            const uint32_t vdst = kdst + Cfg::kKvTileBytes;
+            const int32_t ky = static_cast<int32_t>(k_array + row + r0 + g0 * 16);
+            const int32_t vy = static_cast<int32_t>(v_array + row + r0 + g0 * 16);
+#pragma unroll
+            for (int h = 0; h < HALVES; ++h) {
+                tma_load_2d(kdst + h * HALF_BYTES, box, h * 64, ky, full_bar(stage));
+                tma_load_2d(vdst + h * HALF_BYTES, box, h * 64, vy, full_bar(stage));
+            }
+        };
+
+        // descriptors of the CTA's first 32 items (the very first came with the record)
+        int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
+        if (it_begin + lane < it_end) {
+            mine_a = __ldg(p.items + 2 * (it_begin + lane));
+            mine_b = __ldg(p.items + 2 * (it_begin + lane) + 1);
+        }
+        auto item_of = [&](int j, int4& a, int4& b) {     // descriptor held by lane j, to all lanes
+            a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
+            a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
+            a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
+            a.w = __shfl_sync(0xFFFFFFFFu, mine_a.w, j);
+            b.x = __shfl_sync(0xFFFFFFFFu, mine_b.x, j);
+            b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
+            b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
+            b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
+        };
+        // Early start: the safe rows of the CTA's first tiles (one per pipeline stage) are
+        // requested before the dependency wait, so that HBM is already streaming while the
+        // previous grid finishes; queries, new tokens and the rows in flux come after it.
+        int n_early = 0;
+        if (MODE != kModePaged) {
+            for (int j = 0; j < 32 && it_begin + j < it_end && n_early < static_cast<int>(STAGES); ++j) {
+                int4 a = first_a, b = first_b;
+                if (j > 0) item_of(j, a, b);
+                const Rows r = rows_of(a, b);
+                const int ntiles = (r.ntok + kTile - 1) / kTile;
+                for (int t = 0; t < ntiles && n_early < static_cast<int>(STAGES); ++t, ++n_early)
+                    if (lane == 0) issue_slab_tile(static_cast<uint32_t>(n_early), b.z, t, r, 1);
+            }
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+        uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
+        int n_tile = 0;                               // tiles issued so far (the first n_early only need their rest)
         for (int it = it_begin;; ++it) {
             const int j = (it - it_begin) & 31;
-            if (j == 0 && it + lane < it_end) {
+            if (j == 0 && it != it_begin && it + lane < it_end) {
                 mine_a = __ldg(p.items + 2 * (it + lane));
                 mine_b = __ldg(p.items + 2 * (it + lane) + 1);
             }
-            int4 a = first_a, b = first_b;               // the first item came with the CTA record
-            if (it != it_begin) {
-                a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
-                a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
-                a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
-                a.w = __shfl_sync(0xFFFFFFFFu, mine_a.w, j);
-                b.x = __shfl_sync(0xFFFFFFFFu, mine_b.x, j);
-                b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
-                b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
-                b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
-            }
+            int4 a = first_a, b = first_b;
+            if (it != it_begin) item_of(j, a, b);
             int more = 0;
             if (lane == 0) do {
                 ok = mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit);
@@ -408,15 +472,11 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     break;
                 }
                 const int req = a.x, head = a.y, tok0 = a.z;
+                const Rows r = rows_of(a, b);
+                const int ntok = r.ntok;
+                const bool has_new = r.has_new;
                 dsc[0] = req;
                 dsc[1] = head;
-                // With the append fused in, the stream's last token is not in the slab yet: it
-                // is not streamed; the finishers take it from k_new / v_new and write it there.
-                const bool has_new = p.k_new != nullptr && (b.x & 2);
-                // a piece that ends its stream ends where the stream ends NOW (the plan may be
-                // an earlier step's, made when the stream was a little shorter)
-                const int ntok_now = (lens.n > 0 && (b.x & 2)) ? lens.len[req] - tok0 : a.w;
-                const int ntok = ntok_now - (has_new ? 1 : 0);
                 dsc[2] = ntok;
                 dsc[3] = b.x & 1;                        // direct
                 dsc[4] = b.y;                            // slot
@@ -440,55 +500,35 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     qphase ^= 1u;
                 }
                 const int64_t row = b.z;
-                const int32_t* pages = nullptr;
-                if (MODE == kModePaged)
-                    pages = p.page_table + static_cast<size_t>(req) * p.max_pages + tok0 / 16;
                 const int ntiles = (ntok + kTile - 1) / kTile;
-                for (int t = (it == it_begin ? early : 0); t < ntiles; ++t) {   // the early tiles are under way
-                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit);
-                    if (!ok) break;
-                    const int valid = min(kTile, ntok - t * kTile);
-                    const uint32_t kdst = kv_u32 + stage * Cfg::kStageBytes;
-                    const uint32_t vdst = kdst + Cfg::kKvTileBytes;
-                    if (MODE != kModePaged && valid == kTile) {
-                        mbar_expect_tx(full_bar(stage), Cfg::kStageBytes);
-                        const int32_t ky = static_cast<int32_t>(k_array + row + t * kTile);
-                        const int32_t vy = static_cast<int32_t>(v_array + row + t * kTile);
-#pragma unroll
-                        for (int h = 0; h < HALVES; ++h) {
-                            tma_load_2d(kdst + h * HALF_BYTES, &tm.box[3], h * 64, ky, full_bar(stage));
-                            tma_load_2d(vdst + h * HALF_BYTES, &tm.box[3], h * 64, vy, full_bar(stage));
-                        }
+                for (int t = 0; t < ntiles; ++t, ++n_tile) {
+                    if (n_tile < n_early) {              // first use of the stage, part 1 under way
+                        issue_slab_tile(stage, row, t, r, 2);
                     } else {
-                        const int nb = (valid + 15) >> 4;     // 16-row units; never past ceil16(len)
-                        mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
-                        if (MODE == kModePaged) {             // one 16-row box per page
+                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit);
+                        if (!ok) break;
+                        if (MODE != kModePaged) {
+                            issue_slab_tile(stage, row, t, r, 0);
+                        } else {                         // one 16-row box per page
+                            const int32_t* pages = p.page_table + static_cast<size_t>(req) * p.max_pages + tok0 / 16;
+                            const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
+                            const uint32_t kdst = kv_u32 + stage * Cfg::kStageBytes;
+                            const uint32_t vdst = kdst + Cfg::kKvTileBytes;
+                            mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                            issued_any |= 1u << stage;
+                            issued_odd ^= 1u << stage;
                             for (int bx = 0; bx < nb; ++bx) {
-                                const int64_t prow =
-                                    (static_cast<int64_t>(pages[t * 4 + bx]) * p.kv_heads + head) * 16;
+                                const int64_t prow = (static_cast<int64_t>(pages[t * 4 + bx]) * p.kv_heads + head) * 16;
                                 const int32_t ky = static_cast<int32_t>(k_array + prow);
                                 const int32_t vy = static_cast<int32_t>(v_array + prow);
 #pragma unroll
                                 for (int h = 0; h < HALVES; ++h) {
-                                    tma_load_2d(kdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, ky,
-                                                full_bar(stage));
-                                    tma_load_2d(vdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, vy,
-                                                full_bar(stage));
+                                    tma_load_2d(kdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, ky, full_bar(stage));
+                                    tma_load_2d(vdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, vy, full_bar(stage));
                                 }
-                            }
-                        } else {                              // a ragged tail: one box of 16, 32 or 48 rows
-                            const CUtensorMap* box = &tm.box[nb - 1];
-                            const int32_t ky = static_cast<int32_t>(k_array + row + t * kTile);
-                            const int32_t vy = static_cast<int32_t>(v_array + row + t * kTile);
-#pragma unroll
-                            for (int h = 0; h < HALVES; ++h) {
-                                tma_load_2d(kdst + h * HALF_BYTES, box, h * 64, ky, full_bar(stage));
-                                tma_load_2d(vdst + h * HALF_BYTES, box, h * 64, vy, full_bar(stage));
                             }
                         }
                     }
-                    issued_any |= 1u << stage;
-                    issued_odd ^= 1u << stage;
                     if (++stage == STAGES) {
                         stage = 0;
                         phase ^= 1u;
@@ -561,7 +601,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float e = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);   // warps without keys
+                        const float e = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);   // warps without keys
                         L = fmaf(lw[w], e, L);
                         a.x = fmaf(x[w].x, e, a.x);
                         a.y = fmaf(x[w].y, e, a.y);
@@ -577,10 +617,10 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     if (ftid + i * fthreads >= total) continue;
                     const int r = rr[i], d0 = dd[i];
                     if (direct) {
-                        const float inv = 1.f / acc_l[i];
+                        const float inv = fast_rcp(acc_l[i]);
                         const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
                         store4(out + row * D + d0, acc[i].x * inv, acc[i].y * inv, acc[i].z * inv, acc[i].w * inv);
-                        if (d0 == 0 && p.lse) p.lse[row] = (acc_m[i] + log2f(acc_l[i])) * 0.6931471805599453f;
+                        if (d0 == 0 && p.lse) p.lse[row] = (acc_m[i] + fast_log2(acc_l[i])) * 0.6931471805599453f;
                     } else {
                         const size_t prow = static_cast<size_t>(slot) * group + r;
                         *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = acc[i];
@@ -641,9 +681,9 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
                     if (ftid + i * fthreads >= total) continue;
-                    const float inv = 1.f / fl[i];
+                    const float inv = fast_rcp(fl[i]);
                     store4(out + (orow0 + rr[i]) * D + dd[i], fa[i].x * inv, fa[i].y * inv, fa[i].z * inv, fa[i].w * inv);
-                    if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + log2f(fl[i])) * 0.6931471805599453f;
+                    if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + fast_log2(fl[i])) * 0.6931471805599453f;
                 }
             }
         }
@@ -831,9 +871,9 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     }
                     const float mn0 = fmaxf(m_run[nt][0], mx0 * scale), mn1 = fmaxf(m_run[nt][1], mx1 * scale);
                     const float mu0 = (mn0 == -INFINITY) ? 0.f : mn0, mu1 = (mn1 == -INFINITY) ? 0.f : mn1;
-                    const float corr0 = exp2f(m_run[nt][0] - mu0), corr1 = exp2f(m_run[nt][1] - mu1);
-                    const float p0 = exp2f(fmaf(c0, scale, -mu0)), p1 = exp2f(fmaf(c1, scale, -mu1));
-                    const float p2 = exp2f(fmaf(c2, scale, -mu0)), p3 = exp2f(fmaf(c3, scale, -mu1));
+                    const float corr0 = fast_exp2(m_run[nt][0] - mu0), corr1 = fast_exp2(m_run[nt][1] - mu1);
+                    const float p0 = fast_exp2(fmaf(c0, scale, -mu0)), p1 = fast_exp2(fmaf(c1, scale, -mu1));
+                    const float p2 = fast_exp2(fmaf(c2, scale, -mu0)), p3 = fast_exp2(fmaf(c3, scale, -mu1));
                     l_run[nt][0] = fmaf(l_run[nt][0], corr0, p0 + p2);
                     l_run[nt][1] = fmaf(l_run[nt][1], corr1, p1 + p3);
                     m_run[nt][0] = mn0;
