@@ -314,6 +314,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
     // the producer's first loads are in flight while the barriers are being set up
     int4 rec = make_int4(0, 0, 0, 0), first_a = rec, first_b = rec;
+    int4 mine_a = rec, mine_b = rec;                 // producer: descriptor of item `lane` of the CTA's current 32
     if (warp == kProducerWarp) {
         const int4* r = p.cta + 3 * cta;
         rec = __ldg(r);
@@ -324,23 +325,21 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     } else if (warp >= kFinisherWarp0 && lane == 0) {
         rec = __ldg(p.cta + 3 * cta);
     }
-    if (tid == 0) {
-        for (uint32_t s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), 1);
-            mbar_init(empty_bar(s), kConsumerGroups * kConsumerWarps);
+    if (tid < kNumBars) {                            // one barrier per thread
+        constexpr uint32_t all_consumers = kConsumerGroups * kConsumerWarps;
+        const uint32_t b = static_cast<uint32_t>(tid);
+        const uint32_t count = b < kMaxStages                        ? 1u               // full
+                               : b < 2 * kMaxStages                  ? all_consumers    // empty
+                               : b < 2 * kMaxStages + kMaxQSlots     ? 1u               // query slot full
+                               : b < 2 * kMaxStages + 2 * kMaxQSlots ? all_consumers    // query slot empty
+                               : b < 2 * kMaxStages + 2 * kMaxQSlots + kMergeBufs
+                                   ? static_cast<uint32_t>(kConsumerWarps)              // merge buffer ready
+                                   : static_cast<uint32_t>(kFinisherWarps);             // done / stored / counted
+        mbar_init(bar0 + 8u * b, count);
+        if (tid == 0) {
+            *abort_flag = 0;
+            *last_flag = 0;
         }
-        for (uint32_t s = 0; s < QSLOTS; ++s) {
-            mbar_init(qfull_bar(s), 1);
-            mbar_init(qempty_bar(s), kConsumerGroups * kConsumerWarps);
-        }
-        for (uint32_t s = 0; s < kMergeBufs; ++s) {
-            mbar_init(mready_bar(s), kConsumerWarps);
-            mbar_init(mdone_bar(s), kFinisherWarps);
-        }
-        mbar_init(fstored_bar, kFinisherWarps);
-        mbar_init(fcounted_bar, kFinisherWarps);
-        *abort_flag = 0;
-        *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -360,14 +359,18 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        // Lane 0 issues every copy.  The other lanes only fetch item descriptors: 32 at a
-        // time, one per lane, handed to lane 0 by shuffles, so that the table reads of short
-        // items are off the issuing lane's critical path.
+        // Every lane fetches item descriptors (32 at a time, one per lane) and works out its
+        // item's rows; the values reach all lanes by shuffles.  Waits are taken by the whole
+        // warp; lane 0 arms the barriers; a tile's copies (one per 128-byte column block of K
+        // and of V) are issued by as many lanes at once, so are the copies of an item's
+        // queries and new K / V rows: the time the warp spends per copy is what bounds the
+        // rate of short items.
         const int it_begin = rec.x, it_end = rec.y;       // every lane read the record
         uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
         bool ok = true;
         const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
         const int64_t v_array = k_array + p.rows_per_array;
+        constexpr int COPIES = 2 * HALVES;            // copies per box position: K and V, each column block
 
         // An item's rows as this step sees them.  A piece that ends its stream ends where the
         // stream ends NOW (the plan may be an earlier step's, made when the stream was a little
@@ -394,37 +397,41 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // 128-byte column block of K and of V (a box of 16, 32, 48 or 64 rows; never past
         // ceil16 of the stream's length).  part 0: the whole tile; part 1: only the groups that
         // lie wholly in the safe rows, with the barrier told to expect the whole tile; part 2:
-        // the rest of a tile whose part 1 is under way.
-        auto issue_slab_tile = [&](uint32_t stage, int64_t row, int t, const Rows& r, int part) {
+        // the rest of a tile whose part 1 is under way.  Called by the whole warp.
+        auto issue_slab_tile = [&](uint32_t stage, int64_t row, int t, int ntok, int safe, int part) {
             const int r0 = t * kTile;
-            const int nb = (min(kTile, r.ntok - r0) + 15) >> 4;
-            const int ge = min(nb, max(r.safe - r0, 0) >> 4);
+            const int nb = (min(kTile, ntok - r0) + 15) >> 4;
+            const int ge = min(nb, max(safe - r0, 0) >> 4);
             const int g0 = part == 2 ? ge : 0, g1 = part == 1 ? ge : nb;
             if (part != 2) {
-                mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                if (lane == 0) mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
                 issued_any |= 1u << stage;
                 issued_odd ^= 1u << stage;
+                __syncwarp();
             }
-            if (g1 <= g0) return;
-            const CUtensorMap* box = &tm.box[g1 - g0 - 1];
-            const uint32_t kdst = kv_u32 + stage * Cfg::kStageBytes + g0 * 2048;
-            const uint32_t vdst = kdst + Cfg::kKvTileBytes;
-            const int32_t ky = static_cast<int32_t>(k_array + row + r0 + g0 * 16);
-            const int32_t vy = static_cast<int32_t>(v_array + row + r0 + g0 * 16);
-#pragma unroll
-            for (int h = 0; h < HALVES; ++h) {
-                tma_load_2d(kdst + h * HALF_BYTES, box, h * 64, ky, full_bar(stage));
-                tma_load_2d(vdst + h * HALF_BYTES, box, h * 64, vy, full_bar(stage));
-            }
+            if (g1 <= g0 || lane >= COPIES) return;
+            const int h = lane >> 1, kv = lane & 1;
+            const uint32_t dst = kv_u32 + stage * Cfg::kStageBytes + kv * Cfg::kKvTileBytes + g0 * 2048 + h * HALF_BYTES;
+            const int32_t y = static_cast<int32_t>((kv ? v_array : k_array) + row + r0 + g0 * 16);
+            tma_load_2d(dst, &tm.box[g1 - g0 - 1], h * 64, y, full_bar(stage));
         };
 
-        // descriptors of the CTA's first 32 items (the very first came with the record)
-        int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
+        // descriptors of the CTA's first 32 items (the very first came with the record), each
+        // lane's resolved on the spot: n_tokens becomes the rows to stream, the combine word's
+        // place is kept, and the safe row count travels in a register of its own
+        int mine_safe = 0;
+        auto resolve_mine = [&]() {
+            const Rows r = rows_of(mine_a, mine_b);
+            mine_a.w = r.ntok;
+            mine_safe = r.safe;
+        };
         if (it_begin + lane < it_end) {
             mine_a = __ldg(p.items + 2 * (it_begin + lane));
             mine_b = __ldg(p.items + 2 * (it_begin + lane) + 1);
+            resolve_mine();
         }
-        auto item_of = [&](int j, int4& a, int4& b) {     // descriptor held by lane j, to all lanes
+        const Rows first_r = rows_of(first_a, first_b);
+        auto item_of = [&](int j, int4& a, int4& b, int& safe) {     // item held by lane j, to all lanes
             a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
             a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
             a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
@@ -433,6 +440,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
             b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
             b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
+            safe = __shfl_sync(0xFFFFFFFFu, mine_safe, j);
         };
         // Early start: the safe rows of the CTA's first tiles (one per pipeline stage) are
         // requested before the dependency wait, so that HBM is already streaming while the
@@ -441,11 +449,12 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         if (MODE != kModePaged) {
             for (int j = 0; j < 32 && it_begin + j < it_end && n_early < static_cast<int>(STAGES); ++j) {
                 int4 a = first_a, b = first_b;
-                if (j > 0) item_of(j, a, b);
-                const Rows r = rows_of(a, b);
-                const int ntiles = (r.ntok + kTile - 1) / kTile;
+                int safe = first_r.safe;
+                a.w = first_r.ntok;
+                if (j > 0) item_of(j, a, b, safe);
+                const int ntiles = (a.w + kTile - 1) / kTile;
                 for (int t = 0; t < ntiles && n_early < static_cast<int>(STAGES); ++t, ++n_early)
-                    if (lane == 0) issue_slab_tile(static_cast<uint32_t>(n_early), b.z, t, r, 1);
+                    issue_slab_tile(static_cast<uint32_t>(n_early), b.z, t, a.w, safe, 1);
             }
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -458,23 +467,26 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             if (j == 0 && it != it_begin && it + lane < it_end) {
                 mine_a = __ldg(p.items + 2 * (it + lane));
                 mine_b = __ldg(p.items + 2 * (it + lane) + 1);
+                resolve_mine();
             }
             int4 a = first_a, b = first_b;
-            if (it != it_begin) item_of(j, a, b);
-            int more = 0;
-            if (lane == 0) do {
-                ok = mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit);
-                if (!ok) break;
-                int* dsc = desc + qs * 8;
-                if (it >= it_end) {                      // end marker
+            int safe = first_r.safe;
+            a.w = first_r.ntok;
+            if (it != it_begin) item_of(j, a, b, safe);
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit));
+            if (!ok) break;
+            int* dsc = desc + qs * 8;
+            if (it >= it_end) {                          // end marker
+                if (lane == 0) {
                     dsc[6] = 0;
                     mbar_arrive(qfull_bar(qs));
-                    break;
                 }
-                const int req = a.x, head = a.y, tok0 = a.z;
-                const Rows r = rows_of(a, b);
-                const int ntok = r.ntok;
-                const bool has_new = r.has_new;
+                break;
+            }
+            const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
+            const bool has_new = p.k_new != nullptr && (b.x & 2);
+            const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
+            if (lane == 0) {
                 dsc[0] = req;
                 dsc[1] = head;
                 dsc[2] = ntok;
@@ -483,60 +495,56 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 dsc[5] = b.w;                            // combine record
                 dsc[6] = 1;                              // a real item
                 dsc[7] = has_new ? b.z + ntok : -1;      // pool row of the new token
-                const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
                 mbar_expect_tx(qfull_bar(qs), q_bytes + (has_new ? Cfg::kNewBytes : 0));
+            }
+            __syncwarp();
+            if (lane == 0) {
                 bulk_load(q_u32 + qs * Cfg::kQSlotBytes,
                           static_cast<const uint8_t*>(p.q) +
                               (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
                           q_bytes, qfull_bar(qs));
-                if (has_new) {                           // the new token's K and V rows ride behind the queries
-                    const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
-                    const uint32_t ndst = q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes;
-                    bulk_load(ndst, static_cast<const uint8_t*>(p.k_new) + nrow, D * 2, qfull_bar(qs));
-                    bulk_load(ndst + D * 2, static_cast<const uint8_t*>(p.v_new) + nrow, D * 2, qfull_bar(qs));
-                }
-                if (++qs == QSLOTS) {
-                    qs = 0;
-                    qphase ^= 1u;
-                }
-                const int64_t row = b.z;
-                const int ntiles = (ntok + kTile - 1) / kTile;
-                for (int t = 0; t < ntiles; ++t, ++n_tile) {
-                    if (n_tile < n_early) {              // first use of the stage, part 1 under way
-                        issue_slab_tile(stage, row, t, r, 2);
-                    } else {
-                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit);
-                        if (!ok) break;
-                        if (MODE != kModePaged) {
-                            issue_slab_tile(stage, row, t, r, 0);
-                        } else {                         // one 16-row box per page
-                            const int32_t* pages = p.page_table + static_cast<size_t>(req) * p.max_pages + tok0 / 16;
-                            const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
-                            const uint32_t kdst = kv_u32 + stage * Cfg::kStageBytes;
-                            const uint32_t vdst = kdst + Cfg::kKvTileBytes;
-                            mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
-                            issued_any |= 1u << stage;
-                            issued_odd ^= 1u << stage;
-                            for (int bx = 0; bx < nb; ++bx) {
-                                const int64_t prow = (static_cast<int64_t>(pages[t * 4 + bx]) * p.kv_heads + head) * 16;
-                                const int32_t ky = static_cast<int32_t>(k_array + prow);
-                                const int32_t vy = static_cast<int32_t>(v_array + prow);
-#pragma unroll
-                                for (int h = 0; h < HALVES; ++h) {
-                                    tma_load_2d(kdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, ky, full_bar(stage));
-                                    tma_load_2d(vdst + h * HALF_BYTES + bx * 2048, &tm.box[0], h * 64, vy, full_bar(stage));
-                                }
-                            }
+            } else if (lane < 3 && has_new) {            // the new token's K and V rows ride behind the queries
+                const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
+                const uint8_t* src = static_cast<const uint8_t*>(lane == 1 ? p.k_new : p.v_new) + nrow;
+                bulk_load(q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes + (lane - 1) * D * 2, src, D * 2, qfull_bar(qs));
+            }
+            if (++qs == QSLOTS) {
+                qs = 0;
+                qphase ^= 1u;
+            }
+            const int64_t row = b.z;
+            const int ntiles = (ntok + kTile - 1) / kTile;
+            for (int t = 0; t < ntiles; ++t, ++n_tile) {
+                if (n_tile < n_early) {                  // first use of the stage, part 1 under way
+                    issue_slab_tile(stage, row, t, ntok, safe, 2);
+                } else {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit));
+                    if (!ok) break;
+                    if (MODE != kModePaged) {
+                        issue_slab_tile(stage, row, t, ntok, safe, 0);
+                    } else {                             // one 16-row box per page, all of them at once
+                        const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
+                        if (lane == 0) mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                        issued_any |= 1u << stage;
+                        issued_odd ^= 1u << stage;
+                        __syncwarp();
+                        const int bx = lane / COPIES, w = lane - bx * COPIES;
+                        if (bx < nb) {
+                            const int h = w >> 1, kv = w & 1;
+                            const int32_t page = p.page_table[static_cast<size_t>(req) * p.max_pages + tok0 / 16 + t * 4 + bx];
+                            const int64_t prow = (static_cast<int64_t>(page) * p.kv_heads + head) * 16;
+                            tma_load_2d(kv_u32 + stage * Cfg::kStageBytes + kv * Cfg::kKvTileBytes + h * HALF_BYTES + bx * 2048,
+                                        &tm.box[0], h * 64, static_cast<int32_t>((kv ? v_array : k_array) + prow),
+                                        full_bar(stage));
                         }
                     }
-                    if (++stage == STAGES) {
-                        stage = 0;
-                        phase ^= 1u;
-                    }
                 }
-                more = ok ? 1 : 0;
-            } while (false);
-            if (!__shfl_sync(0xFFFFFFFFu, more, 0)) break;
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            if (!ok) break;
         }
         if (lane == 0 && !ok) {
             // Something timed out.  Before the CTA's shared memory can be handed to another
