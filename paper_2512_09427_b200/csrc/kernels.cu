@@ -160,7 +160,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // decode attention, tensor-core path (bf16, head_dim 64 or 128, group <= 16)
 // =============================================================================================
 //
-// Roles: warps 0..7 consume, warp 8 produces, warps 9..11 finish.  A pipeline stage holds one
+// Roles: warps 0..7 consume, warp 8 streams the K/V tiles, warp 9 hands out the items (their
+// descriptors, queries and new K/V rows), warps 10..11 finish.  A pipeline stage holds one
 // tile of 64 keys and 64 values of one stream, written by TMA with the 128-byte swizzle so
 // that ldmatrix reads are conflict-free.  The tiles of the CTA's item list are numbered in the
 // order they are streamed; tile n belongs to consumer warp n mod 8, whole: the warp computes
@@ -195,11 +196,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kFinisherWarp0 = kProducerWarp + 1;
-constexpr int kFinisherWarps = 3;                 // 12 warps in all: three per scheduler, 168 registers each
+constexpr int kProducerWarp = kConsumerWarps;     // streams the K/V tiles
+constexpr int kQueryWarp = kProducerWarp + 1;     // hands out the items: descriptors, queries, new K/V rows
+constexpr int kFinisherWarp0 = kQueryWarp + 1;
+constexpr int kFinisherWarps = 2;                 // 12 warps in all: three per scheduler, 168 registers each
 constexpr int kFinisherThreads = kFinisherWarps * 32;
-constexpr int kTcThreads = kConsumerThreads + 32 + kFinisherThreads;
+constexpr int kTcThreads = kConsumerThreads + 2 * 32 + kFinisherThreads;
 constexpr int kTile = 64;
 constexpr int kKeyBlocks = kTile / 16;
 constexpr int kMaxStages = 8;
@@ -431,9 +433,9 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        // Waits are taken by the whole warp; lane 0 tags the stages and arms the barriers; a
-        // tile's copies (one per 128-byte column block of K and of V) are issued by as many
-        // lanes at once, so are the copies of an item's queries and new K / V rows.
+        // Streams the tiles of the CTA's items in order.  Waits are taken by the whole warp;
+        // lane 0 tags the stages and arms the barriers; a tile's copies (one per 128-byte column
+        // block of K and of V) are issued by as many lanes at once.
         const int it_begin = rec.x, it_end = rec.y;       // every lane read the record
         uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
         bool ok = true;
@@ -488,54 +490,16 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-        uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
+        uint32_t stage = 0, phase = 0;
         int n_tile = 0;                               // tiles issued so far (the first n_early only need their rest)
-        for (int it = it_begin;; ++it) {
+        for (int it = it_begin; it < it_end && ok; ++it) {
             const int j = (it - it_begin) & 31;
             if (j == 0 && it != it_begin) fetch_items(it, it_end);
             int4 a = first_a, b = first_b;
             int safe = first_r.safe;
             a.w = first_r.ntok;
             if (it != it_begin) item_of(j, a, b, safe);
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit));
-            if (!ok) break;
-            int* dsc = desc + qs * 8;
-            if (it >= it_end) {                          // end marker
-                if (lane == 0) {
-                    dsc[6] = 0;
-                    mbar_arrive(qfull_bar(qs));
-                }
-                break;
-            }
             const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
-            const bool has_new = p.k_new != nullptr && (b.x & 2);
-            const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
-            if (lane == 0) {
-                dsc[0] = req;
-                dsc[1] = head;
-                dsc[2] = ntok;
-                dsc[3] = b.x & 1;                        // direct
-                dsc[4] = b.y;                            // slot
-                dsc[5] = b.w;                            // combine record
-                dsc[6] = 1;                              // a real item
-                dsc[7] = has_new ? b.z + ntok : -1;      // pool row of the new token
-                mbar_expect_tx(qfull_bar(qs), q_bytes + (has_new ? Cfg::kNewBytes : 0));
-            }
-            __syncwarp();
-            if (lane == 0) {
-                bulk_load(q_u32 + qs * Cfg::kQSlotBytes,
-                          static_cast<const uint8_t*>(p.q) +
-                              (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
-                          q_bytes, qfull_bar(qs));
-            } else if (lane < 3 && has_new) {            // the new token's K and V rows ride behind the queries
-                const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
-                const uint8_t* src = static_cast<const uint8_t*>(lane == 1 ? p.k_new : p.v_new) + nrow;
-                bulk_load(q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes + (lane - 1) * D * 2, src, D * 2, qfull_bar(qs));
-            }
-            if (++qs == QSLOTS) {
-                qs = 0;
-                qphase ^= 1u;
-            }
             const int64_t row = b.z;
             const int ntiles = (ntok + kTile - 1) / kTile;
             for (int t = 0; t < ntiles; ++t, ++n_tile) {
@@ -565,7 +529,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     phase ^= 1u;
                 }
             }
-            if (!ok) break;
         }
         if (lane == 0 && !ok) {
             // Something timed out.  Before the CTA's shared memory can be handed to another
@@ -574,6 +537,64 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
                     mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
                                    limit / 4 + 1);
+        }
+        return;
+    }
+
+    if (warp == kQueryWarp) {
+        // ------------------------------------------------------------------ query warp
+        // One ring slot per item: its descriptor, the queries of its GQA group and, with the
+        // append fused in, the stream's new K and V rows behind them (one copy each, from three
+        // lanes at once).  Runs as far ahead of the consumers as the ring is deep.
+        const int it_begin = rec.x, it_end = rec.y;
+        fetch_items(it_begin, it_end);
+        const Rows first_r = rows_of(first_a, first_b);
+        uint32_t qs = 0, qphase = 0;
+        for (int it = it_begin;; ++it) {
+            const int j = (it - it_begin) & 31;
+            if (j == 0 && it != it_begin) fetch_items(it, it_end);
+            int4 a = first_a, b = first_b;
+            int safe = first_r.safe;
+            a.w = first_r.ntok;
+            if (it != it_begin) item_of(j, a, b, safe);
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit))) break;
+            int* dsc = desc + qs * 8;
+            if (it >= it_end) {                          // end marker
+                if (lane == 0) {
+                    dsc[6] = 0;
+                    mbar_arrive(qfull_bar(qs));
+                }
+                break;
+            }
+            const int req = a.x, head = a.y, ntok = a.w;
+            const bool has_new = p.k_new != nullptr && (b.x & 2);
+            const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
+            if (lane == 0) {
+                dsc[0] = req;
+                dsc[1] = head;
+                dsc[2] = ntok;
+                dsc[3] = b.x & 1;                        // direct
+                dsc[4] = b.y;                            // slot
+                dsc[5] = b.w;                            // combine record
+                dsc[6] = 1;                              // a real item
+                dsc[7] = has_new ? b.z + ntok : -1;      // pool row of the new token
+                mbar_expect_tx(qfull_bar(qs), q_bytes + (has_new ? Cfg::kNewBytes : 0));
+            }
+            __syncwarp();
+            if (lane == 0) {
+                bulk_load(q_u32 + qs * Cfg::kQSlotBytes,
+                          static_cast<const uint8_t*>(p.q) +
+                              (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
+                          q_bytes, qfull_bar(qs));
+            } else if (lane < 3 && has_new) {
+                const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
+                const uint8_t* src = static_cast<const uint8_t*>(lane == 1 ? p.k_new : p.v_new) + nrow;
+                bulk_load(q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes + (lane - 1) * D * 2, src, D * 2, qfull_bar(qs));
+            }
+            if (++qs == QSLOTS) {
+                qs = 0;
+                qphase ^= 1u;
+            }
         }
         return;
     }
