@@ -160,29 +160,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // decode attention, tensor-core path (bf16, head_dim 64 or 128, group <= 16)
 // =============================================================================================
 //
-// Roles: warps 0..7 consume, warp 8 streams the K/V tiles, warp 9 hands out the items (their
-// descriptors, queries and new K/V rows), warps 10..11 finish.  A pipeline stage holds one
-// tile of 64 keys and 64 values of one stream, written by TMA with the 128-byte swizzle so
-// that ldmatrix reads are conflict-free.  The tiles of the CTA's item list are numbered in the
-// order they are streamed; tile n belongs to consumer warp n mod 8, whole: the warp computes
-// all 64 keys of it (four blocks of 16, independent chains that hide each other's latency)
-// and frees the stage by itself, so up to one tile per pipeline stage is being worked on at
-// any time and short items (one or two tiles each) run side by side instead of one after the
-// other.  A warp keeps a running (max, sum, output) over its tiles of the current item.
-//   * An item of one tile that is a whole stream is finished by its warp alone: it transposes
-//     the result through its own slot of shared memory and writes it out.
-//   * Otherwise the warps that had tiles of the item (up to 8) leave their partial results in
-//     their slots; the finisher warps merge them in warp order, write the item's result (or
-//     partial result) to global memory and, for a split stream, count the piece in and merge
-//     all pieces if it was the last one.
-// Queries and item descriptors travel through a ring of 4..8 slots so the producer can run
-// several short items ahead of the consumers; every consumer warp reads every descriptor (it
-// tells the warp which tiles are its own).
-//
-// A consumer waits for a tile it has not been following, so the barrier's parity alone cannot
-// tell it which phase the stage is in (two phases look alike).  The producer therefore writes
-// the tile's number into the stage's tag before it arms the barrier; the consumer waits for
-// the tag, then for the barrier.
+// Roles: warps 0..7 consume (two groups of four), warp 8 produces, warps 9.. finish.  A
+// pipeline stage holds one tile of 64 keys and 64 values of one stream, written by TMA with the
+// 128-byte swizzle so that ldmatrix reads are conflict-free.  The CTA's items go to the two
+// consumer groups in turn (short items are latency chains; two in flight hide each other).
+// Warp w of a group owns keys [16w, 16w+16) of every tile of the group's item and keeps its own
+// running (max, sum, output).  When an item ends the four warps drop their partial results
+// into the group's merge buffer and go straight on to the group's next item; the finisher warps merge the four, write the item's result (or partial result) to
+// global memory and, for a split stream, count the piece in and merge all pieces if it was
+// the last one.  Queries and item descriptors travel through a ring of 4..8 slots so the
+// producer can run several short items ahead of the consumers.
 //
 // The contraction is arranged with the KEYS on the M side of the MMA tiles and the query heads
 // of the GQA group on the N side (8 heads per n-tile; columns >= group hold whatever the
@@ -194,20 +181,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // softmax weights go from the first product's accumulator to the second product's B operand
 // with one 8x8 register transpose (movmatrix) per eight keys.
 
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kProducerWarp = kConsumerWarps;     // streams the K/V tiles
-constexpr int kQueryWarp = kProducerWarp + 1;     // hands out the items: descriptors, queries, new K/V rows
-constexpr int kFinisherWarp0 = kQueryWarp + 1;
-constexpr int kFinisherWarps = 2;                 // 12 warps in all: three per scheduler, 168 registers each
+constexpr int kConsumerWarps = 4;                 // per consumer group: one tile is shared by four warps
+constexpr int kConsumerGroups = 2;                // items go to the groups in turn
+constexpr int kConsumerThreads = kConsumerGroups * kConsumerWarps * 32;
+constexpr int kProducerWarp = kConsumerGroups * kConsumerWarps;
+constexpr int kFinisherWarp0 = kProducerWarp + 1;
+constexpr int kFinisherWarps = 3;                 // 12 warps in all: three per scheduler, 168 registers each
 constexpr int kFinisherThreads = kFinisherWarps * 32;
-constexpr int kTcThreads = kConsumerThreads + 2 * 32 + kFinisherThreads;
+constexpr int kTcThreads = kConsumerThreads + 32 + kFinisherThreads;
 constexpr int kTile = 64;
-constexpr int kKeyBlocks = kTile / 16;
 constexpr int kMaxStages = 8;
 constexpr int kMinQSlots = 4, kMaxQSlots = 8;
-// barriers: stage full / empty, query slot full / empty, warp slot ready / done, stored, counted
-constexpr int kNumBars = 2 * kMaxStages + 2 * kMaxQSlots + 2 * kConsumerWarps + 2;
+constexpr int kMergeBufs = 2;
+constexpr int kNumBars = 2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs + 2;
 
 template <int D, int NT>
 struct TcConfig {
@@ -218,10 +204,11 @@ struct TcConfig {
     static constexpr int kNewBytes = 2 * D * 2;            // the step's new K row and V row of the item's stream
     static constexpr int kQSlotBytes = kQBytes + kNewBytes;
     static constexpr int kMoStride = D + 4;
-    static constexpr int kSlotFloats = kRows * kMoStride + kRows * 2;   // a warp's partial: output rows, then (max, sum) per row
-    // warp slots, descriptor ring, stage tags, barriers, flags
-    static constexpr int kFixedBytes = kConsumerWarps * kSlotFloats * 4 + kMaxQSlots * 32 + kMaxStages * 4 +
-                                       kNumBars * 8 + 64;
+    static constexpr int kMergeFloats = kConsumerWarps * kRows * kMoStride;
+    static constexpr int kMlFloats = kConsumerWarps * kRows * 2;
+    // merge buffers (+ their item headers), descriptor ring, barriers, flags
+    static constexpr int kFixedBytes = kMergeBufs * ((kMergeFloats + kMlFloats) * 4 + 32) +
+                                       kMaxQSlots * 32 + kNumBars * 8 + 64;
     static constexpr int kAlignSlack = 1024;
     static int smem_bytes(int stages, int q_slots) {
         return stages * kStageBytes + q_slots * kQSlotBytes + kFixedBytes + kAlignSlack;
@@ -285,27 +272,6 @@ __device__ __forceinline__ void combine_stream(const float* part_o, const float*
     }
 }
 
-// Bounded wait for a stage's tag to show tile `want` (see the note on tags above).
-__device__ __forceinline__ bool tag_wait(const volatile int* tag, int want, volatile int* abort_flag,
-                                         uint32_t* status, int64_t limit_ns) {
-    if (*tag == want) return true;
-    uint64_t t0 = 0;
-    for (uint32_t i = 1;; ++i) {
-        if (*tag == want) return true;
-        if ((i & 63u) == 0u) {
-            if (*abort_flag) return false;
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (static_cast<int64_t>(now - t0) > limit_ns) {
-                *abort_flag = 1;
-                atomicOr(status, kStatusTimeout);
-                return false;
-            }
-        }
-    }
-}
-
 template <int D, int NT, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
@@ -323,10 +289,11 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* kv = smem;
     uint8_t* qbuf = kv + STAGES * Cfg::kStageBytes;
-    float* slots = reinterpret_cast<float*>(qbuf + QSLOTS * Cfg::kQSlotBytes);     // one per consumer warp
-    int* desc = reinterpret_cast<int*>(slots + kConsumerWarps * Cfg::kSlotFloats);  // 8 ints per query slot
-    volatile int* tags = desc + kMaxQSlots * 8;                                     // tile number per stage
-    uint64_t* bars = reinterpret_cast<uint64_t*>(const_cast<int*>(tags) + kMaxStages);
+    float* mrg_o = reinterpret_cast<float*>(qbuf + QSLOTS * Cfg::kQSlotBytes);
+    float* mrg_ml = mrg_o + kMergeBufs * Cfg::kMergeFloats;
+    int* mrg_hdr = reinterpret_cast<int*>(mrg_ml + kMergeBufs * Cfg::kMlFloats);   // 8 ints per buffer
+    int* desc = mrg_hdr + kMergeBufs * 8;                                           // 8 ints per slot
+    uint64_t* bars = reinterpret_cast<uint64_t*>(desc + kMaxQSlots * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars);
     volatile int* last_flag = abort_flag + 1;    // finishers: this CTA delivered a stream's last piece
 
@@ -335,9 +302,9 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kMaxStages + s); };
     auto qfull_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + s); };
     auto qempty_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + kMaxQSlots + s); };
-    auto sready_bar = [&](uint32_t w) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + w); };
-    auto sdone_bar = [&](uint32_t w) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + kConsumerWarps + w); };
-    const uint32_t fstored_bar = bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + 2 * kConsumerWarps);
+    auto mready_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + s); };
+    auto mdone_bar = [&](uint32_t s) { return bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + kMergeBufs + s); };
+    const uint32_t fstored_bar = bar0 + 8u * (2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs);
     const uint32_t fcounted_bar = fstored_bar + 8u;
 
     const int tid = threadIdx.x;
@@ -345,46 +312,30 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     const int64_t limit = p.wait_limit_ns;
     const int cta = blockIdx.x;
 
-    // An item's rows as this step sees them.  A piece that ends its stream ends where the
-    // stream ends NOW (the plan may be an earlier step's, made when the stream was a little
-    // shorter).  With the append fused in, the stream's last token is not in the slab yet: it is
-    // not streamed (a consumer warp takes it from k_new / v_new and writes it there).  `safe` =
-    // rows that no kernel still running can be writing: the previous kernel of the stream (the
-    // only one that can overlap with this one) may be this kernel one step earlier, whose new
-    // token is the stream's last row but one; the last row is this step's own.
-    struct Rows {
-        int ntok, safe;
-        bool has_new;
-    };
-    auto rows_of = [&](const int4& a, const int4& b) {
-        Rows r;
-        const bool ends = (b.x & 2) != 0;
-        const int ntok_now = (lens.n > 0 && ends) ? lens.len[a.x] - a.z : a.w;
-        r.has_new = p.k_new != nullptr && ends;
-        r.ntok = ntok_now - (r.has_new ? 1 : 0);
-        r.safe = ends ? ntok_now - 2 : ntok_now;
-        return r;
-    };
-
-    // the producer's and the finishers' first loads are in flight while the barriers are set up
+    // the producer's first loads are in flight while the barriers are being set up
     int4 rec = make_int4(0, 0, 0, 0), first_a = rec, first_b = rec;
-    if (warp >= kProducerWarp) {
+    int4 mine_a = rec, mine_b = rec;                 // producer: descriptor of item `lane` of the CTA's current 32
+    if (warp == kProducerWarp) {
         const int4* r = p.cta + 3 * cta;
         rec = __ldg(r);
         first_a = __ldg(r + 1);
         first_b = __ldg(r + 2);
-        if (warp == kProducerWarp && lane < 4)
+        if (lane < 4)
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[lane])) : "memory");
+    } else if (warp >= kFinisherWarp0 && lane == 0) {
+        rec = __ldg(p.cta + 3 * cta);
     }
     if (tid < kNumBars) {                            // one barrier per thread
+        constexpr uint32_t all_consumers = kConsumerGroups * kConsumerWarps;
         const uint32_t b = static_cast<uint32_t>(tid);
-        const uint32_t count = b < 2 * kMaxStages                                       ? 1u   // full, empty
-                               : b < 2 * kMaxStages + kMaxQSlots                        ? 1u   // query slot full
-                               : b < 2 * kMaxStages + 2 * kMaxQSlots                    ? static_cast<uint32_t>(kConsumerWarps)
-                               : b < 2 * kMaxStages + 2 * kMaxQSlots + kConsumerWarps   ? 1u   // warp slot ready
-                                                                                        : static_cast<uint32_t>(kFinisherWarps);
+        const uint32_t count = b < kMaxStages                        ? 1u               // full
+                               : b < 2 * kMaxStages                  ? all_consumers    // empty
+                               : b < 2 * kMaxStages + kMaxQSlots     ? 1u               // query slot full
+                               : b < 2 * kMaxStages + 2 * kMaxQSlots ? all_consumers    // query slot empty
+                               : b < 2 * kMaxStages + 2 * kMaxQSlots + kMergeBufs
+                                   ? static_cast<uint32_t>(kConsumerWarps)              // merge buffer ready
+                                   : static_cast<uint32_t>(kFinisherWarps);             // done / stored / counted
         mbar_init(bar0 + 8u * b, count);
-        if (tid < kMaxStages) tags[tid] = -1;
         if (tid == 0) {
             *abort_flag = 0;
             *last_flag = 0;
@@ -406,36 +357,14 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
 
-    // Item descriptors, 32 at a time, one per lane of the calling warp (producer, finishers):
-    // each lane resolves its item's rows on the spot, the values reach all lanes by shuffles.
-    int4 mine_a = make_int4(0, 0, 0, 0), mine_b = mine_a;
-    int mine_safe = 0;
-    auto fetch_items = [&](int it0, int it_end) {
-        if (it0 + lane < it_end) {
-            mine_a = __ldg(p.items + 2 * (it0 + lane));
-            mine_b = __ldg(p.items + 2 * (it0 + lane) + 1);
-            const Rows r = rows_of(mine_a, mine_b);
-            mine_a.w = r.ntok;                    // n_tokens becomes the rows to stream
-            mine_safe = r.safe;
-        }
-    };
-    auto item_of = [&](int j, int4& a, int4& b, int& safe) {     // item held by lane j, to all lanes
-        a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
-        a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
-        a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
-        a.w = __shfl_sync(0xFFFFFFFFu, mine_a.w, j);
-        b.x = __shfl_sync(0xFFFFFFFFu, mine_b.x, j);
-        b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
-        b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
-        b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
-        safe = __shfl_sync(0xFFFFFFFFu, mine_safe, j);
-    };
-
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer
-        // Streams the tiles of the CTA's items in order.  Waits are taken by the whole warp;
-        // lane 0 tags the stages and arms the barriers; a tile's copies (one per 128-byte column
-        // block of K and of V) are issued by as many lanes at once.
+        // Every lane fetches item descriptors (32 at a time, one per lane) and works out its
+        // item's rows; the values reach all lanes by shuffles.  Waits are taken by the whole
+        // warp; lane 0 arms the barriers; a tile's copies (one per 128-byte column block of K
+        // and of V) are issued by as many lanes at once, so are the copies of an item's
+        // queries and new K / V rows: the time the warp spends per copy is what bounds the
+        // rate of short items.
         const int it_begin = rec.x, it_end = rec.y;       // every lane read the record
         uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number
         bool ok = true;
@@ -443,35 +372,76 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const int64_t v_array = k_array + p.rows_per_array;
         constexpr int COPIES = 2 * HALVES;            // copies per box position: K and V, each column block
 
-        // One tile (number n of the CTA) of a slab stream = up to four groups of 16 rows,
-        // fetched with one copy per 128-byte column block of K and of V (a box of 16, 32, 48 or
-        // 64 rows; never past ceil16 of the stream's length).  part 0: the whole tile; part 1:
-        // only the groups that lie wholly in the safe rows, with the barrier told to expect the
-        // whole tile; part 2: the rest of a tile whose part 1 is under way.
-        auto arm = [&](uint32_t stage, int n, uint32_t bytes) {
-            if (lane == 0) {
-                tags[stage] = n;
-                mbar_expect_tx(full_bar(stage), bytes);
-            }
-            issued_any |= 1u << stage;
-            issued_odd ^= 1u << stage;
-            __syncwarp();
+        // An item's rows as this step sees them.  A piece that ends its stream ends where the
+        // stream ends NOW (the plan may be an earlier step's, made when the stream was a little
+        // shorter).  With the append fused in, the stream's last token is not in the slab yet:
+        // it is not streamed (a consumer warp takes it from k_new / v_new and writes it there).
+        // `safe` = rows that no kernel still running can be writing: the previous kernel of the
+        // stream (the only one that can overlap with this one) may be this kernel one step
+        // earlier, whose new token is the stream's last row but one; the last row is this
+        // step's own.
+        struct Rows {
+            int ntok, safe;
+            bool has_new;
         };
-        auto issue_slab_tile = [&](uint32_t stage, int n, int64_t row, int t, int ntok, int safe, int part) {
+        auto rows_of = [&](const int4& a, const int4& b) {
+            Rows r;
+            const bool ends = (b.x & 2) != 0;
+            const int ntok_now = (lens.n > 0 && ends) ? lens.len[a.x] - a.z : a.w;
+            r.has_new = p.k_new != nullptr && ends;
+            r.ntok = ntok_now - (r.has_new ? 1 : 0);
+            r.safe = ends ? ntok_now - 2 : ntok_now;
+            return r;
+        };
+        // One tile of a slab stream = up to four groups of 16 rows, fetched with one copy per
+        // 128-byte column block of K and of V (a box of 16, 32, 48 or 64 rows; never past
+        // ceil16 of the stream's length).  part 0: the whole tile; part 1: only the groups that
+        // lie wholly in the safe rows, with the barrier told to expect the whole tile; part 2:
+        // the rest of a tile whose part 1 is under way.  Called by the whole warp.
+        auto issue_slab_tile = [&](uint32_t stage, int64_t row, int t, int ntok, int safe, int part) {
             const int r0 = t * kTile;
             const int nb = (min(kTile, ntok - r0) + 15) >> 4;
             const int ge = min(nb, max(safe - r0, 0) >> 4);
             const int g0 = part == 2 ? ge : 0, g1 = part == 1 ? ge : nb;
-            if (part != 2) arm(stage, n, static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+            if (part != 2) {
+                if (lane == 0) mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                issued_any |= 1u << stage;
+                issued_odd ^= 1u << stage;
+                __syncwarp();
+            }
             if (g1 <= g0 || lane >= COPIES) return;
-            const int h = lane >> 1, kvsel = lane & 1;
-            const uint32_t dst = kv_u32 + stage * Cfg::kStageBytes + kvsel * Cfg::kKvTileBytes + g0 * 2048 + h * HALF_BYTES;
-            const int32_t y = static_cast<int32_t>((kvsel ? v_array : k_array) + row + r0 + g0 * 16);
+            const int h = lane >> 1, kv = lane & 1;
+            const uint32_t dst = kv_u32 + stage * Cfg::kStageBytes + kv * Cfg::kKvTileBytes + g0 * 2048 + h * HALF_BYTES;
+            const int32_t y = static_cast<int32_t>((kv ? v_array : k_array) + row + r0 + g0 * 16);
             tma_load_2d(dst, &tm.box[g1 - g0 - 1], h * 64, y, full_bar(stage));
         };
 
-        fetch_items(it_begin, it_end);                // the CTA's first 32 items (the very first came with the record)
+        // descriptors of the CTA's first 32 items (the very first came with the record), each
+        // lane's resolved on the spot: n_tokens becomes the rows to stream, the combine word's
+        // place is kept, and the safe row count travels in a register of its own
+        int mine_safe = 0;
+        auto resolve_mine = [&]() {
+            const Rows r = rows_of(mine_a, mine_b);
+            mine_a.w = r.ntok;
+            mine_safe = r.safe;
+        };
+        if (it_begin + lane < it_end) {
+            mine_a = __ldg(p.items + 2 * (it_begin + lane));
+            mine_b = __ldg(p.items + 2 * (it_begin + lane) + 1);
+            resolve_mine();
+        }
         const Rows first_r = rows_of(first_a, first_b);
+        auto item_of = [&](int j, int4& a, int4& b, int& safe) {     // item held by lane j, to all lanes
+            a.x = __shfl_sync(0xFFFFFFFFu, mine_a.x, j);
+            a.y = __shfl_sync(0xFFFFFFFFu, mine_a.y, j);
+            a.z = __shfl_sync(0xFFFFFFFFu, mine_a.z, j);
+            a.w = __shfl_sync(0xFFFFFFFFu, mine_a.w, j);
+            b.x = __shfl_sync(0xFFFFFFFFu, mine_b.x, j);
+            b.y = __shfl_sync(0xFFFFFFFFu, mine_b.y, j);
+            b.z = __shfl_sync(0xFFFFFFFFu, mine_b.z, j);
+            b.w = __shfl_sync(0xFFFFFFFFu, mine_b.w, j);
+            safe = __shfl_sync(0xFFFFFFFFu, mine_safe, j);
+        };
         // Early start: the safe rows of the CTA's first tiles (one per pipeline stage) are
         // requested before the dependency wait, so that HBM is already streaming while the
         // previous grid finishes; queries, new tokens and the rows in flux come after it.
@@ -484,80 +454,27 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if (j > 0) item_of(j, a, b, safe);
                 const int ntiles = (a.w + kTile - 1) / kTile;
                 for (int t = 0; t < ntiles && n_early < static_cast<int>(STAGES); ++t, ++n_early)
-                    issue_slab_tile(static_cast<uint32_t>(n_early), n_early, b.z, t, a.w, safe, 1);
+                    issue_slab_tile(static_cast<uint32_t>(n_early), b.z, t, a.w, safe, 1);
             }
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-        uint32_t stage = 0, phase = 0;
+        uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
         int n_tile = 0;                               // tiles issued so far (the first n_early only need their rest)
-        for (int it = it_begin; it < it_end && ok; ++it) {
-            const int j = (it - it_begin) & 31;
-            if (j == 0 && it != it_begin) fetch_items(it, it_end);
-            int4 a = first_a, b = first_b;
-            int safe = first_r.safe;
-            a.w = first_r.ntok;
-            if (it != it_begin) item_of(j, a, b, safe);
-            const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
-            const int64_t row = b.z;
-            const int ntiles = (ntok + kTile - 1) / kTile;
-            for (int t = 0; t < ntiles; ++t, ++n_tile) {
-                if (n_tile < n_early) {                  // first use of the stage, part 1 under way
-                    issue_slab_tile(stage, n_tile, row, t, ntok, safe, 2);
-                } else {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit));
-                    if (!ok) break;
-                    if (MODE != kModePaged) {
-                        issue_slab_tile(stage, n_tile, row, t, ntok, safe, 0);
-                    } else {                             // one 16-row box per page, all of them at once
-                        const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
-                        arm(stage, n_tile, static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
-                        const int bx = lane / COPIES, w = lane - bx * COPIES;
-                        if (bx < nb) {
-                            const int h = w >> 1, kvsel = w & 1;
-                            const int32_t page = p.page_table[static_cast<size_t>(req) * p.max_pages + tok0 / 16 + t * 4 + bx];
-                            const int64_t prow = (static_cast<int64_t>(page) * p.kv_heads + head) * 16;
-                            tma_load_2d(kv_u32 + stage * Cfg::kStageBytes + kvsel * Cfg::kKvTileBytes + h * HALF_BYTES + bx * 2048,
-                                        &tm.box[0], h * 64, static_cast<int32_t>((kvsel ? v_array : k_array) + prow),
-                                        full_bar(stage));
-                        }
-                    }
-                }
-                if (++stage == STAGES) {
-                    stage = 0;
-                    phase ^= 1u;
-                }
-            }
-        }
-        if (lane == 0 && !ok) {
-            // Something timed out.  Before the CTA's shared memory can be handed to another
-            // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
-            for (uint32_t s = 0; s < STAGES; ++s)
-                if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
-                    mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
-                                   limit / 4 + 1);
-        }
-        return;
-    }
-
-    if (warp == kQueryWarp) {
-        // ------------------------------------------------------------------ query warp
-        // One ring slot per item: its descriptor, the queries of its GQA group and, with the
-        // append fused in, the stream's new K and V rows behind them (one copy each, from three
-        // lanes at once).  Runs as far ahead of the consumers as the ring is deep.
-        const int it_begin = rec.x, it_end = rec.y;
-        fetch_items(it_begin, it_end);
-        const Rows first_r = rows_of(first_a, first_b);
-        uint32_t qs = 0, qphase = 0;
         for (int it = it_begin;; ++it) {
             const int j = (it - it_begin) & 31;
-            if (j == 0 && it != it_begin) fetch_items(it, it_end);
+            if (j == 0 && it != it_begin && it + lane < it_end) {
+                mine_a = __ldg(p.items + 2 * (it + lane));
+                mine_b = __ldg(p.items + 2 * (it + lane) + 1);
+                resolve_mine();
+            }
             int4 a = first_a, b = first_b;
             int safe = first_r.safe;
             a.w = first_r.ntok;
             if (it != it_begin) item_of(j, a, b, safe);
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit))) break;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(qempty_bar(qs), qphase ^ 1u, abort_flag, p.status, limit));
+            if (!ok) break;
             int* dsc = desc + qs * 8;
             if (it >= it_end) {                          // end marker
                 if (lane == 0) {
@@ -566,7 +483,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 }
                 break;
             }
-            const int req = a.x, head = a.y, ntok = a.w;
+            const int req = a.x, head = a.y, tok0 = a.z, ntok = a.w;
             const bool has_new = p.k_new != nullptr && (b.x & 2);
             const uint32_t q_bytes = static_cast<uint32_t>(p.group) * D * 2u;
             if (lane == 0) {
@@ -586,7 +503,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                           static_cast<const uint8_t*>(p.q) +
                               (static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * p.group) * D * 2,
                           q_bytes, qfull_bar(qs));
-            } else if (lane < 3 && has_new) {
+            } else if (lane < 3 && has_new) {            // the new token's K and V rows ride behind the queries
                 const size_t nrow = (static_cast<size_t>(req) * p.kv_heads + head) * D * 2;
                 const uint8_t* src = static_cast<const uint8_t*>(lane == 1 ? p.k_new : p.v_new) + nrow;
                 bulk_load(q_u32 + qs * Cfg::kQSlotBytes + Cfg::kQBytes + (lane - 1) * D * 2, src, D * 2, qfull_bar(qs));
@@ -595,18 +512,57 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 qs = 0;
                 qphase ^= 1u;
             }
+            const int64_t row = b.z;
+            const int ntiles = (ntok + kTile - 1) / kTile;
+            for (int t = 0; t < ntiles; ++t, ++n_tile) {
+                if (n_tile < n_early) {                  // first use of the stage, part 1 under way
+                    issue_slab_tile(stage, row, t, ntok, safe, 2);
+                } else {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, limit));
+                    if (!ok) break;
+                    if (MODE != kModePaged) {
+                        issue_slab_tile(stage, row, t, ntok, safe, 0);
+                    } else {                             // one 16-row box per page, all of them at once
+                        const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
+                        if (lane == 0) mbar_expect_tx(full_bar(stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                        issued_any |= 1u << stage;
+                        issued_odd ^= 1u << stage;
+                        __syncwarp();
+                        const int bx = lane / COPIES, w = lane - bx * COPIES;
+                        if (bx < nb) {
+                            const int h = w >> 1, kv = w & 1;
+                            const int32_t page = p.page_table[static_cast<size_t>(req) * p.max_pages + tok0 / 16 + t * 4 + bx];
+                            const int64_t prow = (static_cast<int64_t>(page) * p.kv_heads + head) * 16;
+                            tma_load_2d(kv_u32 + stage * Cfg::kStageBytes + kv * Cfg::kKvTileBytes + h * HALF_BYTES + bx * 2048,
+                                        &tm.box[0], h * 64, static_cast<int32_t>((kv ? v_array : k_array) + prow),
+                                        full_bar(stage));
+                        }
+                    }
+                }
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            if (!ok) break;
+        }
+        if (lane == 0 && !ok) {
+            // Something timed out.  Before the CTA's shared memory can be handed to another
+            // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
+            for (uint32_t s = 0; s < STAGES; ++s)
+                if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
+                    mbar_wait_slow(full_bar(s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status,
+                                   limit / 4 + 1);
         }
         return;
     }
 
     if (warp >= kFinisherWarp0) {
         // ------------------------------------------------------------------ finishers
-        // They walk the CTA's item list themselves (same descriptors, same tile numbering as
-        // the consumers), so they know which warps leave a partial result for each item.
         if (MODE == kModeProbe) return;
         const int ftid = tid - kFinisherWarp0 * 32;
         constexpr int fthreads = kFinisherThreads;
-        const int it_begin = rec.x, it_end = rec.y;
+        const int n_items = __shfl_sync(0xFFFFFFFFu, rec.y - rec.x, 0);
         const int group = p.group;
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
         constexpr int PER_ROW = D / 4;                   // float4 chunks per head
@@ -614,128 +570,136 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // CH = chunks of four output elements per thread; every thread computes CH chunks
         // (indices past the end are clamped, their results dropped) so the code is branch-free
         constexpr int CH = (ROWS * PER_ROW + kFinisherThreads - 1) / kFinisherThreads;
-        int rr[CH], dd[CH];
+        {
+            uint32_t n_split = 0;
+            for (int k = 0; k < n_items; ++k) {
+                const uint32_t mb = static_cast<uint32_t>(k) & 1u;
+                if (!mbar_wait(mready_bar(mb), (static_cast<uint32_t>(k) >> 1) & 1u, abort_flag, p.status, limit))
+                    return;
+                const int* hdr = mrg_hdr + mb * 8;
+                const int req = hdr[0], head = hdr[1], direct = hdr[2], slot = hdr[3], comb = hdr[4];
+                const bool count_in = !direct && p.counters != nullptr;
+                int4 cr = make_int4(0, 0, 0, 0);         // {request, head, first slot, pieces}
+                if (count_in) cr = __ldg(p.combine + comb);
+                const float* bo = mrg_o + mb * Cfg::kMergeFloats;
+                const float* bml = mrg_ml + mb * Cfg::kMlFloats;
+                float4 acc[CH];
+                float acc_m[CH], acc_l[CH];
+                int rr[CH], dd[CH];
 #pragma unroll
-        for (int i = 0; i < CH; ++i) {
-            const int idx = min(ftid + i * fthreads, total - 1);
-            rr[i] = idx / PER_ROW;
-            dd[i] = (idx - rr[i] * PER_ROW) * 4;
-        }
-        fetch_items(it_begin, it_end);
-        const Rows first_r = rows_of(first_a, first_b);
-        uint32_t n_split = 0;
-        uint32_t ready_parity = 0;                       // per warp slot: parity of its next deposit
-        int n0 = 0;                                      // number of the item's first tile
-        for (int it = it_begin; it < it_end; ++it) {
-            const int j = (it - it_begin) & 31;
-            if (j == 0 && it != it_begin) fetch_items(it, it_end);
-            int4 a = first_a, b = first_b;
-            int safe = first_r.safe;
-            a.w = first_r.ntok;
-            if (it != it_begin) item_of(j, a, b, safe);
-            const int ntiles = (a.w + kTile - 1) / kTile;
-            const int parts = ntiles == 0 ? 1 : min(ntiles, kConsumerWarps);
-            const int w0 = n0 & (kConsumerWarps - 1);
-            n0 += ntiles;
-            const int direct = b.x & 1, slot = b.y, comb = b.w;
-            if (parts == 1 && direct) continue;          // finished by its warp alone
-            const bool count_in = !direct && p.counters != nullptr;
-            int4 cr = make_int4(0, 0, 0, 0);             // {request, head, first slot, pieces}
-            if (count_in) cr = __ldg(p.combine + comb);
-            float4 acc[CH];
-            float acc_m[CH], acc_l[CH];
+                for (int i = 0; i < CH; ++i) {
+                    const int idx = min(ftid + i * fthreads, total - 1);
+                    rr[i] = idx / PER_ROW;
+                    dd[i] = (idx - rr[i] * PER_ROW) * 4;
+                }
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                acc_m[i] = -INFINITY;
-                acc_l[i] = 0.f;
-            }
-            bool ok = true;
-            for (int i = 0; i < parts && ok; ++i) {      // the warps' partial results, in tile order
-                const uint32_t w = static_cast<uint32_t>(w0 + i) & (kConsumerWarps - 1);
-                ok = mbar_wait(sready_bar(w), (ready_parity >> w) & 1u, abort_flag, p.status, limit);
-                ready_parity ^= 1u << w;
-                const float* so = slots + w * Cfg::kSlotFloats;
-                const float* sml = so + ROWS * MO;
+                for (int i = 0; i < CH; ++i) {
+                    const int r = rr[i], d0 = dd[i];
+                    float mw[kConsumerWarps], lw[kConsumerWarps], M = -INFINITY;
+                    float4 x[kConsumerWarps];
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const float2 ml = *reinterpret_cast<const float2*>(sml + rr[c] * 2);
-                    const float4 x = *reinterpret_cast<const float4*>(so + rr[c] * MO + dd[c]);
-                    lse_fold(acc_m[c], acc_l[c], acc[c], ml.x, ml.y, x);
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float2 ml = *reinterpret_cast<const float2*>(bml + (w * ROWS + r) * 2);
+                        mw[w] = ml.x;
+                        lw[w] = ml.y;
+                        x[w] = *reinterpret_cast<const float4*>(bo + (w * ROWS + r) * MO + d0);
+                        M = fmaxf(M, ml.x);
+                    }
+                    float L = 0.f;
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float e = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);   // warps without keys
+                        L = fmaf(lw[w], e, L);
+                        a.x = fmaf(x[w].x, e, a.x);
+                        a.y = fmaf(x[w].y, e, a.y);
+                        a.z = fmaf(x[w].z, e, a.z);
+                        a.w = fmaf(x[w].w, e, a.w);
+                    }
+                    acc[i] = a;
+                    acc_m[i] = M;
+                    acc_l[i] = L;
+                }
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    if (ftid + i * fthreads >= total) continue;
+                    const int r = rr[i], d0 = dd[i];
+                    if (direct) {
+                        const float inv = fast_rcp(acc_l[i]);
+                        const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
+                        store4(out + row * D + d0, acc[i].x * inv, acc[i].y * inv, acc[i].z * inv, acc[i].w * inv);
+                        if (d0 == 0 && p.lse) p.lse[row] = (acc_m[i] + fast_log2(acc_l[i])) * 0.6931471805599453f;
+                    } else {
+                        const size_t prow = static_cast<size_t>(slot) * group + r;
+                        *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = acc[i];
+                        if (d0 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(acc_m[i], acc_l[i]);
+                    }
+                }
+                {   // (the branch needs the merged sums, so the buffer reads are complete before the
+                    //  arrive below lets the group overwrite it; the sums are never negative)
+                    float seen = 0.f;
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) seen += acc_l[i];
+                    if (seen < 0.f) *(abort_flag + 2) = 1;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(sdone_bar(w));     // the warp may refill its slot
-            }
-            if (!ok) return;
-#pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                if (ftid + i * fthreads >= total) continue;
-                const int r = rr[i], d0 = dd[i];
-                if (direct) {
-                    const float inv = fast_rcp(acc_l[i]);
-                    const size_t row = static_cast<size_t>(a.x) * p.q_heads + static_cast<size_t>(a.y) * group + r;
-                    store4(out + row * D + d0, acc[i].x * inv, acc[i].y * inv, acc[i].z * inv, acc[i].w * inv);
-                    if (d0 == 0 && p.lse) p.lse[row] = (acc_m[i] + fast_log2(acc_l[i])) * 0.6931471805599453f;
-                } else {
-                    const size_t prow = static_cast<size_t>(slot) * group + r;
-                    *reinterpret_cast<float4*>(p.part_o + prow * D + d0) = acc[i];
-                    if (d0 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(acc_m[i], acc_l[i]);
+                if (lane == 0) {
+                    mbar_arrive(mdone_bar(mb));          // the buffer may be refilled
+                    if (count_in) mbar_arrive(fstored_bar);
                 }
-            }
-            if (!count_in) continue;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(fstored_bar);
-            // The CTA that delivers a split stream's last piece merges all of them.  Once
-            // every finisher thread has issued its partial stores, one thread fences them,
-            // counts this piece in and tells the rest whether the count is complete; if so
-            // each thread folds all pieces in slot order, its own from the registers it
-            // still holds, the others read back through L2.
-            if (!mbar_wait(fstored_bar, n_split & 1u, abort_flag, p.status, limit)) return;
-            if (ftid == 0) {
+                if (!count_in) continue;
+                // The CTA that delivers a split stream's last piece merges all of them.  Once
+                // every finisher thread has issued its partial stores, one thread fences them,
+                // counts this piece in and tells the rest whether the count is complete; if so
+                // each thread folds all pieces in slot order, its own from the registers it
+                // still holds, the others read back through L2.
+                if (!mbar_wait(fstored_bar, n_split & 1u, abort_flag, p.status, limit)) return;
+                if (ftid == 0) {
+                    __threadfence();
+                    const uint32_t seen = atomicAdd(p.counters + comb, 1u);
+                    const int last = seen + 1u == static_cast<uint32_t>(cr.w);
+                    if (last) p.counters[comb] = 0u;      // ready for the next launch
+                    *last_flag = last;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(fcounted_bar);
+                if (!mbar_wait(fcounted_bar, n_split & 1u, abort_flag, p.status, limit)) return;
+                ++n_split;
+                if (!*last_flag) continue;
                 __threadfence();
-                const uint32_t seen = atomicAdd(p.counters + comb, 1u);
-                const int last = seen + 1u == static_cast<uint32_t>(cr.w);
-                if (last) p.counters[comb] = 0u;      // ready for the next launch
-                *last_flag = last;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(fcounted_bar);
-            if (!mbar_wait(fcounted_bar, n_split & 1u, abort_flag, p.status, limit)) return;
-            ++n_split;
-            if (!*last_flag) continue;
-            __threadfence();
-            const size_t orow0 = static_cast<size_t>(cr.x) * p.q_heads + static_cast<size_t>(cr.y) * group;
-            float fm[CH], fl[CH];
-            float4 fa[CH];
+                const size_t orow0 = static_cast<size_t>(cr.x) * p.q_heads + static_cast<size_t>(cr.y) * group;
+                float fm[CH], fl[CH];
+                float4 fa[CH];
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                fm[i] = -INFINITY;
-                fl[i] = 0.f;
-                fa[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            for (int s = 0; s < cr.w; ++s) {
-                if (cr.z + s == slot) {               // this CTA's own piece
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], acc_m[i], acc_l[i], acc[i]);
-                    continue;
+                for (int i = 0; i < CH; ++i) {
+                    fm[i] = -INFINITY;
+                    fl[i] = 0.f;
+                    fa[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-                float2 ml[CH];
-                float4 x[CH];
+                for (int s = 0; s < cr.w; ++s) {
+                    if (cr.z + s == slot) {               // this CTA's own piece
 #pragma unroll
-                for (int i = 0; i < CH; ++i) {        // all loads of the piece first
-                    const size_t prow = static_cast<size_t>(cr.z + s) * group + rr[i];
-                    ml[i] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
-                    x[i] = ldcg4(p.part_o + prow * D + dd[i]);
+                        for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], acc_m[i], acc_l[i], acc[i]);
+                        continue;
+                    }
+                    float2 ml[CH];
+                    float4 x[CH];
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) {        // all loads of the piece first
+                        const size_t prow = static_cast<size_t>(cr.z + s) * group + rr[i];
+                        ml[i] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
+                        x[i] = ldcg4(p.part_o + prow * D + dd[i]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], ml[i].x, ml[i].y, x[i]);
                 }
 #pragma unroll
-                for (int i = 0; i < CH; ++i) lse_fold(fm[i], fl[i], fa[i], ml[i].x, ml[i].y, x[i]);
-            }
-#pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                if (ftid + i * fthreads >= total) continue;
-                const float inv = fast_rcp(fl[i]);
-                store4(out + (orow0 + rr[i]) * D + dd[i], fa[i].x * inv, fa[i].y * inv, fa[i].z * inv, fa[i].w * inv);
-                if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + fast_log2(fl[i])) * 0.6931471805599453f;
+                for (int i = 0; i < CH; ++i) {
+                    if (ftid + i * fthreads >= total) continue;
+                    const float inv = fast_rcp(fl[i]);
+                    store4(out + (orow0 + rr[i]) * D + dd[i], fa[i].x * inv, fa[i].y * inv, fa[i].z * inv, fa[i].w * inv);
+                    if (dd[i] == 0 && p.lse) p.lse[orow0 + rr[i]] = (fm[i] + fast_log2(fl[i])) * 0.6931471805599453f;
+                }
             }
         }
         return;
@@ -744,41 +708,50 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // ---------------------------------------------------------------------- consumers
     const int qd = lane >> 2, qt = lane & 3;          // row within 8, position within the quad
     const int mi = lane >> 3, r8 = lane & 7;          // ldmatrix: matrix id, row within it
-    // K block as the A operand: matrices (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15)
-    const uint32_t k_lane_off = ((mi & 1) * 8 + r8) * 128;
+    // K tile as the A operand: matrices (keys 0-7, d 0-7) (keys 8-15, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 8-15)
+    const int cw = warp & (kConsumerWarps - 1);       // warp within its group
+    const uint32_t grp = static_cast<uint32_t>(warp) / kConsumerWarps;
+    const uint32_t k_lane_off = (cw * 16 + (mi & 1) * 8 + r8) * 128;
     const uint32_t xk = (mi >> 1) ^ r8;
-    // V block, transposed on load, as the A operand: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
-    const uint32_t v_lane_off = ((mi >> 1) * 8 + r8) * 128;
+    // V tile, transposed on load, as the A operand: (keys 0-7, d 0-7) (keys 0-7, d 8-15) (keys 8-15, d 0-7) (keys 8-15, d 8-15)
+    const uint32_t v_lane_off = (cw * 16 + (mi >> 1) * 8 + r8) * 128;
     const uint32_t xv = (mi & 1) ^ r8;
     // Q as the B operand: four consecutive 16-byte chunks of head r8
     const uint32_t q_lane_off = r8 * (D * 2) + mi * 16;
+    const int key_lo = cw * 16 + qd;                // the thread's two key rows: key_lo, key_lo + 8
+    const int vkey0 = cw * 16 + qt * 2;             // keys of its value fragments: vkey0, +1, +8, +9
     const float scale = p.scale_log2;
-    float* my_o = slots + warp * Cfg::kSlotFloats;    // this warp's slot: partial output rows ...
-    float* my_ml = my_o + ROWS * MO;                  // ... and (max, sum) per row
-    const int group = p.group;
 
-    uint32_t qs = 0, qphase = 0;
-    uint32_t n_dep = 0;                               // partial results this warp has left for the finishers
-    int n0 = 0;                                       // number of the current item's first tile
+    uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
     bool ok = true;
     for (uint32_t k_item = 0; ok; ++k_item) {
         ok = mbar_wait(qfull_bar(qs), qphase, abort_flag, p.status, limit);
         if (!ok) break;
         const int* dsc = desc + qs * 8;
-        const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3];
+        const int req = dsc[0], head = dsc[1], ntok = dsc[2], direct = dsc[3], slot = dsc[4], comb = dsc[5];
         const int new_row = dsc[7];
         if (dsc[6] == 0) break;
         const int ntiles = (ntok + kTile - 1) / kTile;
-        const int t_first = (warp - n0) & (kConsumerWarps - 1);      // this warp's first tile of the item
-        const bool owns_start = t_first == 0;                        // tile 0, or the new token of an item without tiles
-        const int first_n = n0;
-        n0 += ntiles;
-        if (t_first >= ntiles && !(owns_start && new_row >= 0)) {    // nothing of this item is this warp's
+        if ((k_item & 1u) != grp) {
+            // The other group's item: let go of the slot and walk over its tiles in step with
+            // the ring.  A barrier's parity tells apart only two consecutive phases, so neither
+            // group may fall a whole phase behind or run one ahead of any stage: every warp of
+            // both groups waits for each tile to land and signs the stage off, the owners after
+            // using it, the others at once.
             __syncwarp();
             if (lane == 0) mbar_arrive(qempty_bar(qs));
             if (++qs == QSLOTS) {
                 qs = 0;
                 qphase ^= 1u;
+            }
+            for (int t = 0; t < ntiles; ++t) {
+                ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, limit);
+                if (!ok) break;
+                if (lane == 0) mbar_arrive(empty_bar(stage));
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
             }
             continue;
         }
@@ -806,18 +779,18 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             m_run[nt][0] = m_run[nt][1] = -INFINITY;
             l_run[nt][0] = l_run[nt][1] = 0.f;
         }
-        if (MODE == kModeSlab && new_row >= 0 && owns_start) {
+        if (MODE == kModeSlab && new_row >= 0 && cw == 0) {
             // The token appended this step (the piece ends its stream and the append is fused
-            // in): its K and V rows sit behind the queries in the slot.  The warp that has the
-            // item's first tile starts from it instead of from nothing: running maximum = its
-            // score, sum = 1, output = its value row; and it writes the two rows into the slab
-            // for the steps to come.  Each lane holds, of head qd, elements kk*16 + 2qt +
-            // {0, 1, 8, 9} of the query: it adds up its part of the score, the quad completes it.
+            // in): its K and V rows sit behind the queries in the slot.  The group's first warp
+            // starts from it instead of from nothing: running maximum = its score, sum = 1,
+            // output = its value row; and it writes the two rows into the slab for the steps
+            // to come.  Each lane holds, of head qd, elements kk*16 + 2qt + {0, 1, 8, 9} of the
+            // query: it adds up its part of the score, the quad completes it.
             const uint8_t* nk = qbuf + qs * Cfg::kQSlotBytes + Cfg::kQBytes;
             const uint8_t* nv = nk + D * 2;
-            float dot[NT][2];
+            float dot[NT];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) dot[nt][0] = dot[nt][1] = 0.f;
+            for (int nt = 0; nt < NT; ++nt) dot[nt] = 0.f;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t k0 = *reinterpret_cast<const uint32_t*>(nk + (kk * 16 + qt * 2) * 2);
@@ -825,21 +798,19 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const uint32_t q0 = qb[nt][kk][0], q1 = qb[nt][kk][1];
-                    float& d = dot[nt][kk & 1];
-                    d = fmaf(__uint_as_float(q0 << 16), __uint_as_float(k0 << 16), d);
-                    d = fmaf(__uint_as_float(q0 & 0xFFFF0000u), __uint_as_float(k0 & 0xFFFF0000u), d);
-                    d = fmaf(__uint_as_float(q1 << 16), __uint_as_float(k1 << 16), d);
-                    d = fmaf(__uint_as_float(q1 & 0xFFFF0000u), __uint_as_float(k1 & 0xFFFF0000u), d);
+                    dot[nt] = fmaf(__uint_as_float(q0 << 16), __uint_as_float(k0 << 16), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q0 & 0xFFFF0000u), __uint_as_float(k0 & 0xFFFF0000u), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q1 << 16), __uint_as_float(k1 << 16), dot[nt]);
+                    dot[nt] = fmaf(__uint_as_float(q1 & 0xFFFF0000u), __uint_as_float(k1 & 0xFFFF0000u), dot[nt]);
                 }
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                float d = dot[nt][0] + dot[nt][1];
-                d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-                d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
+                dot[nt] += __shfl_xor_sync(0xFFFFFFFFu, dot[nt], 1);
+                dot[nt] += __shfl_xor_sync(0xFFFFFFFFu, dot[nt], 2);
                 // the accumulator columns of this lane are heads 2qt and 2qt + 1
-                m_run[nt][0] = __shfl_sync(0xFFFFFFFFu, d, qt * 8) * scale;
-                m_run[nt][1] = __shfl_sync(0xFFFFFFFFu, d, qt * 8 + 4) * scale;
+                m_run[nt][0] = __shfl_sync(0xFFFFFFFFu, dot[nt], qt * 8) * scale;
+                m_run[nt][1] = __shfl_sync(0xFFFFFFFFu, dot[nt], qt * 8 + 4) * scale;
                 l_run[nt][0] = l_run[nt][1] = qd == 0 ? 1.f : 0.f;      // summed over qd when the item ends
 #pragma unroll
                 for (int dt = 0; dt < D / 16; ++dt) {
@@ -851,11 +822,23 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             }
             constexpr int ROW_VECS = D * 2 / 16;
             if (lane < 2 * ROW_VECS) {                   // K row, then V row, 16 bytes per lane
-                const int kvsel = lane / ROW_VECS, vec = lane - kvsel * ROW_VECS;
+                const int kv = lane / ROW_VECS, vec = lane - kv * ROW_VECS;
                 uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
-                             ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + new_row) * ROW_VECS + vec;
+                             ((static_cast<int64_t>(p.layer) * 2 + kv) * p.rows_per_array + new_row) * ROW_VECS + vec;
                 *dst = *reinterpret_cast<const uint4*>(nk + lane * 16);
             }
+        }
+        if (MODE != kModeProbe) {
+            // The slot is refilled the moment its last reader lets go of it, and ldmatrix results
+            // may still be on their way to the registers when a later arrive is performed.  A
+            // use of every fragment register (the branch needs them all) keeps the arrive behind
+            // the loads; the store never happens in practice and touches a word nobody reads.
+            uint32_t fold = 0;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) fold ^= qb[nt][kk][0] + 3u * qb[nt][kk][1];
+            if (fold == 0x9E3779B9u) *(abort_flag + 2) = 1;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(qempty_bar(qs));
@@ -864,54 +847,50 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             qphase ^= 1u;
         }
 
-        for (int t = t_first; t < ntiles; t += kConsumerWarps) {
-            const uint32_t nn = static_cast<uint32_t>(first_n + t);
-            const uint32_t round = nn / STAGES, stage = nn - round * STAGES;
-            ok = tag_wait(tags + stage, static_cast<int>(nn), abort_flag, p.status, limit) &&
-                 mbar_wait(full_bar(stage), round & 1u, abort_flag, p.status, limit);
+        for (int t = 0; t < ntiles; ++t) {
+            ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, limit);
             if (!ok) break;
             const int valid = min(kTile, ntok - t * kTile);
-            if (MODE != kModeProbe) {
+            if (MODE != kModeProbe && cw * 16 < valid) {
                 const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
                 const uint32_t vbase = kbase + Cfg::kKvTileBytes;
-                const int nkb = (valid + 15) >> 4;            // key blocks that hold keys of the item
-                // ---- S^T = K Q^T, one accumulator per block of 16 keys (independent chains)
-                float s[kKeyBlocks][NT][4];
+                // ---- S^T = K Q^T for this warp's 16 keys; two accumulators shorten the chain
+                float s[NT][4], s2[NT][4];
 #pragma unroll
-                for (int kb = 0; kb < kKeyBlocks; ++kb)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) s[kb][nt][i] = 0.f;
+                    for (int i = 0; i < 4; ++i) s[nt][i] = s2[nt][i] = 0.f;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
+                    uint32_t a[4];
+                    ldmatrix_x4(a, kbase + (kk >> 2) * HALF_BYTES + k_lane_off + ((((kk & 3) * 2) ^ xk) << 4));
 #pragma unroll
-                    for (int kb = 0; kb < kKeyBlocks; ++kb) {
-                        if (kb < nkb) {
-                            uint32_t a[4];
-                            ldmatrix_x4(a, kbase + (kk >> 2) * HALF_BYTES + kb * 2048 + k_lane_off + ((((kk & 3) * 2) ^ xk) << 4));
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt)
-                                mma_bf16(s[kb][nt], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
-                        }
+                    for (int nt = 0; nt < NT; ++nt) {
+                        if (kk & 1)
+                            mma_bf16(s2[nt], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
+                        else
+                            mma_bf16(s[nt], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
                     }
                 }
-                // ---- online softmax, fp32, over the tile's keys.  Keys at or beyond the item's
-                //      end get the score -inf (selected, never added to); a head's maximum is
-                //      shared by the eight lanes that hold its keys (shuffles over the lane bits
-                //      that select the key row).
-                uint32_t pb[kKeyBlocks][NT][2];
+                // ---- keys at or beyond the item's end: scores are selected to -inf (never
+                //      added to), value rows are zeroed in registers below
+                const bool ragged = valid < kTile;
+                const bool in_lo = key_lo < valid, in_hi = key_lo + 8 < valid;
+                uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
+                if (ragged) {
+                    vm0 = (vkey0 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 1 < valid ? 0xFFFF0000u : 0u);
+                    vm1 = (vkey0 + 8 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 9 < valid ? 0xFFFF0000u : 0u);
+                }
+                // ---- online softmax, fp32; a head's maximum is shared by the eight lanes that
+                //      hold its keys (shuffles over the lane bits that select the key row)
+                uint32_t pb[NT][2];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-                    for (int kb = 0; kb < kKeyBlocks; ++kb) {
-                        const int key = kb * 16 + qd;
-                        if (key >= valid) s[kb][nt][0] = s[kb][nt][1] = -INFINITY;
-                        if (key + 8 >= valid) s[kb][nt][2] = s[kb][nt][3] = -INFINITY;
-                        mx0 = fmaxf(mx0, fmaxf(s[kb][nt][0], s[kb][nt][2]));
-                        mx1 = fmaxf(mx1, fmaxf(s[kb][nt][1], s[kb][nt][3]));
-                    }
+                    float c0 = s[nt][0] + s2[nt][0], c1 = s[nt][1] + s2[nt][1];
+                    float c2 = s[nt][2] + s2[nt][2], c3 = s[nt][3] + s2[nt][3];
+                    if (!in_lo) c0 = c1 = -INFINITY;
+                    if (!in_hi) c2 = c3 = -INFINITY;
+                    float mx0 = fmaxf(c0, c2), mx1 = fmaxf(c1, c3);
 #pragma unroll
                     for (int off = 4; off < 32; off <<= 1) {
                         mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, off));
@@ -920,19 +899,10 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     const float mn0 = fmaxf(m_run[nt][0], mx0 * scale), mn1 = fmaxf(m_run[nt][1], mx1 * scale);
                     const float mu0 = (mn0 == -INFINITY) ? 0.f : mn0, mu1 = (mn1 == -INFINITY) ? 0.f : mn1;
                     const float corr0 = fast_exp2(m_run[nt][0] - mu0), corr1 = fast_exp2(m_run[nt][1] - mu1);
-                    float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                    for (int kb = 0; kb < kKeyBlocks; ++kb) {
-                        const float p0 = fast_exp2(fmaf(s[kb][nt][0], scale, -mu0)), p1 = fast_exp2(fmaf(s[kb][nt][1], scale, -mu1));
-                        const float p2 = fast_exp2(fmaf(s[kb][nt][2], scale, -mu0)), p3 = fast_exp2(fmaf(s[kb][nt][3], scale, -mu1));
-                        sum0 += p0 + p2;
-                        sum1 += p1 + p3;
-                        // P[key][head] -> P^T fragments: (head qd; keys 2qt, 2qt+1) and (+8, +9)
-                        pb[kb][nt][0] = movmatrix_trans(pack_bf16(p0, p1));
-                        pb[kb][nt][1] = movmatrix_trans(pack_bf16(p2, p3));
-                    }
-                    l_run[nt][0] = fmaf(l_run[nt][0], corr0, sum0);
-                    l_run[nt][1] = fmaf(l_run[nt][1], corr1, sum1);
+                    const float p0 = fast_exp2(fmaf(c0, scale, -mu0)), p1 = fast_exp2(fmaf(c1, scale, -mu1));
+                    const float p2 = fast_exp2(fmaf(c2, scale, -mu0)), p3 = fast_exp2(fmaf(c3, scale, -mu1));
+                    l_run[nt][0] = fmaf(l_run[nt][0], corr0, p0 + p2);
+                    l_run[nt][1] = fmaf(l_run[nt][1], corr1, p1 + p3);
                     m_run[nt][0] = mn0;
                     m_run[nt][1] = mn1;
 #pragma unroll
@@ -942,44 +912,37 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                         o[nt][i][2] *= corr0;
                         o[nt][i][3] *= corr1;
                     }
+                    // P[key][head] -> P^T fragments: (head qd; keys 2qt, 2qt+1) and (+8, +9)
+                    pb[nt][0] = movmatrix_trans(pack_bf16(p0, p1));
+                    pb[nt][1] = movmatrix_trans(pack_bf16(p2, p3));
                 }
-                // ---- O^T += V^T P^T; value rows at or beyond the item's end are zeroed in
-                //      registers (their weights are 0, but the rows may hold anything)
+                // ---- O^T += V^T P^T
 #pragma unroll
-                for (int kb = 0; kb < kKeyBlocks; ++kb) {
-                    if (kb < nkb) {
-                        const int vkey0 = kb * 16 + qt * 2;       // keys of the fragments: vkey0, +1, +8, +9
-                        const bool ragged = valid < kb * 16 + 16;
-                        uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
-                        if (ragged) {
-                            vm0 = (vkey0 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 1 < valid ? 0xFFFF0000u : 0u);
-                            vm1 = (vkey0 + 8 < valid ? 0x0000FFFFu : 0u) | (vkey0 + 9 < valid ? 0xFFFF0000u : 0u);
-                        }
-#pragma unroll
-                        for (int dt = 0; dt < D / 16; ++dt) {
-                            uint32_t a[4];
-                            ldmatrix_x4_trans(a, vbase + (dt >> 2) * HALF_BYTES + kb * 2048 + v_lane_off + ((((dt & 3) * 2) ^ xv) << 4));
-                            if (ragged) {
-                                a[0] &= vm0;
-                                a[1] &= vm0;
-                                a[2] &= vm1;
-                                a[3] &= vm1;
-                            }
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt)
-                                mma_bf16(o[nt][dt], a[0], a[1], a[2], a[3], pb[kb][nt][0], pb[kb][nt][1]);
-                        }
+                for (int dt = 0; dt < D / 16; ++dt) {
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, vbase + (dt >> 2) * HALF_BYTES + v_lane_off + ((((dt & 3) * 2) ^ xv) << 4));
+                    if (ragged) {
+                        a[0] &= vm0;
+                        a[1] &= vm0;
+                        a[2] &= vm1;
+                        a[3] &= vm1;
                     }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        mma_bf16(o[nt][dt], a[0], a[1], a[2], a[3], pb[nt][0], pb[nt][1]);
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar(stage));
+            if (++stage == STAGES) {
+                stage = 0;
+                phase ^= 1u;
+            }
         }
         if (!ok) break;
         if (MODE == kModeProbe) continue;
 
-        // ---- the warp's part of the item is done: through its slot to global memory (an item
-        //      of one tile that is a whole stream) or to the finishers
+        // ---- hand the warp's partial result to the finishers and move on
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -987,48 +950,41 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 l_run[nt][0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][0], off);
                 l_run[nt][1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][1], off);
             }
-        if (n_dep > 0) {                              // the finishers have read what the slot held
-            ok = mbar_wait(sdone_bar(warp), (n_dep - 1u) & 1u, abort_flag, p.status, limit);
+        const uint32_t mb = k_item & 1u;              // = grp: each group has its own buffer
+        if (k_item >= 2) {                            // the finishers are done with item k_item - 2
+            ok = mbar_wait(mdone_bar(mb), ((k_item >> 1) - 1u) & 1u, abort_flag, p.status, limit);
             if (!ok) break;
         }
+        float* mo = mrg_o + mb * Cfg::kMergeFloats + cw * ROWS * MO;
+        float* mml = mrg_ml + mb * Cfg::kMlFloats + cw * ROWS * 2;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int h0 = nt * 8 + qt * 2;
 #pragma unroll
             for (int dt = 0; dt < D / 16; ++dt) {
                 const int d = dt * 16 + qd;
-                my_o[h0 * MO + d] = o[nt][dt][0];
-                my_o[(h0 + 1) * MO + d] = o[nt][dt][1];
-                my_o[h0 * MO + d + 8] = o[nt][dt][2];
-                my_o[(h0 + 1) * MO + d + 8] = o[nt][dt][3];
+                mo[h0 * MO + d] = o[nt][dt][0];
+                mo[(h0 + 1) * MO + d] = o[nt][dt][1];
+                mo[h0 * MO + d + 8] = o[nt][dt][2];
+                mo[(h0 + 1) * MO + d + 8] = o[nt][dt][3];
             }
             if (qd == 0) {
-                my_ml[h0 * 2] = m_run[nt][0];
-                my_ml[h0 * 2 + 1] = l_run[nt][0];
-                my_ml[h0 * 2 + 2] = m_run[nt][1];
-                my_ml[h0 * 2 + 3] = l_run[nt][1];
+                mml[h0 * 2] = m_run[nt][0];
+                mml[h0 * 2 + 1] = l_run[nt][0];
+                mml[h0 * 2 + 2] = m_run[nt][1];
+                mml[h0 * 2 + 3] = l_run[nt][1];
             }
+        }
+        if (cw == 0 && lane == 0) {
+            int* hdr = mrg_hdr + mb * 8;
+            hdr[0] = req;
+            hdr[1] = head;
+            hdr[2] = direct;
+            hdr[3] = slot;
+            hdr[4] = comb;
         }
         __syncwarp();
-        if (ntiles <= 1 && direct) {
-            // alone with the whole stream: normalise and write it out, one head per pass,
-            // four output elements per lane
-            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-            constexpr int PER_ROW = D / 4;
-            for (int idx = lane; idx < group * PER_ROW; idx += 32) {
-                const int r = idx / PER_ROW, d0 = (idx - r * PER_ROW) * 4;
-                const float2 ml = *reinterpret_cast<const float2*>(my_ml + r * 2);
-                const float4 x = *reinterpret_cast<const float4*>(my_o + r * MO + d0);
-                const float inv = fast_rcp(ml.y);
-                const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + r;
-                store4(out + row * D + d0, x.x * inv, x.y * inv, x.z * inv, x.w * inv);
-                if (d0 == 0 && p.lse) p.lse[row] = (ml.x + fast_log2(ml.y)) * 0.6931471805599453f;
-            }
-            __syncwarp();                             // the slot is free again
-        } else {
-            if (lane == 0) mbar_arrive(sready_bar(warp));
-            ++n_dep;
-        }
+        if (lane == 0) mbar_arrive(mready_bar(mb));
     }
 }
 
