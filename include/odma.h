@@ -222,9 +222,13 @@ int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int
                               const odma_tables* tables, void* out, float* lse, void* stream);
 
 /* One decode step of one layer from HOST buffers: builds the tables for reqs (one new token
- * each), copies h_q [n,q_heads,head_dim], h_k_new, h_v_new [n,kv_heads,head_dim] to the
- * device, appends, attends and copies the result to h_out [n,q_heads,head_dim]; all
- * asynchronous on `stream` (pinned host memory recommended).  Does not commit lengths. */
+ * each), takes h_q [n,q_heads,head_dim], h_k_new, h_v_new [n,kv_heads,head_dim], appends,
+ * attends and leaves the result in h_out [n,q_heads,head_dim]; asynchronous on `stream`
+ * (h_out is complete once the stream has been synchronised).  When all four buffers are
+ * page-locked (cudaHostAlloc, cudaHostRegister, a framework's pinned tensors) and 16-byte
+ * aligned, the kernel reads and writes them in place over the bus: the step is one launch and
+ * no copy.  Otherwise the inputs are staged through the pool's device scratch (three
+ * host-to-device copies) and the result is copied back.  Does not commit lengths. */
 int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, const uint64_t* reqs,
                               int32_t n, const void* h_q, const void* h_k_new, const void* h_v_new,
                               void* h_out, void* stream);

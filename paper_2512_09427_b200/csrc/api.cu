@@ -262,6 +262,17 @@ int32_t plan_into(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, i
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The device-side address of a page-locked (pinned or registered) host buffer, NULL for
+// anything else (pageable host memory, device memory, managed memory).
+const void* device_alias(const void* host) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 int32_t check_tables(const odma_pool* pool, const odma_tables* t) {
     if (!t || !t->d_table || t->n < 1 || t->n_items < 1 || t->n_ctas < 1) return ODMA_ERR_INVALID;
     if (t->n_items > pool->slots_max) return ODMA_ERR_INVALID;
@@ -689,6 +700,18 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
     const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
     const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
     cudaStream_t s = as_stream(stream);
+    // Page-locked buffers are addressable from the device: the kernel then takes the queries
+    // and the new rows straight from host memory (one bulk copy per stream, issued by the
+    // producer while the KV tiles stream) and writes the result there, and the step is a single
+    // launch with no staging copy on either side.
+    {
+        const void* dq = device_alias(h_q);
+        const void* dk = device_alias(h_k_new);
+        const void* dv = device_alias(h_v_new);
+        void* dout = const_cast<void*>(device_alias(h_out));
+        if (dq && dk && dv && dout && aligned16(dq) && aligned16(dk) && aligned16(dv) && aligned16(dout))
+            return odma_decode_step(pool, layer, 1, q_heads, reqs, n, dq, dk, dv, dout, nullptr, stream, nullptr);
+    }
     if (cudaMemcpyAsync(pool->d_q, h_q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
         cudaMemcpyAsync(pool->d_k_new, h_k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
         cudaMemcpyAsync(pool->d_v_new, h_v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)

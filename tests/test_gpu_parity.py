@@ -97,6 +97,28 @@ def test_bf16_ragged_lengths_span_tiles_and_splits(ctas, fused):
     print("bf16 ragged", ctas, fused, err)
 
 
+@pytest.mark.parametrize("ctas", [1, 3])
+def test_repeated_launches_with_many_items_per_cta_are_bit_identical(ctas):
+    """52 items on one CTA (or three): the query ring wraps six times and its slots are refilled
+    the moment they are released, merge buffers and stages are reused back to back.  The kernel
+    is deterministic, so every repeat of the launch must give the bits of the first one (which is
+    checked against the checker); a slot refilled while a consumer still reads it shows up here
+    as a few rows that differ in some repeats."""
+    w = qwen_small([L - 1 for L in RAGGED])
+    s, reqs, res = run_decode(w, cfg_over={"plan_ctas": ctas})
+    check_all(s, reqs, res, f"many items per CTA, ctas={ctas}")
+    out0, lse0, q = res[0]
+    t = s.last_tables
+    assert t.n_items >= 52 and t.n_ctas == ctas
+    for rep in range(24):
+        out = torch.full_like(out0, float("nan"))
+        lse = torch.full_like(lse0, float("nan"))
+        s.pool.decode_attention(0, q.data_ptr(), w.q_heads, t, out.data_ptr(), lse.data_ptr(), s.stream)
+        torch.cuda.synchronize()
+        assert s.pool.check_status(s.stream) == 0
+        assert torch.equal(out, out0) and torch.equal(lse, lse0), f"repeat {rep} differs"
+
+
 def test_fused_and_separate_combine_agree_bit_for_bit():
     w = qwen_small([L - 1 for L in RAGGED] + [4000])
     outs = []
@@ -216,7 +238,11 @@ def test_read_probe_and_bounded_wait_selftest():
     check_all(s, reqs, res2, "after the timeout self-test")
 
 
-def test_decode_step_from_host_buffers_matches_the_device_path():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_from_host_buffers_matches_the_device_path(pinned):
+    """Page-locked buffers are read and written in place by the kernel (no copy); pageable ones
+    are staged through device scratch.  Same result either way, and the new rows are in the slab."""
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     w = qwen_small([10, 200, 64, 999])
     s = Session(w)
     s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
@@ -225,10 +251,11 @@ def test_decode_step_from_host_buffers_matches_the_device_path():
     s.append(reqs, [int(c) for c in w.context])
     for r in reqs:
         s.ls.ensure(r, s.lens[r] + 1)
-    q = s.queries(0, reqs, w.q_heads).cpu().pin_memory()
-    k_new = torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu().pin_memory()
-    v_new = torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu().pin_memory()
-    out = torch.empty_like(q).pin_memory()
+    q = pin(s.queries(0, reqs, w.q_heads).cpu())
+    k_new = pin(torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu())
+    v_new = pin(torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).cpu())
+    out = pin(torch.full_like(q, float("nan")))
+    assert q.is_pinned() == pinned and out.is_pinned() == pinned
     s.pool.decode_step_host(0, w.q_heads, reqs, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
                             out.data_ptr(), s.stream)
     torch.cuda.synchronize()
@@ -237,6 +264,9 @@ def test_decode_step_from_host_buffers_matches_the_device_path():
         s.kv.append(r, 0, k_new[i:i + 1], v_new[i:i + 1])
     ref, _, _ = s.oracle_out(0, reqs, q, w.q_heads)
     assert_close(out, ref, w.dtype, "host step")
+    s.ls.commit(reqs, 1)                              # pool_rows reads up to the committed length
+    for i, r in enumerate(reqs):                      # the step's rows sit behind each context
+        assert torch.equal(s.pool_rows(0, 0, r)[-1].cpu(), k_new[i]) and torch.equal(s.pool_rows(0, 1, r)[-1].cpu(), v_new[i])
 
 
 @pytest.mark.parametrize("fused_append", [1, 0])
