@@ -101,6 +101,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Asks for a box of a tensor to be brought into L2 (no shared memory, no barrier involved).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
+                 : "memory");
+}
+
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
                                           uint32_t bar) {
     asm volatile(
@@ -201,6 +207,7 @@ constexpr int kTile = 64;
 constexpr int kMaxStages = 8;
 constexpr int kMinQSlots = 4, kMaxQSlots = 8;
 constexpr int kMergeBufs = 2;
+constexpr int kPrefetchRounds = 1;                // tiles each consumer warp asks into L2 at the start of the kernel
 constexpr int kNumBars = 2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs + 2;
 
 template <int D, int NT>
@@ -330,8 +337,10 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         first_b = __ldg(r + 2);
         if (lane < 4)
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[lane])) : "memory");
-    } else if (warp >= kFinisherWarp0 && lane == 0) {
-        rec = __ldg(p.cta + 3 * cta);
+    } else if (warp >= kFinisherWarp0) {
+        if (lane == 0) rec = __ldg(p.cta + 3 * cta);
+    } else {
+        rec = __ldg(p.cta + 3 * cta);                // consumers: for the L2 prefetch below
     }
     if (tid < kNumBars) {                            // one barrier per thread
         constexpr uint32_t all_consumers = kConsumerGroups * kConsumerWarps;
@@ -360,6 +369,48 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     if (warp != kProducerWarp) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    if (warp < kProducerWarp && MODE != kModePaged) {
+        // While the producer requests the CTA's first tiles (one per pipeline stage) and until
+        // the queries arrive, nothing else would be asked of HBM: no stage is free before the
+        // first tile has been consumed.  The consumer warps, idle until then, ask for the tiles
+        // after those to be brought into L2 (one tile per warp and round), so HBM keeps
+        // streaming through the previous kernel's tail, the dependency wait and the queries'
+        // latency, and the producer's later copies find their rows in L2.  A prefetch writes
+        // nothing the kernel reads, so rows still being written are no concern here.
+        const int it_begin = rec.x, it_end = rec.y;
+        int4 ia = make_int4(0, 0, 0, 0), ib = ia;
+        int my_tiles = 0, my_ntok = 0;
+        if (it_begin + lane < it_end) {               // lane j: item j of the CTA
+            ia = __ldg(p.items + 2 * (it_begin + lane));
+            ib = __ldg(p.items + 2 * (it_begin + lane) + 1);
+            const bool ends = (ib.x & 2) != 0;
+            const int ntok_now = (lens.n > 0 && ends) ? lens.len[ia.x] - ia.z : ia.w;
+            my_ntok = ntok_now - ((p.k_new != nullptr && ends) ? 1 : 0);
+            my_tiles = (my_ntok + kTile - 1) / kTile;
+        }
+        int upto = my_tiles;                          // tiles of items 0..j
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int v = __shfl_up_sync(0xFFFFFFFFu, upto, off);
+            if (lane >= off) upto += v;
+        }
+        const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
+        for (int round = 0; round < kPrefetchRounds; ++round) {
+            const int tile = static_cast<int>(STAGES) + round * (kConsumerGroups * kConsumerWarps) + warp;
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, upto - my_tiles <= tile && tile < upto);
+            if (hit == 0) break;                      // beyond the CTA's first 32 items, or beyond its work
+            const int j = __ffs(hit) - 1;
+            const int t = tile - __shfl_sync(0xFFFFFFFFu, upto - my_tiles, j);
+            const int ntok = __shfl_sync(0xFFFFFFFFu, my_ntok, j);
+            const int row = __shfl_sync(0xFFFFFFFFu, ib.z, j);
+            const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
+            if (lane < 2 * HALVES) {                  // K and V, each 128-byte column block
+                const int h = lane >> 1, kvsel = lane & 1;
+                tma_prefetch_2d(&tm.box[nb - 1], h * 64,
+                                static_cast<int32_t>(k_array + kvsel * p.rows_per_array + row + t * kTile));
+            }
+        }
     }
 
     const uint32_t kv_u32 = smem_u32(kv);
