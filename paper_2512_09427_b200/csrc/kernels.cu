@@ -101,12 +101,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
-// Asks for a box of a tensor to be brought into L2 (no shared memory, no barrier involved).
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t x, int32_t y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
-                 : "memory");
-}
-
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
                                           uint32_t bar) {
     asm volatile(
@@ -169,7 +163,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Roles: warps 0..7 consume (two groups of four), warp 8 produces, warps 9.. finish.  A
 // pipeline stage holds one tile of 64 keys and 64 values of one stream, written by TMA with the
 // 128-byte swizzle so that ldmatrix reads are conflict-free.  The CTA's items go to the two
-// consumer groups in turn (short items are latency chains; two in flight hide each other).
+// consumer groups in turn (short items are latency chains; two in flight hide each other, and
+// one group's hand-over runs under the other's streaming); a stream of 16 tiles or more is
+// worked on by both groups, its tiles going to them in turn (two tiles in flight).
 // Warp w of a group owns keys [16w, 16w+16) of every tile of the group's item and keeps its own
 // running (max, sum, output): the four warps sit on the four schedulers of the SM, and an
 // mma.sync.m16n8k16 holds a scheduler's tensor pipe for some 32 cycles here, so spreading a
@@ -207,7 +203,7 @@ constexpr int kTile = 64;
 constexpr int kMaxStages = 8;
 constexpr int kMinQSlots = 4, kMaxQSlots = 8;
 constexpr int kMergeBufs = 2;
-constexpr int kPrefetchRounds = 1;                // tiles each consumer warp asks into L2 at the start of the kernel
+constexpr int kBothGroupsTiles = 16;              // streams this long are worked on by both consumer groups at once                // tiles each consumer warp asks into L2 at the start of the kernel
 constexpr int kNumBars = 2 * kMaxStages + 2 * kMaxQSlots + 2 * kMergeBufs + 2;
 
 template <int D, int NT>
@@ -337,10 +333,8 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         first_b = __ldg(r + 2);
         if (lane < 4)
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[lane])) : "memory");
-    } else if (warp >= kFinisherWarp0) {
-        if (lane == 0) rec = __ldg(p.cta + 3 * cta);
-    } else {
-        rec = __ldg(p.cta + 3 * cta);                // consumers: for the L2 prefetch below
+    } else if (warp >= kFinisherWarp0 && lane == 0) {
+        rec = __ldg(p.cta + 3 * cta);
     }
     if (tid < kNumBars) {                            // one barrier per thread
         constexpr uint32_t all_consumers = kConsumerGroups * kConsumerWarps;
@@ -370,49 +364,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
-    if (warp < kProducerWarp && MODE != kModePaged) {
-        // While the producer requests the CTA's first tiles (one per pipeline stage) and until
-        // the queries arrive, nothing else would be asked of HBM: no stage is free before the
-        // first tile has been consumed.  The consumer warps, idle until then, ask for the tiles
-        // after those to be brought into L2 (one tile per warp and round), so HBM keeps
-        // streaming through the previous kernel's tail, the dependency wait and the queries'
-        // latency, and the producer's later copies find their rows in L2.  A prefetch writes
-        // nothing the kernel reads, so rows still being written are no concern here.
-        const int it_begin = rec.x, it_end = rec.y;
-        int4 ia = make_int4(0, 0, 0, 0), ib = ia;
-        int my_tiles = 0, my_ntok = 0;
-        if (it_begin + lane < it_end) {               // lane j: item j of the CTA
-            ia = __ldg(p.items + 2 * (it_begin + lane));
-            ib = __ldg(p.items + 2 * (it_begin + lane) + 1);
-            const bool ends = (ib.x & 2) != 0;
-            const int ntok_now = (lens.n > 0 && ends) ? lens.len[ia.x] - ia.z : ia.w;
-            my_ntok = ntok_now - ((p.k_new != nullptr && ends) ? 1 : 0);
-            my_tiles = (my_ntok + kTile - 1) / kTile;
-        }
-        int upto = my_tiles;                          // tiles of items 0..j
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int v = __shfl_up_sync(0xFFFFFFFFu, upto, off);
-            if (lane >= off) upto += v;
-        }
-        const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
-        for (int round = 0; round < kPrefetchRounds; ++round) {
-            const int tile = static_cast<int>(STAGES) + round * (kConsumerGroups * kConsumerWarps) + warp;
-            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, upto - my_tiles <= tile && tile < upto);
-            if (hit == 0) break;                      // beyond the CTA's first 32 items, or beyond its work
-            const int j = __ffs(hit) - 1;
-            const int t = tile - __shfl_sync(0xFFFFFFFFu, upto - my_tiles, j);
-            const int ntok = __shfl_sync(0xFFFFFFFFu, my_ntok, j);
-            const int row = __shfl_sync(0xFFFFFFFFu, ib.z, j);
-            const int nb = (min(kTile, ntok - t * kTile) + 15) >> 4;
-            if (lane < 2 * HALVES) {                  // K and V, each 128-byte column block
-                const int h = lane >> 1, kvsel = lane & 1;
-                tma_prefetch_2d(&tm.box[nb - 1], h * 64,
-                                static_cast<int32_t>(k_array + kvsel * p.rows_per_array + row + t * kTile));
-            }
-        }
-    }
-
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
 
@@ -631,17 +582,18 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         constexpr int CH = (ROWS * PER_ROW + kFinisherThreads - 1) / kFinisherThreads;
         {
             uint32_t n_split = 0;
+            uint32_t handed = 0;                         // per merge buffer: parity of its next hand-over
             for (int k = 0; k < n_items; ++k) {
-                const uint32_t mb = static_cast<uint32_t>(k) & 1u;
-                if (!mbar_wait(mready_bar(mb), (static_cast<uint32_t>(k) >> 1) & 1u, abort_flag, p.status, limit))
-                    return;
-                const int* hdr = mrg_hdr + mb * 8;
+                // the item's start group first, then (long streams) the other one
+                const uint32_t g0 = static_cast<uint32_t>(k) & 1u;
+                if (!mbar_wait(mready_bar(g0), (handed >> g0) & 1u, abort_flag, p.status, limit)) return;
+                handed ^= 1u << g0;
+                const int* hdr = mrg_hdr + g0 * 8;
                 const int req = hdr[0], head = hdr[1], direct = hdr[2], slot = hdr[3], comb = hdr[4];
+                const int parts = hdr[5] ? 2 : 1;
                 const bool count_in = !direct && p.counters != nullptr;
                 int4 cr = make_int4(0, 0, 0, 0);         // {request, head, first slot, pieces}
                 if (count_in) cr = __ldg(p.combine + comb);
-                const float* bo = mrg_o + mb * Cfg::kMergeFloats;
-                const float* bml = mrg_ml + mb * Cfg::kMlFloats;
                 float4 acc[CH];
                 float acc_m[CH], acc_l[CH];
                 int rr[CH], dd[CH];
@@ -650,34 +602,36 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     const int idx = min(ftid + i * fthreads, total - 1);
                     rr[i] = idx / PER_ROW;
                     dd[i] = (idx - rr[i] * PER_ROW) * 4;
+                    acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    acc_m[i] = -INFINITY;
+                    acc_l[i] = 0.f;
                 }
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int r = rr[i], d0 = dd[i];
-                    float mw[kConsumerWarps], lw[kConsumerWarps], M = -INFINITY;
-                    float4 x[kConsumerWarps];
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float2 ml = *reinterpret_cast<const float2*>(bml + (w * ROWS + r) * 2);
-                        mw[w] = ml.x;
-                        lw[w] = ml.y;
-                        x[w] = *reinterpret_cast<const float4*>(bo + (w * ROWS + r) * MO + d0);
-                        M = fmaxf(M, ml.x);
+                for (int part = 0; part < parts; ++part) {
+                    const uint32_t g = g0 ^ static_cast<uint32_t>(part);
+                    if (part == 1) {
+                        if (!mbar_wait(mready_bar(g), (handed >> g) & 1u, abort_flag, p.status, limit)) return;
+                        handed ^= 1u << g;
                     }
-                    float L = 0.f;
-                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float* bo = mrg_o + g * Cfg::kMergeFloats;
+                    const float* bml = mrg_ml + g * Cfg::kMlFloats;
 #pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float e = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);   // warps without keys
-                        L = fmaf(lw[w], e, L);
-                        a.x = fmaf(x[w].x, e, a.x);
-                        a.y = fmaf(x[w].y, e, a.y);
-                        a.z = fmaf(x[w].z, e, a.z);
-                        a.w = fmaf(x[w].w, e, a.w);
+                    for (int w = 0; w < kConsumerWarps; ++w) {      // a warp without keys left max = -inf
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) {
+                            const float2 ml = *reinterpret_cast<const float2*>(bml + (w * ROWS + rr[i]) * 2);
+                            const float4 x = *reinterpret_cast<const float4*>(bo + (w * ROWS + rr[i]) * MO + dd[i]);
+                            lse_fold(acc_m[i], acc_l[i], acc[i], ml.x, ml.y, x);
+                        }
                     }
-                    acc[i] = a;
-                    acc_m[i] = M;
-                    acc_l[i] = L;
+                    {   // (the branch needs the folded sums, so the buffer reads are complete before
+                        //  the arrive below lets the group overwrite it; the sums are never negative)
+                        float seen = 0.f;
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) seen += acc_l[i];
+                        if (seen < 0.f) *(abort_flag + 2) = 1;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(mdone_bar(g));        // the buffer may be refilled
                 }
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
@@ -694,18 +648,8 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                         if (d0 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(acc_m[i], acc_l[i]);
                     }
                 }
-                {   // (the branch needs the merged sums, so the buffer reads are complete before the
-                    //  arrive below lets the group overwrite it; the sums are never negative)
-                    float seen = 0.f;
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) seen += acc_l[i];
-                    if (seen < 0.f) *(abort_flag + 2) = 1;
-                }
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(mdone_bar(mb));          // the buffer may be refilled
-                    if (count_in) mbar_arrive(fstored_bar);
-                }
+                if (lane == 0 && count_in) mbar_arrive(fstored_bar);
                 if (!count_in) continue;
                 // The CTA that delivers a split stream's last piece merges all of them.  Once
                 // every finisher thread has issued its partial stores, one thread fences them,
@@ -782,6 +726,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     const float scale = p.scale_log2;
 
     uint32_t stage = 0, phase = 0, qs = 0, qphase = 0;
+    uint32_t n_dep = 0;                               // partial results this group has left for the finishers
     bool ok = true;
     for (uint32_t k_item = 0; ok; ++k_item) {
         ok = mbar_wait(qfull_bar(qs), qphase, abort_flag, p.status, limit);
@@ -791,8 +736,14 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const int new_row = dsc[7];
         if (dsc[6] == 0) break;
         const int ntiles = (ntok + kTile - 1) / kTile;
-        if ((k_item & 1u) != grp) {
-            // The other group's item: let go of the slot and walk over its tiles in step with
+        // Items go to the two groups in turn: while one group hands an item over and starts its
+        // next one, the other is in the middle of its own.  A long stream is worked on by both
+        // groups, its tiles going to them in turn from the start group (two tiles in flight:
+        // there the hand-over is a small part, and the tile rate is what counts).
+        const bool starts = (k_item & 1u) == grp;
+        const bool both = ntiles >= kBothGroupsTiles;
+        if (!starts && !both) {
+            // Nothing of this item is this group's: let go of the slot and walk over its tiles in step with
             // the ring.  A barrier's parity tells apart only two consecutive phases, so neither
             // group may fall a whole phase behind or run one ahead of any stage: every warp of
             // both groups waits for each tile to land and signs the stage off, the owners after
@@ -838,7 +789,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             m_run[nt][0] = m_run[nt][1] = -INFINITY;
             l_run[nt][0] = l_run[nt][1] = 0.f;
         }
-        if (MODE == kModeSlab && new_row >= 0 && cw == 0) {
+        if (MODE == kModeSlab && new_row >= 0 && cw == 0 && starts) {
             // The token appended this step (the piece ends its stream and the append is fused
             // in): its K and V rows sit behind the queries in the slot.  The group's first warp
             // starts from it instead of from nothing: running maximum = its score, sum = 1,
@@ -910,7 +861,8 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, limit);
             if (!ok) break;
             const int valid = min(kTile, ntok - t * kTile);
-            if (MODE != kModeProbe && cw * 16 < valid) {
+            const bool mine = !both || ((t & 1) == 0) == starts;     // of a shared stream, even tiles are the start group's
+            if (MODE != kModeProbe && mine && cw * 16 < valid) {
                 const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
                 const uint32_t vbase = kbase + Cfg::kKvTileBytes;
                 // ---- S^T = K Q^T for this warp's 16 keys; two accumulators shorten the chain
@@ -1009,11 +961,12 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 l_run[nt][0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][0], off);
                 l_run[nt][1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[nt][1], off);
             }
-        const uint32_t mb = k_item & 1u;              // = grp: each group has its own buffer
-        if (k_item >= 2) {                            // the finishers are done with item k_item - 2
-            ok = mbar_wait(mdone_bar(mb), ((k_item >> 1) - 1u) & 1u, abort_flag, p.status, limit);
+        const uint32_t mb = grp;                      // each group has its own buffer
+        if (n_dep > 0) {                              // the finishers are done with what the group left there last
+            ok = mbar_wait(mdone_bar(mb), (n_dep - 1u) & 1u, abort_flag, p.status, limit);
             if (!ok) break;
         }
+        ++n_dep;
         float* mo = mrg_o + mb * Cfg::kMergeFloats + cw * ROWS * MO;
         float* mml = mrg_ml + mb * Cfg::kMlFloats + cw * ROWS * 2;
 #pragma unroll
@@ -1041,6 +994,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             hdr[2] = direct;
             hdr[3] = slot;
             hdr[4] = comb;
+            hdr[5] = both;                            // the other group leaves a partial result too
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(mready_bar(mb));
