@@ -49,13 +49,14 @@ TRAFFIC = {"config2": 72.79e6 + 1.44e6}
 # workload set-up through the C ABI (no checker code on this path)
 # ---------------------------------------------------------------------------------------------
 
-def pick_workload(name: str, rank: int = 0, copies_override: int = 0):
+def pick_workload(name: str, rank: int = 0, copies_override: int = 0, layers_override: int = 0):
     """Returns (workload, layers stepped per step, number of rotating KV copies).
 
     config2 is one layer; the pool is given several `layers`, each an independent copy of the
     single-layer cache, and consecutive steps rotate over them so that no step finds its KV in
     L2 (one copy is ~90 MB, L2 is 126 MB).  config3/config5 step through all their layers,
-    which together are far larger than L2."""
+    which together are far larger than L2; `layers_override` keeps only that many of them (same
+    per-layer sizes, pool shrunk in proportion) for captures that must stay small."""
     seed_off = 1000 * rank
     if name == "config2":
         base = wl.config2(seed=950902 + seed_off)
@@ -71,6 +72,9 @@ def pick_workload(name: str, rank: int = 0, copies_override: int = 0):
         copies, step_layers = 1, w.layers
     else:
         raise SystemExit(f"unknown workload {name}")
+    if layers_override and name != "config2" and layers_override < w.layers:
+        w = wl.scaled(w, layers=layers_override, pool_bytes=w.pool_bytes * layers_override // w.layers)
+        step_layers = layers_override
     return w, step_layers, copies
 
 
@@ -448,7 +452,7 @@ def run_ours(args):
 
     phases = set(args.phases.split(","))
     K, W = args.steps, args.warmup
-    w, step_layers, copies = pick_workload(args.workload, rank, args.copies)
+    w, step_layers, copies = pick_workload(args.workload, rank, args.copies, args.layers)
     sd = SlabDecode(w, step_layers, dev, fused=args.fused_combine)
     bounds, epoch = sd.learn_boundaries()
     sd.admit_and_fill()
@@ -702,6 +706,9 @@ def main():
                          "paged (page-16 ablation of the decode kernel on the same inputs)")
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="config3/config5: step through this many layers only (0 = all 28; a reduced size for profiler "
+                         "captures, not the benchmark configuration)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
