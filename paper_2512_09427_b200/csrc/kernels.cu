@@ -789,7 +789,10 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             m_run[nt][0] = m_run[nt][1] = -INFINITY;
             l_run[nt][0] = l_run[nt][1] = 0.f;
         }
-        if (MODE == kModeSlab && new_row >= 0 && cw == 0 && starts) {
+        // (which warp: the group's last one when the stream is so short that this warp has no keys
+        // of its own, 48 tokens or fewer; else the first)
+        const int new_cw = ntok <= kTile - 16 ? kConsumerWarps - 1 : 0;
+        if (MODE == kModeSlab && new_row >= 0 && cw == new_cw && starts) {
             // The token appended this step (the piece ends its stream and the append is fused
             // in): its K and V rows sit behind the queries in the slot.  The group's first warp
             // starts from it instead of from nothing: running maximum = its score, sum = 1,
