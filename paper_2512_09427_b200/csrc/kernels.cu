@@ -167,9 +167,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // one group's hand-over runs under the other's streaming); a stream of 16 tiles or more is
 // worked on by both groups, its tiles going to them in turn (two tiles in flight).
 // Warp w of a group owns keys [16w, 16w+16) of every tile of the group's item and keeps its own
-// running (max, sum, output): the four warps sit on the four schedulers of the SM, and an
-// mma.sync.m16n8k16 holds a scheduler's tensor pipe for some 32 cycles here, so spreading a
-// tile over them is what keeps a tile's latency short (0.4 us against 1.3 us for one warp).
+// running (max, sum, output): the four warps sit on the four schedulers of the SM.  A warp's
+// work on 16 keys is a chain of dependent steps (ldmatrix, mma chains of 21 cycles a link,
+// shuffles, ex2, movmatrix, mma: 770 cycles), so spreading a tile over four warps is what
+// keeps a tile's latency short (0.4 us against 1.3 us for one warp on all 64 keys).
 // When an item ends the four warps drop their partial results into the group's merge buffer
 // and go straight on to the group's next item; the finisher warps merge the four, write the
 // item's result (or partial result) to global memory and, for a split stream, count the piece
