@@ -59,8 +59,8 @@ def test_config3_full_pool_noisy_predictions_and_migrations():
 
 def test_config5_long_contexts_split_streams_and_paged_ablation():
     """Batch 32, contexts U[16384, 32768] (two of the 28 layers, the full per-layer size of
-    1.6 GB): every stream is split over several CTAs.  Sampled requests against the checker;
-    the page-16 copy (pages shuffled) must give the same bits as the slab layout."""
+    1.6 GB): every stream is split over several CTAs.  All 32 requests against the checker on
+    both layers; the page-16 copy (pages shuffled) must give the same bits as the slab layout."""
     odma = lib()
     base = wl.config5()
     w = wl.scaled(base, layers=2, pool_bytes=base.pool_bytes // 14)
@@ -72,9 +72,7 @@ def test_config5_long_contexts_split_streams_and_paged_ablation():
     res = s.decode_step(reqs, w.q_heads)
     t = s.last_tables
     assert t.n_combine >= w.batch * w.kv_heads // 2           # long streams: most are split
-    longest = int(np.argmax(w.context))
-    sample = sorted({0, 7, 31, longest})
-    check_sample(s, w, res, reqs, sample, "config5")
+    check_sample(s, w, res, reqs, reqs, "config5")
     # page-16 ablation on identical inputs
     host_len = [s.lens[r] for r in reqs]
     max_pages = max(-(-L // 16) for L in host_len)

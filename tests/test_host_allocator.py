@@ -129,3 +129,78 @@ def test_window_turnover_gives_quantiles_of_the_new_distribution():
     b, _ = pool.get_buckets()
     want = [int(-(-np.quantile(lens[-200:], q, method="inverted_cdf") // 16) * 16) for q in (0.25, 0.5, 0.75, 1.0)]
     assert list(b) == want
+
+
+@pytest.mark.parametrize("case,large_fixed", [("LF", 1), ("SP", 0)])
+def test_large_bucket_hand_computed_trace(case, large_fixed):
+    from test_oracle_allocator import _large_bucket_rows
+    odma = lib()
+    cfg = odma.config_default()
+    cfg.safety_pct, cfg.max_len, cfg.granule, cfg.large_fixed = 50, 512, 16, large_fixed
+    pool = odma.Pool(0, 2048 * 512, 1, 1, 64, odma.DTYPE_F32, cfg)
+    assert pool.set_buckets([64, 128, 256]) == 0
+    for ev, req, arg, rc, slab, mig, live, peak in _large_bucket_rows(case):
+        if ev == "alloc":
+            got, s = pool.alloc(req, arg)
+            assert got == rc and (s[:4] if got == 0 else None) == slab, (ev, req, arg, got, s)
+        elif ev == "ensure":
+            got, s, m = pool.ensure_capacity(req, arg)
+            assert got == rc and (s[:4] if got == 0 else None) == slab, (ev, req, arg, got, s)
+            if rc == 0:
+                assert m == mig
+        elif ev == "grow":
+            assert pool.commit_step([req], [arg]) == rc
+        else:
+            assert pool.free(req) == rc
+        st = pool.get_stats()
+        assert (st["safety_live"], st["safety_peak"]) == (live, peak), (ev, req, arg, st)
+
+
+def test_random_trace_lockstep_with_fixed_size_large_bucket():
+    # large_fixed = 1: every Large Bucket slab is max_len tokens, on both sides, event by event
+    w = wl.scaled(wl.config1("a"), pool_bytes=8192 * 512, safety_pct=50, window=50, refresh=7)
+    ls = LockStep(host_pool(w, large_fixed=1), oracle_allocator(w, large_fixed=1))
+    assert ls.pool.set_buckets([32, 64, 128]) == ls.oracle.set_buckets([32, 64, 128]) == 0
+    rng = np.random.default_rng(11)
+    live, nxt, large_caps = {}, 0, set()
+    for _ in range(3000):
+        op = rng.random()
+        if op < 0.45 or not live:
+            if rng.random() < 0.3:
+                rc, slab = ls.alloc_uncertain(nxt, int(rng.integers(1, 200)), int(rng.integers(0, 1001)))
+            else:
+                slab = ls.alloc(nxt, int(rng.integers(1, 300)))
+                rc = 0 if slab is not None else 2
+            if rc == 0:
+                live[nxt] = 0
+                if slab[2] == 1:
+                    large_caps.add(slab[1])
+            nxt += 1
+        elif op < 0.8:
+            r = int(rng.choice(list(live)))
+            need = live[r] + int(rng.integers(1, 60))
+            rc, slab, mig = ls.ensure_rc(r, need)
+            if rc == 0:
+                if mig:
+                    large_caps.add(slab[1])
+                ls.commit([r], need - live[r])
+                live[r] = need
+        else:
+            r = int(rng.choice(list(live)))
+            ls.free(r)
+            del live[r]
+    st = ls.check_stats()
+    assert large_caps == {w.max_len}
+    assert st["migrations"] > 5 and st["routed_large"] > 5 and st["nomem"] > 0
+
+
+@pytest.mark.slow
+def test_config4_full_drift_stream_lockstep():
+    # the whole 10,000-request stream of the drift workload, bit-exact at every event
+    w = wl.config4()
+    ls = LockStep(host_pool(w), oracle_allocator(w))
+    assert ls.pool.set_buckets(list(w.static_buckets)) == ls.oracle.set_buckets(list(w.static_buckets)) == 0
+    res = wl.run_closed_loop(ls, w.context, w.predicted, w.extra["concurrency"])
+    assert res.admitted == 10000 and len(res.boundary_log) == 10000 // w.refresh
+    st = ls.check_stats()
+    assert st["completed"] == 10000 and ls.events > 20000

@@ -254,3 +254,39 @@ def test_utilisation_formula_counts_capacity_at_completion():
     a.ensure_capacity(2, 65); a.add_len(2, 1); a.release(2)  # 65 / 128 (capacity held at completion)
     s = a.stats()
     assert (s["sum_len_completed"], s["sum_cap_completed"]) == (115, 192)
+
+
+def _large_bucket_rows(case):
+    """Rows of tests/golden/large_bucket.txt for one case: (event, req, arg, expected fields)."""
+    for row in read_golden("large_bucket.txt"):
+        if row[0] != case:
+            continue
+        row = [x for x in row if x != "|"]
+        ev, req, arg, rc = row[1], int(row[2]), int(row[3]), int(row[4])
+        slab = None if row[5] == "-" else tuple(int(x) for x in row[5:9])
+        mig = None if row[9] == "-" else int(row[9])
+        yield ev, req, arg, rc, slab, mig, int(row[10]), int(row[11])
+
+
+@pytest.mark.parametrize("case,large_fixed", [("LF", 1), ("SP", 0)])
+def test_large_bucket_hand_computed_trace(case, large_fixed):
+    # Section III-D / IV-C: Large Bucket slab sizes (one worst-case size when large_fixed),
+    # allocate-then-release order of a migration, and what safety_live / safety_peak count
+    a = ora.Allocator(2048 * 512, 1, 1, 64, 4, safety_pct=50, max_len=512, granule=16, large_fixed=large_fixed)
+    assert (a.T, a.S, a.M) == (2048, 1024, 1024)
+    assert a.set_buckets([64, 128, 256]) == ora.OK
+    for ev, req, arg, rc, slab, mig, live, peak in _large_bucket_rows(case):
+        if ev == "alloc":
+            got, s = a.reserve(req, arg)
+            assert got == rc and (s[:4] if s else None) == slab, (ev, req, arg, got, s)
+        elif ev == "ensure":
+            got, s, m = a.ensure_capacity(req, arg)
+            assert got == rc and (s[:4] if s else None) == slab, (ev, req, arg, got, s)
+            if rc == ora.OK:
+                assert m == mig
+        elif ev == "grow":
+            assert a.add_len(req, arg) == rc
+        else:
+            assert a.release(req) == rc
+        st = a.stats()
+        assert (st["safety_live"], st["safety_peak"]) == (live, peak), (ev, req, arg, st)
