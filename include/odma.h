@@ -59,6 +59,9 @@ enum {
 
 enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1 };
 
+/* which tensor-core decode kernel a bf16 pool runs (odma_config.decode_kernel) */
+enum { ODMA_DECODE_AUTO = 0, ODMA_DECODE_TCGEN05 = 1, ODMA_DECODE_MMA_SYNC = 2 };
+
 /* kernels that odma_profile_read can report */
 enum { ODMA_K_APPEND = 0, ODMA_K_DECODE = 1, ODMA_K_COMBINE = 2, ODMA_K_MIGRATE = 3,
        ODMA_K_PROBE = 4, ODMA_K_COUNT = 5 };
@@ -93,6 +96,9 @@ typedef struct odma_config {
                                 kernel take the step's new token from k_new / v_new and write
                                 it into the slab itself (one launch per layer); 0: they launch
                                 the append kernel first (1) */
+    int32_t decode_kernel;   /* bf16 decode kernel: ODMA_DECODE_AUTO picks per shape,
+                                ODMA_DECODE_TCGEN05 the tcgen05 / tensor-memory kernel,
+                                ODMA_DECODE_MMA_SYNC the mma.sync kernel (0) */
 } odma_config;
 
 typedef struct odma_slab {

@@ -345,6 +345,7 @@ void odma_config_default(odma_config* cfg) {
     cfg->plan_ctas = 0;
     cfg->fused_combine = 1;
     cfg->fused_append = 1;
+    cfg->decode_kernel = ODMA_DECODE_AUTO;
 }
 
 const char* odma_strerror(int32_t code) {
@@ -373,6 +374,7 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
     if (layers < 1 || kv_heads < 1 || head_dim < 1 || (static_cast<int64_t>(head_dim) * esz) % 16 != 0)
         return ODMA_ERR_INVALID;
     if (cfg.max_batch < 1 || cfg.max_group < 1 || cfg.plan_ctas < 0) return ODMA_ERR_INVALID;
+    if (cfg.decode_kernel < ODMA_DECODE_AUTO || cfg.decode_kernel > ODMA_DECODE_MMA_SYNC) return ODMA_ERR_INVALID;
     if (dev_base && (reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0) return ODMA_ERR_INVALID;
 
     odma_pool* p = new (std::nothrow) odma_pool();
@@ -578,6 +580,18 @@ bool uses_tc(const odma_pool* pool, int32_t q_heads) {
     return pool->has_maps && tc_supported(pool->head_dim, q_heads / pool->kv_heads);
 }
 
+// Which of the two tensor-core kernels runs a launch: the tcgen05 one unless the pool was
+// configured for mma.sync.
+bool uses_umma(const odma_pool* pool, int32_t group) {
+    return pool->alloc.config().decode_kernel != ODMA_DECODE_MMA_SYNC && umma_supported(pool->head_dim, group);
+}
+
+cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, const DecodeParams& p, int mode,
+                                 int n_ctas, cudaStream_t stream, const InlineLens* lens) {
+    return uses_umma(pool, p.group) ? launch_decode_umma(maps, p, mode, n_ctas, stream, lens)
+                                    : launch_decode_tc(maps, p, mode, n_ctas, stream, lens);
+}
+
 // odma_decode_attention; with k_new / v_new the tensor-core kernel also appends the step's
 // token (one per request) instead of finding it in the slab.
 int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
@@ -599,7 +613,7 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
             if (p.stages < 2) return ODMA_ERR_INVALID;
             fused = p.counters != nullptr;
-            e = launch_decode_tc(pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens);
+            e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens);
         } else if (generic_supported(pool->head_dim)) {
             p.counters = nullptr;
             e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
@@ -938,7 +952,7 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
     cudaError_t e;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
-        e = launch_decode_tc(paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream));
+        e = launch_tensor_decode(pool, paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream), nullptr);
     }
     if (e != cudaSuccess) return ODMA_ERR_CUDA;
     if (tables->n_combine > 0 && p.counters == nullptr) {

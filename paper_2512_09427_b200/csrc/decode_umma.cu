@@ -1,0 +1,912 @@
+// Split decode attention on the fifth-generation tensor cores (tcgen05 / tensor memory), bf16.
+//
+// Same contract as decode_tc_kernel (kernels.cu): persistent CTAs walk the items of the
+// host-built plan; an item is a run of tokens of one (request, KV head) stream; K and V tiles
+// of 64 tokens arrive by TMA in the 128-byte-swizzled layout.  Here the two products of a tile
+// are issued as tcgen05.mma instructions that read K, V, Q and P straight from shared memory
+// and accumulate in tensor memory:
+//     S[heads x 64 keys] = Q[heads x D]   . K[64 keys x D]^T      A, B K-major
+//     O[heads x D]      += P[heads x 64]  . V[64 keys x D]        A K-major, B MN-major
+// The GQA group's query heads are the first rows of an M = 64 operand.  A row of the result
+// depends on that row of A only, so the other rows of the A descriptors (whatever shared memory
+// follows the real rows) cost nothing but tensor throughput, of which this path uses little.
+// With M = 64, rows 0..15 of an accumulator live in lanes 0..15 of tensor memory, which warps
+// 0 and 4 of a CTA can read.
+//
+// Two items are in flight per CTA ("lanes": items go to them in turn), each with its own
+// softmax warp, two S buffers and one O accumulator in tensor memory and two P buffers in
+// shared memory, so one item's hand-over runs under the other's streaming.  Warp roles:
+//     0, 4   softmax + finish of lane 0 / 1: S from tensor memory (one thread holds 16 keys of
+//            one head), masking, running reference maximum, P = 2^(s - m) to shared memory; on
+//            an item's last tile the value rows between the item's end and the next multiple of
+//            16 are zeroed (the second product runs over whole groups of 16 keys); when the item
+//            ends, O from tensor memory, normalise, write out (or leave a partial result and,
+//            for the last piece of a split stream, merge all pieces).  With the append fused in,
+//            the step's new token never enters the tensor-core path: its score is a dot product
+//            on the plain ALUs and its value row is added when the item ends.
+//     2      MMA issue (one thread, both lanes): S(t+1) is issued before P(t).V(t), so the
+//            softmax of the next tile overlaps the second product of this one; tcgen05.commit
+//            releases pipeline stages, query slots and buffers
+//     1      producer: TMA loads of K/V tiles into the stage ring
+//     3      query loader: the group's query rows, global -> swizzled shared memory; the step's
+//            new K/V rows to a side buffer and into the slab
+//
+// A parity wait can tell apart only the current phase of a barrier and the one before, so every
+// barrier here is waited on, phase after phase, by ONE role that sees each of its phases: the
+// stage ring by the MMA thread (which therefore issues the first products in ring order), the
+// per-lane barriers by that lane's softmax warp or by the MMA thread, a query slot (slot = item
+// number mod 8, so a slot always serves the same lane) by the MMA thread and that lane's softmax
+// warp.  The MMA thread never blocks on one barrier: it polls what it could issue next (the
+// next tile's first product, each lane's oldest second product).  Roles that need ring
+// positions (which stage a tile sits in) count tiles over the CTA's whole item list.
+//
+// The softmax keeps a reference m per head that is the maximum seen when the item started and
+// is raised only when a tile's maximum exceeds it by more than 2^8: P stays below 256, which
+// bf16 and the fp32 accumulator hold without loss, and the accumulator in tensor memory is
+// rescaled (read, multiplied, written back) only on that rare path.  (m, l, O) with such a
+// reference is a valid partial result for the log-sum-exp merge.
+#include <algorithm>
+
+#include "device_utils.cuh"
+#include "odma.h"
+
+namespace odma {
+namespace {
+
+using namespace dev;
+
+constexpr int kTile = 64;
+constexpr int kUmmaWarps = 5;
+constexpr int kUmmaThreads = kUmmaWarps * 32;
+constexpr int kMaxStages = 8;
+constexpr int kQSlots = 8;
+constexpr int kLanes = 2;
+constexpr float kRescaleAbove = 8.f;      // log2 units a tile's maximum may pass the reference by
+
+// barrier indices
+constexpr int kBarFull = 0, kBarEmpty = kMaxStages;
+constexpr int kBarQFull = 2 * kMaxStages, kBarQEmpty = kBarQFull + kQSlots;
+constexpr int kBarLane0 = kBarQEmpty + kQSlots;
+constexpr int kBarPerLane = 10;           // s_full[2] s_empty[2] p_full[2] p_empty[2] o_full o_empty
+constexpr int kBarDrain = kBarLane0 + kLanes * kBarPerLane;
+constexpr int kNumBars = kBarDrain + 1;
+
+constexpr int kTmemCols = 512;            // all of it: one CTA per SM
+constexpr int kTmemLaneCols = 256;        // per lane: S0 at +0, S1 at +64, O at +128
+
+template <int D, int NT>
+struct UmmaConfig {
+    static constexpr int kHalves = D / 64;                 // 128-byte column blocks per row
+    static constexpr int kKvTileBytes = kTile * D * 2;
+    static constexpr int kStageBytes = 2 * kKvTileBytes;
+    static constexpr int kQHalfBytes = NT * 1024;          // 8 NT rows of 128 bytes
+    static constexpr int kQSlotBytes = kHalves * kQHalfBytes;
+    static constexpr int kPBufBytes = NT * 1024;           // 8 NT rows of 64 keys
+    static constexpr int kPBytes = kLanes * 2 * kPBufBytes;
+    static constexpr int kQBytes = kQSlots * kQSlotBytes;
+    static constexpr int kNewBytes = 2 * D * 2;            // the step's new K row and V row of an item's stream
+    static constexpr int kNewBufBytes = ((kQSlots * kNewBytes + 1023) / 1024) * 1024;
+    static constexpr int kTailBytes = kNumBars * 8 + 64;
+    static constexpr int kAlignSlack = 1024;
+    static int smem_bytes(int stages) {
+        return kNewBufBytes + kPBytes + kQBytes + stages * kStageBytes + kTailBytes + kAlignSlack;
+    }
+};
+
+// ---- tcgen05 wrappers -------------------------------------------------------------------------
+
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride byte
+// offsets in 16-byte units, descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, A K-major.
+__host__ __device__ constexpr uint32_t umma_idesc(int m, int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) |
+           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
+        "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
+// The barrier receives one arrival once every tcgen05.mma this thread has issued is complete.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 16 lanes x 64 columns of 32 bits: lane t of the warp receives, in register 4i + j, row
+// t/4 + 8 (j/2), column 8i + 2 (t%4) + (j%2) (the accumulator layout of m16n8 tiles, repeated
+// along the columns).
+__device__ __forceinline__ void tmem_ld_x8(uint32_t addr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr)
+        : "memory");
+}
+// 16 lanes x 32 columns
+__device__ __forceinline__ void tmem_ld_x4(uint32_t addr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(addr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_x4(uint32_t addr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(addr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ---- items ------------------------------------------------------------------------------------
+
+// What an item of the plan means in this step.  A piece that ends its stream ends where the
+// stream ends NOW (the plan may be an earlier step's, made when the stream was a little
+// shorter).  With the append fused in, the stream's last token is not in the slab yet: it is
+// not streamed; the softmax warp takes it from k_new / v_new.
+struct Item {
+    int req, head, tok0;
+    int n_slab;       // rows streamed from the slab
+    int tiles;        // ceil(n_slab / 64); 0 when the item is nothing but the new token
+    int safe;         // rows of the piece that no kernel still running can be writing
+    int row0;         // first row of the piece inside one K (or V) array of the pool
+    int direct, slot, comb;
+    bool has_new;
+};
+
+__device__ __forceinline__ Item item_of(const int4& a, const int4& b, const InlineLens& lens, bool fused) {
+    Item it;
+    const bool ends = (b.x & 2) != 0;
+    it.req = a.x;
+    it.head = a.y;
+    it.tok0 = a.z;
+    const int n_keys = (lens.n > 0 && ends) ? lens.len[a.x] - a.z : a.w;
+    it.has_new = fused && ends;
+    it.n_slab = n_keys - (it.has_new ? 1 : 0);
+    it.tiles = (it.n_slab + kTile - 1) / kTile;
+    // the previous kernel of the stream (the only one that can overlap with this one) may be
+    // this kernel one step earlier, whose new token is the stream's last row but one
+    it.safe = ends ? n_keys - 2 : n_keys;
+    it.row0 = b.z;
+    it.direct = b.x & 1;
+    it.slot = b.y;
+    it.comb = b.w;
+    return it;
+}
+
+template <int D, int NT, int MODE>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
+                   const __grid_constant__ InlineLens lens) {
+    using Cfg = UmmaConfig<D, NT>;
+    constexpr int HALVES = Cfg::kHalves;
+    constexpr int HALF_BYTES = kTile * 128;           // one 128-byte column block of a K or V tile
+    constexpr int ROW_CHUNKS = D * 2 / 16;            // 16-byte chunks per row
+    constexpr int QK_STEPS = D / 16;                  // K = 16 per instruction
+    const uint32_t STAGES = static_cast<uint32_t>(p.stages);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // New-row buffers, P buffers and query slots come first: an M = 64 descriptor reads 8 KB
+    // from its base, and what follows the last of them is the stage ring.
+    uint8_t* newbuf = smem;
+    uint8_t* pbuf = newbuf + Cfg::kNewBufBytes;
+    uint8_t* qbuf = pbuf + Cfg::kPBytes;
+    uint8_t* kv = qbuf + Cfg::kQBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(kv + STAGES * Cfg::kStageBytes);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(abort_flag) + 1);
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar = [&](int idx) { return bar0 + 8u * static_cast<uint32_t>(idx); };
+    auto lane_bar = [&](int L, int idx) { return bar0 + 8u * static_cast<uint32_t>(kBarLane0 + L * kBarPerLane + idx); };
+    enum { S_FULL = 0, S_EMPTY = 2, P_FULL = 4, P_EMPTY = 6, O_FULL = 8, O_EMPTY = 9 };
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int64_t limit = p.wait_limit_ns;
+    const int cta = blockIdx.x;
+    const bool fused = p.k_new != nullptr;
+
+    // a query slot is handed back by two parties: the MMA thread and the lane's softmax warp
+    if (tid < kNumBars) mbar_init(bar(tid), (tid >= kBarQEmpty && tid < kBarQEmpty + kQSlots) ? 2u : 1u);
+    if (tid == 0) {
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows of the query slots beyond the group stay zero for the whole kernel
+    for (int i = tid; i < Cfg::kQBytes / 16; i += kUmmaThreads)
+        reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(static_cast<uint32_t>(kTmemCols))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    const int4 rec = __ldg(p.cta + 3 * cta);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const int it_begin = rec.x, it_end = rec.y;
+    const uint32_t kv_u32 = smem_u32(kv);
+    const uint32_t q_u32 = smem_u32(qbuf);
+    const uint32_t p_u32 = smem_u32(pbuf);
+
+    // Programmatic dependent launch: all of the above may run while the previous kernel of the
+    // stream drains, and so may the producer's first loads of rows nobody can be writing; the
+    // rest comes after the dependency wait.  The next kernel is let go only after this wait, so
+    // a kernel can overlap with its immediate predecessor only.
+    if (warp != 1) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+
+    // item walk shared by the roles: descriptor of item `it`, the next one already on its way
+    int4 nxt_a = make_int4(0, 0, 0, 0), nxt_b = nxt_a;
+    auto fetch = [&](int it) {
+        if (it < it_end) {
+            nxt_a = __ldg(p.items + 2 * it);
+            nxt_b = __ldg(p.items + 2 * it + 1);
+        }
+    };
+
+    bool ok = true;
+    if (warp == 1) {
+        // ------------------------------------------------------------------ producer
+        uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number of times
+        const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
+        const int64_t v_array = k_array + p.rows_per_array;
+        constexpr int COPIES = 2 * HALVES;            // copies per box position: K and V, each column block
+        // One tile of a slab stream = up to four groups of 16 rows, fetched with one copy per
+        // 128-byte column block of K and of V (a box of 16, 32, 48 or 64 rows; never past
+        // ceil16 of the rows to stream).  part 0: the whole tile; part 1: only the groups that
+        // lie wholly in the safe rows, with the barrier told to expect the whole tile; part 2:
+        // the rest of a tile whose part 1 is under way.  Called by the whole warp.
+        auto issue_tile = [&](uint32_t stage, const Item& im, int t, int part) {
+            const int r0 = t * kTile;
+            const int nb = (min(kTile, im.n_slab - r0) + 15) >> 4;
+            const int ge = min(nb, max(im.safe - r0, 0) >> 4);
+            const int g0 = part == 2 ? ge : 0, g1 = part == 1 ? ge : nb;
+            if (part != 2) {
+                if (lane == 0) mbar_expect_tx(bar(kBarFull + stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                issued_any |= 1u << stage;
+                issued_odd ^= 1u << stage;
+                __syncwarp();
+            }
+            if (MODE == kModePaged) {                 // one 16-row box per page, all of them at once
+                const int bx = lane / COPIES, w = lane - bx * COPIES;
+                if (bx < nb) {
+                    const int h = w >> 1, kvsel = w & 1;
+                    const int32_t page = p.page_table[static_cast<size_t>(im.req) * p.max_pages + im.tok0 / 16 + t * 4 + bx];
+                    const int64_t prow = (static_cast<int64_t>(page) * p.kv_heads + im.head) * 16;
+                    tma_load_2d(kv_u32 + stage * Cfg::kStageBytes + kvsel * Cfg::kKvTileBytes + h * HALF_BYTES + bx * 2048,
+                                &tm.box[0], h * 64, static_cast<int32_t>((kvsel ? v_array : k_array) + prow),
+                                bar(kBarFull + stage));
+                }
+                return;
+            }
+            if (g1 <= g0 || lane >= COPIES) return;
+            const int h = lane >> 1, kvsel = lane & 1;
+            const uint32_t dst = kv_u32 + stage * Cfg::kStageBytes + kvsel * Cfg::kKvTileBytes + g0 * 2048 + h * HALF_BYTES;
+            const int32_t y = static_cast<int32_t>((kvsel ? v_array : k_array) + im.row0 + r0 + g0 * 16);
+            tma_load_2d(dst, &tm.box[g1 - g0 - 1], h * 64, y, bar(kBarFull + stage));
+        };
+        if (lane < 4)
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm.box[lane])) : "memory");
+        // Early start: the safe rows of the CTA's first tiles (one per pipeline stage) are
+        // requested before the dependency wait, so that HBM is already streaming while the
+        // previous grid finishes.
+        int n_early = 0;
+        if (MODE != kModePaged) {
+            const int4* r = p.cta + 3 * cta;
+            int4 a = __ldg(r + 1), b = __ldg(r + 2);
+            for (int it = it_begin; it < it_end && n_early < static_cast<int>(STAGES); ++it) {
+                if (it != it_begin) {
+                    a = __ldg(p.items + 2 * it);
+                    b = __ldg(p.items + 2 * it + 1);
+                }
+                const Item im = item_of(a, b, lens, fused);
+                for (int t = 0; t < im.tiles && n_early < static_cast<int>(STAGES); ++t, ++n_early)
+                    issue_tile(static_cast<uint32_t>(n_early), im, t, 1);
+            }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+        uint32_t g = 0;                               // tiles issued so far
+        fetch(it_begin);
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const Item im = item_of(nxt_a, nxt_b, lens, fused);
+            fetch(it + 1);
+            for (int t = 0; t < im.tiles; ++t, ++g) {
+                const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
+                if (g < static_cast<uint32_t>(n_early)) {        // first use of the stage, part 1 under way
+                    issue_tile(stage, im, t, 2);
+                    continue;
+                }
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarEmpty + stage), phase ^ 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                issue_tile(stage, im, t, 0);
+            }
+        }
+        if (lane == 0 && (!ok || *abort_flag)) {
+            // Something timed out.  Before the CTA's shared memory can be handed to another
+            // CTA, wait (bounded, ignoring the abort flag) for the loads already in flight.
+            for (uint32_t s = 0; s < STAGES; ++s)
+                if ((issued_any >> s) & 1u)      // parity of the stage's latest phase
+                    mbar_wait_slow(bar(kBarFull + s), ((issued_odd >> s) & 1u) ^ 1u, nullptr, p.status, limit / 4 + 1);
+        }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ query loader
+        // chunk c (16 bytes) of head r of the group goes to row r of column block c / 8, at the
+        // swizzled position (c % 8) ^ (r % 8) of that row; the new K and V rows go, as they
+        // are, to the slot's side buffer and to the slab
+        const uint8_t* qg = static_cast<const uint8_t*>(p.q);
+        constexpr int Q_LOADS = (NT * 8 * ROW_CHUNKS + 31) / 32;
+        fetch(it_begin);
+        for (int it = it_begin; it < it_end; ++it) {
+            const int k = it - it_begin;
+            const Item im = item_of(nxt_a, nxt_b, lens, fused);
+            fetch(it + 1);
+            const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
+            const uint8_t* src = qg + (static_cast<size_t>(im.req) * p.q_heads + static_cast<size_t>(im.head) * p.group) * D * 2;
+            uint4 v[Q_LOADS];
+#pragma unroll
+            for (int i = 0; i < Q_LOADS; ++i) {
+                const int idx = lane + 32 * i;
+                if (idx < p.group * ROW_CHUNKS) v[i] = __ldg(reinterpret_cast<const uint4*>(src) + idx);
+            }
+            uint4 nv = make_uint4(0u, 0u, 0u, 0u);
+            const bool mine = im.has_new && lane < 2 * ROW_CHUNKS;
+            const int kvsel = lane / ROW_CHUNKS, c_new = lane - kvsel * ROW_CHUNKS;
+            if (mine) {
+                const size_t nrow = (static_cast<size_t>(im.req) * p.kv_heads + im.head) * ROW_CHUNKS;
+                nv = __ldg(reinterpret_cast<const uint4*>(kvsel ? p.v_new : p.k_new) + nrow + c_new);
+            }
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQEmpty + slot), (use & 1u) ^ 1u, abort_flag, p.status, limit));
+            if (!ok) break;
+            uint8_t* dst = qbuf + slot * Cfg::kQSlotBytes;
+#pragma unroll
+            for (int i = 0; i < Q_LOADS; ++i) {
+                const int idx = lane + 32 * i;
+                if (idx < p.group * ROW_CHUNKS) {
+                    const int r = idx / ROW_CHUNKS, c = idx - r * ROW_CHUNKS;
+                    *reinterpret_cast<uint4*>(dst + (c >> 3) * Cfg::kQHalfBytes + (r >> 3) * 1024 + (r & 7) * 128 +
+                                              (((c & 7) ^ (r & 7)) << 4)) = v[i];
+                }
+            }
+            if (mine) {
+                *reinterpret_cast<uint4*>(newbuf + slot * Cfg::kNewBytes + lane * 16) = nv;
+                uint4* slab = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
+                              ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
+                *slab = nv;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQFull + slot));
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ MMA issue
+        // One thread polls what can be issued next: the first product of the next tile in ring
+        // order (its stage has landed, its lane's S buffer is free, for an item's first tile its
+        // queries are there) and each lane's oldest pending second product (its P is written,
+        // for an item's first tile the lane's O has been read out).
+        if (lane == 0) {
+            constexpr uint32_t IDESC_QK = umma_idesc(64, kTile, false);
+            constexpr uint32_t IDESC_PV = umma_idesc(64, D, true);
+            uint32_t qk_c[kLanes] = {0, 0}, pv_c[kLanes] = {0, 0};   // tiles of the lane issued so far, per product
+            uint32_t n_items[kLanes] = {0, 0};                      // items of the lane whose first tile has been issued
+            uint32_t info[kLanes][2] = {{0, 0}, {0, 0}};             // pending second products: stage | ksteps << 4 | first << 8 | last << 9 | item parity << 10
+            uint32_t g = 0;
+            int it = it_begin, t = 0;
+            Item im{};
+            bool have = false;                        // `im` is item `it`, with tiles left from t
+            auto advance = [&]() {                    // next item with tiles; items without arrive on their slot at once
+                have = false;
+                while (it < it_end) {
+                    im = item_of(nxt_a, nxt_b, lens, fused);
+                    fetch(it + 1);
+                    if (im.tiles > 0) {
+                        have = true;
+                        t = 0;
+                        return;
+                    }
+                    // an item that is nothing but the step's new token: no product to issue; its
+                    // slot is signed off once it has been filled (not before: the slot's previous
+                    // use must be over)
+                    const uint32_t kk = static_cast<uint32_t>(it - it_begin);
+                    if (!mbar_wait(bar(kBarQFull + kk % kQSlots), (kk / kQSlots) & 1u, abort_flag, p.status, limit)) return;
+                    mbar_arrive(bar(kBarQEmpty + kk % kQSlots));
+                    ++it;
+                }
+            };
+            fetch(it_begin);
+            advance();
+            uint64_t t0 = 0;
+            uint32_t spins = 0;
+            while (have || pv_c[0] < qk_c[0] || pv_c[1] < qk_c[1]) {
+                bool did = false;
+#pragma unroll
+                for (int L = 0; L < kLanes; ++L) {
+                    if (pv_c[L] == qk_c[L]) continue;
+                    const uint32_t cc = pv_c[L], b = cc & 1u, u = cc >> 1, inf = b ? info[L][1] : info[L][0];
+                    const bool first = (inf >> 8) & 1u, last = (inf >> 9) & 1u;
+                    if (!mbar_try(lane_bar(L, P_FULL + b), u & 1u)) continue;
+                    if (first && !mbar_try(lane_bar(L, O_EMPTY), ((inf >> 10) & 1u) ^ 1u)) continue;
+                    tc_fence_after();
+                    const uint32_t st = inf & 15u, ksteps = (inf >> 4) & 15u;
+                    const uint32_t vbase = kv_u32 + st * Cfg::kStageBytes + Cfg::kKvTileBytes;
+                    const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + b) * Cfg::kPBufBytes);
+                    const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
+                    for (uint32_t ks = 0; ks < ksteps; ++ks)
+                        umma_bf16(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * 2048, HALF_BYTES, 1024),
+                                  IDESC_PV, (first && ks == 0) ? 0u : 1u);
+                    umma_commit(bar(kBarEmpty + st));
+                    umma_commit(lane_bar(L, P_EMPTY + b));
+                    if (last) umma_commit(lane_bar(L, O_FULL));
+                    ++pv_c[L];
+                    did = true;
+                }
+#pragma unroll
+                for (int L = 0; L < kLanes; ++L) {
+                    const int k = it - it_begin;
+                    if (!have || (k & 1) != L) continue;
+                    const uint32_t cc = qk_c[L], b = cc & 1u, u = cc >> 1;
+                    const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
+                    const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
+                    if (cc - pv_c[L] >= 2u || (t == 0 && !mbar_try(bar(kBarQFull + slot), use & 1u)) ||
+                        !mbar_try(bar(kBarFull + stage), phase) || !mbar_try(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u))
+                        continue;
+                    tc_fence_after();
+                    const uint32_t qb = q_u32 + slot * Cfg::kQSlotBytes;
+                    const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
+                    const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + b * 64u;
+#pragma unroll
+                    for (int ks = 0; ks < QK_STEPS; ++ks)
+                        umma_bf16(t_s, smem_desc(qb + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
+                                  smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+                    umma_commit(lane_bar(L, S_FULL + b));
+                    const bool last = t == im.tiles - 1;
+                    if (last) umma_commit(bar(kBarQEmpty + slot));
+                    const uint32_t ksteps = last ? static_cast<uint32_t>((im.n_slab - t * kTile + 15) >> 4) : 4u;
+                    const uint32_t inf = stage | (ksteps << 4) | ((t == 0 ? 1u : 0u) << 8) | ((last ? 1u : 0u) << 9) |
+                                         ((n_items[L] & 1u) << 10);
+                    if (b) info[L][1] = inf; else info[L][0] = inf;
+                    if (t == 0) ++n_items[L];
+                    ++qk_c[L];
+                    ++g;
+                    if (last) {
+                        ++it;
+                        advance();
+                    } else {
+                        ++t;
+                    }
+                    did = true;
+                }
+                if (did) {
+                    spins = 0;
+                    t0 = 0;
+                } else if ((++spins & 255u) == 0u) {
+                    if (*abort_flag) break;
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) {
+                        t0 = now;
+                    } else if (static_cast<int64_t>(now - t0) > limit) {
+                        *abort_flag = 1;
+                        atomicOr(p.status, kStatusTimeout);
+                        break;
+                    }
+                }
+            }
+            // nothing may still be running when tensor memory is given back
+            umma_commit(bar(kBarDrain));
+        }
+        __syncwarp();
+        mbar_wait_slow(bar(kBarDrain), 0, nullptr, p.status, limit / 4 + 1);
+    } else if (warp == 0 || warp == 4) {
+        // ------------------------------------------------------------------ softmax + finish
+        const int L = warp == 0 ? 0 : 1;
+        const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols), t_o = t_s + 128u;
+        uint8_t* p_lane = pbuf + L * 2 * Cfg::kPBufBytes;
+        const int hq = lane >> 2, kq = (lane & 3) * 2;      // head row within 8; first of the thread's two keys within 8
+        const float scale = p.scale_log2;
+        const int group = p.group;
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+        uint32_t c = 0, j = 0, g = 0;                       // the lane's tiles and items so far; ring position
+        fetch(it_begin);
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const int k = it - it_begin;
+            const Item im = item_of(nxt_a, nxt_b, lens, fused);
+            fetch(it + 1);
+            const uint32_t g0 = g;
+            g += static_cast<uint32_t>(im.tiles);
+            if ((k & 1) != L) continue;
+            const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
+            if (!ok) break;
+            // The token appended this step: its scaled score per head from the query rows and the
+            // new K row in shared memory (each thread adds up the elements it will also hold of the
+            // output, the quad completes the sum); its value row, packed, for when the item ends.
+            float s_new[NT];
+            uint32_t v_new[D / 8];
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) s_new[rs] = -INFINITY;
+            if (im.has_new) {
+                const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes;
+                const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
+                const uint8_t* nvp = nk + D * 2;
+                float dot[NT];
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) dot[rs] = 0.f;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) {
+                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(nk + (8 * i + kq) * 2);
+                    v_new[i] = *reinterpret_cast<const uint32_t*>(nvp + (8 * i + kq) * 2);
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) {
+                        const uint32_t qq = *reinterpret_cast<const uint32_t*>(
+                            qs + (i >> 3) * Cfg::kQHalfBytes + rs * 1024 + hq * 128 + (((i & 7) ^ hq) << 4) + kq * 2);
+                        dot[rs] = fmaf(__uint_as_float(qq << 16), __uint_as_float(kk << 16), dot[rs]);
+                        dot[rs] = fmaf(__uint_as_float(qq & 0xFFFF0000u), __uint_as_float(kk & 0xFFFF0000u), dot[rs]);
+                    }
+                }
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 1);
+                    dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 2);
+                    s_new[rs] = dot[rs] * scale;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
+
+            float m_ref[NT], l_acc[NT];
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                m_ref[rs] = s_new[rs];
+                l_acc[rs] = 0.f;
+            }
+            for (int t = 0; t < im.tiles; ++t) {
+                const uint32_t b = c & 1u, u = c >> 1;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t r[32];
+                tmem_ld_x8(t_s + b * 64u, r);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, S_EMPTY + b));
+                const int valid = min(kTile, im.n_slab - t * kTile);
+                // scaled scores, keys at or beyond the item's end selected to -inf; tile maximum per head
+                float sc[NT][16], mx[NT];
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    mx[rs] = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float s = __uint_as_float(r[4 * i + 2 * rs + e]) * scale;
+                            if (8 * i + kq + e >= valid) s = -INFINITY;
+                            sc[rs][2 * i + e] = s;
+                            mx[rs] = fmaxf(mx[rs], s);
+                        }
+                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 1));
+                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 2));
+                }
+                if (t == 0) {
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) m_ref[rs] = fmaxf(m_ref[rs], mx[rs]);
+                } else {
+                    bool grow = false;
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) grow = grow || mx[rs] > m_ref[rs] + kRescaleAbove;
+                    if (__any_sync(0xFFFFFFFFu, grow)) {
+                        // Rare: raise the reference of the heads that need it and rescale their
+                        // rows of the accumulator.  Every second product issued so far must be
+                        // complete (the previous tile's releases its P buffer when it is); none
+                        // can be issued before this tile's P is handed over.
+                        const uint32_t pc = c - 1u;
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + (pc & 1u)), (pc >> 1) & 1u, abort_flag,
+                                                              p.status, limit));
+                        if (!ok) break;
+                        tc_fence_after();
+                        float f[2] = {1.f, 1.f};
+#pragma unroll
+                        for (int rs = 0; rs < NT; ++rs) {
+                            const float mn = mx[rs] > m_ref[rs] + kRescaleAbove ? mx[rs] : m_ref[rs];
+                            f[rs] = fast_exp2(m_ref[rs] - mn);
+                            l_acc[rs] *= f[rs];
+                            m_ref[rs] = mn;
+                        }
+#pragma unroll
+                        for (int blk = 0; blk < D / 32; ++blk) {
+                            uint32_t o[16];
+                            tmem_ld_x4(t_o + blk * 32u, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * f[0]);
+                                o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * f[0]);
+                                o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * f[1]);
+                                o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * f[1]);
+                            }
+                            tmem_st_x4(t_o + blk * 32u, o);
+                        }
+                        tmem_wait_st();
+                        tc_fence_before();
+                    }
+                }
+                // P = 2^(s - m) as bf16, 64 keys per head row, in the K-major swizzled layout; the row sums stay fp32
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                uint8_t* pb = p_lane + b * Cfg::kPBufBytes;
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float p0 = fast_exp2(sc[rs][2 * i] - m_ref[rs]), p1 = fast_exp2(sc[rs][2 * i + 1] - m_ref[rs]);
+                        sum += p0 + p1;
+                        *reinterpret_cast<uint32_t*>(pb + rs * 1024 + hq * 128 + ((i ^ hq) << 4) + kq * 2) = pack_bf16(p0, p1);
+                    }
+                    l_acc[rs] += sum;
+                }
+                if (valid & 15) {
+                    // the second product takes whole groups of 16 keys: value rows between the item's
+                    // end and the end of its last group are zeroed (P is zero there; the rows hold
+                    // whatever the slab does, which may not be a finite number)
+                    uint8_t* vt = kv + ((g0 + static_cast<uint32_t>(t)) % STAGES) * Cfg::kStageBytes + Cfg::kKvTileBytes;
+                    const int zero_rows = 16 - (valid & 15);
+                    for (int idx = lane; idx < zero_rows * ROW_CHUNKS; idx += 32) {
+                        const int zr = valid + idx / ROW_CHUNKS, cc = idx % ROW_CHUNKS;
+                        *reinterpret_cast<uint4*>(vt + (cc >> 3) * HALF_BYTES + zr * 128 + (((cc & 7) ^ (zr & 7)) << 4)) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, P_FULL + b));
+                ++c;
+            }
+            if (!ok) break;
+
+            // ---- the item's result: O from tensor memory, then out / partial / merge
+            float oo[NT][D / 4];                          // [rs][2i + e]: head hq + 8 rs, element 8i + kq + e
+            if (im.tiles > 0) {
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int blk = 0; blk < D / 64; ++blk) {
+                    uint32_t r[32];
+                    tmem_ld_x8(t_o + blk * 64u, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int rs = 0; rs < NT; ++rs) {
+                            oo[rs][2 * (8 * blk + i)] = __uint_as_float(r[4 * i + 2 * rs]);
+                            oo[rs][2 * (8 * blk + i) + 1] = __uint_as_float(r[4 * i + 2 * rs + 1]);
+                        }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, O_EMPTY));
+                ++j;
+            } else {
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs)
+#pragma unroll
+                    for (int i = 0; i < D / 4; ++i) oo[rs][i] = 0.f;
+            }
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                l_acc[rs] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[rs], 1);
+                l_acc[rs] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[rs], 2);
+            }
+            if (im.has_new) {
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    const float pn = fast_exp2(s_new[rs] - m_ref[rs]);
+                    l_acc[rs] += pn;
+#pragma unroll
+                    for (int i = 0; i < D / 8; ++i) {
+                        oo[rs][2 * i] = fmaf(pn, __uint_as_float(v_new[i] << 16), oo[rs][2 * i]);
+                        oo[rs][2 * i + 1] = fmaf(pn, __uint_as_float(v_new[i] & 0xFFFF0000u), oo[rs][2 * i + 1]);
+                    }
+                }
+            }
+            auto write_out = [&](int req, int head, int rs, float M, float Lsum, const float (&x)[D / 4]) {
+                const int h = hq + 8 * rs;
+                if (h >= group) return;
+                const float inv = fast_rcp(Lsum);
+                const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + h;
+                __nv_bfloat16* dst = out + row * D + kq;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i)
+                    *reinterpret_cast<uint32_t*>(dst + 8 * i) = pack_bf16(x[2 * i] * inv, x[2 * i + 1] * inv);
+                if ((lane & 3) == 0 && p.lse) p.lse[row] = (M + fast_log2(Lsum)) * 0.6931471805599453f;
+            };
+            if (im.direct) {
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) write_out(im.req, im.head, rs, m_ref[rs], l_acc[rs], oo[rs]);
+                continue;
+            }
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                const int h = hq + 8 * rs;
+                if (h >= group) continue;
+                const size_t prow = static_cast<size_t>(im.slot) * group + h;
+                float* po = p.part_o + prow * D + kq;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) *reinterpret_cast<float2*>(po + 8 * i) = make_float2(oo[rs][2 * i], oo[rs][2 * i + 1]);
+                if ((lane & 3) == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref[rs], l_acc[rs]);
+            }
+            if (p.counters == nullptr) continue;           // a combine kernel follows
+            // The CTA that delivers a split stream's last piece merges all of them, in slot
+            // order (so the result does not depend on which CTA that is): its own piece from the
+            // registers it still holds, the others read back through L2.
+            const int4 cr = __ldg(p.combine + im.comb);   // {request, head, first slot, pieces}
+            __syncwarp();
+            int is_last = 0;
+            if (lane == 0) {
+                __threadfence();
+                const uint32_t seen = atomicAdd(p.counters + im.comb, 1u);
+                is_last = seen + 1u == static_cast<uint32_t>(cr.w);
+                if (is_last) p.counters[im.comb] = 0u;     // ready for the next launch
+            }
+            is_last = __shfl_sync(0xFFFFFFFFu, is_last, 0);
+            if (!is_last) continue;
+            __threadfence();
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                const int h = hq + 8 * rs;
+                if (h >= group) continue;
+                float fm = -INFINITY, fl = 0.f, fa[D / 4];
+#pragma unroll
+                for (int i = 0; i < D / 4; ++i) fa[i] = 0.f;
+                for (int s = 0; s < cr.w; ++s) {
+                    float m, l, x[D / 4];
+                    if (cr.z + s == im.slot) {
+                        m = m_ref[rs];
+                        l = l_acc[rs];
+#pragma unroll
+                        for (int i = 0; i < D / 4; ++i) x[i] = oo[rs][i];
+                    } else {
+                        const size_t prow = static_cast<size_t>(cr.z + s) * group + h;
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
+                        m = ml.x;
+                        l = ml.y;
+                        const float* po = p.part_o + prow * D + kq;
+#pragma unroll
+                        for (int i = 0; i < D / 8; ++i) {
+                            const float2 v = __ldcg(reinterpret_cast<const float2*>(po + 8 * i));
+                            x[2 * i] = v.x;
+                            x[2 * i + 1] = v.y;
+                        }
+                    }
+                    const float mn = fmaxf(fm, m);
+                    const float e0 = fm == -INFINITY ? 0.f : fast_exp2(fm - mn);
+                    const float e1 = m == -INFINITY ? 0.f : fast_exp2(m - mn);
+                    fl = fmaf(fl, e0, l * e1);
+#pragma unroll
+                    for (int i = 0; i < D / 4; ++i) fa[i] = fmaf(fa[i], e0, x[i] * e1);
+                    fm = mn;
+                }
+                write_out(cr.x, cr.y, rs, fm, fl, fa);
+            }
+        }
+    }
+
+    // ---- tear-down: every role comes here, on every path, and tensor memory is given back
+    if (!ok) *abort_flag = 1;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(static_cast<uint32_t>(kTmemCols))
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// launch
+// ---------------------------------------------------------------------------------------------
+
+constexpr int kSmemPerCtaMax = 232448;    // most dynamic shared memory one CTA may ask for
+constexpr int kMaxDevices = 64;
+
+template <int D, int NT>
+int umma_stages() {
+    using Cfg = UmmaConfig<D, NT>;
+    const int n = (kSmemPerCtaMax - Cfg::smem_bytes(0)) / Cfg::kStageBytes;
+    return std::min(n, kMaxStages);
+}
+
+template <int D, int NT, int MODE>
+cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas, cudaStream_t stream,
+                             const InlineLens& lens) {
+    using Cfg = UmmaConfig<D, NT>;
+    static bool configured[kMaxDevices] = {false};     // the opt-in to large shared memory is per device
+    auto kern = decode_umma_kernel<D, NT, MODE>;
+    p.stages = umma_stages<D, NT>();
+    if (p.stages < 2) return cudaErrorInvalidValue;
+    const int smem = Cfg::smem_bytes(p.stages);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas));
+    cfg.blockDim = dim3(kUmmaThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, maps, p, lens);
+}
+
+template <int D, int NT>
+cudaError_t launch_umma_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s,
+                             const InlineLens& lens) {
+    switch (mode) {
+        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab>(maps, p, n_ctas, s, lens);
+        case kModePaged: return launch_umma_inst<D, NT, kModePaged>(maps, p, n_ctas, s, lens);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+bool umma_supported(int32_t head_dim, int32_t group) {
+    return (head_dim == 64 || head_dim == 128) && group >= 1 && group <= 16;
+}
+
+cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
+                               cudaStream_t stream, const InlineLens* lens_in) {
+    static const InlineLens no_lens{};                 // n = 0: lengths as planned
+    const InlineLens& lens = lens_in ? *lens_in : no_lens;
+    const bool two = p.group > 8;
+    if (p.head_dim == 128)
+        return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens)
+                   : launch_umma_mode<128, 1>(maps, p, mode, n_ctas, stream, lens);
+    if (p.head_dim == 64)
+        return two ? launch_umma_mode<64, 2>(maps, p, mode, n_ctas, stream, lens)
+                   : launch_umma_mode<64, 1>(maps, p, mode, n_ctas, stream, lens);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace odma

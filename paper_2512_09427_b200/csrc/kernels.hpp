@@ -64,6 +64,11 @@ bool tc_supported(int32_t head_dim, int32_t group);
 void tc_shape(int32_t head_dim, int32_t group, int32_t* stages, int32_t* q_slots);
 cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
                              cudaStream_t stream, const InlineLens* lens = nullptr);
+// The same decode step on the tcgen05 tensor cores (decode_umma.cu): slab and paged modes;
+// `stages` and `q_slots` of the parameter block are ignored (the kernel sizes its own rings).
+bool umma_supported(int32_t head_dim, int32_t group);
+cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
+                               cudaStream_t stream, const InlineLens* lens = nullptr);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
 bool generic_supported(int32_t head_dim);
 
