@@ -24,21 +24,22 @@
 //            for the last piece of a split stream, merge all pieces).  With the append fused in,
 //            the step's new token never enters the tensor-core path: its score is a dot product
 //            on the plain ALUs and its value row is added when the item ends.
-//     2      MMA issue (one thread, both lanes): S(t+1) is issued before P(t).V(t), so the
-//            softmax of the next tile overlaps the second product of this one; tcgen05.commit
-//            releases pipeline stages, query slots and buffers
+//     2      MMA issue of the first products, both lanes, in ring order (one elected lane of the
+//            converged warp); S(t+1) is issued as soon as S(t-1) has been read out, so the
+//            softmax of the next tile overlaps the second product of this one
+//     5, 6   MMA issue of the second products of lane 0 / 1; tcgen05.commit releases pipeline
+//            stages, query slots and buffers
 //     1      producer: TMA loads of K/V tiles into the stage ring
 //     3      query loader: the group's query rows, global -> swizzled shared memory; the step's
 //            new K/V rows to a side buffer and into the slab
 //
 // A parity wait can tell apart only the current phase of a barrier and the one before, so every
 // barrier here is waited on, phase after phase, by ONE role that sees each of its phases: the
-// stage ring by the MMA thread (which therefore issues the first products in ring order), the
-// per-lane barriers by that lane's softmax warp or by the MMA thread, a query slot (slot = item
-// number mod 8, so a slot always serves the same lane) by the MMA thread and that lane's softmax
-// warp.  The MMA thread never blocks on one barrier: it polls what it could issue next (the
-// next tile's first product, each lane's oldest second product).  Roles that need ring
-// positions (which stage a tile sits in) count tiles over the CTA's whole item list.
+// stage ring by warp 2 (which therefore issues the first products in ring order), the per-lane
+// barriers by that lane's softmax warp, by warp 2 or by the lane's second-product warp, a query
+// slot (slot = item number mod 8, so a slot always serves the same lane) by warp 2 and that
+// lane's softmax warp.  Roles that need ring positions (which stage a tile sits in) count tiles
+// over the CTA's whole item list.
 //
 // The softmax keeps a reference m per head that is the maximum seen when the item started and
 // is raised only when a tile's maximum exceeds it by more than 2^8: P stays below 256, which
@@ -56,7 +57,7 @@ namespace {
 using namespace dev;
 
 constexpr int kTile = 64;
-constexpr int kUmmaWarps = 5;
+constexpr int kUmmaWarps = 7;
 constexpr int kUmmaThreads = kUmmaWarps * 32;
 constexpr int kMaxStages = 8;
 constexpr int kQSlots = 8;
@@ -69,7 +70,7 @@ constexpr int kBarQFull = 2 * kMaxStages, kBarQEmpty = kBarQFull + kQSlots;
 constexpr int kBarLane0 = kBarQEmpty + kQSlots;
 constexpr int kBarPerLane = 10;           // s_full[2] s_empty[2] p_full[2] p_empty[2] o_full o_empty
 constexpr int kBarDrain = kBarLane0 + kLanes * kBarPerLane;
-constexpr int kNumBars = kBarDrain + 1;
+constexpr int kNumBars = kBarDrain + 3;
 
 constexpr int kTmemCols = 512;            // all of it: one CTA per SM
 constexpr int kTmemLaneCols = 256;        // per lane: S0 at +0, S1 at +64, O at +128
@@ -409,123 +410,102 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             if (lane == 0) mbar_arrive(bar(kBarQFull + slot));
         }
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ MMA issue
-        // One thread polls what can be issued next: the first product of the next tile in ring
-        // order (its stage has landed, its lane's S buffer is free, for an item's first tile its
-        // queries are there) and each lane's oldest pending second product (its P is written,
-        // for an item's first tile the lane's O has been read out).
-        if (lane == 0) {
-            constexpr uint32_t IDESC_QK = umma_idesc(64, kTile, false);
-            constexpr uint32_t IDESC_PV = umma_idesc(64, D, true);
-            uint32_t qk_c[kLanes] = {0, 0}, pv_c[kLanes] = {0, 0};   // tiles of the lane issued so far, per product
-            uint32_t n_items[kLanes] = {0, 0};                      // items of the lane whose first tile has been issued
-            uint32_t info[kLanes][2] = {{0, 0}, {0, 0}};             // pending second products: stage | ksteps << 4 | first << 8 | last << 9 | item parity << 10
-            uint32_t g = 0;
-            int it = it_begin, t = 0;
-            Item im{};
-            bool have = false;                        // `im` is item `it`, with tiles left from t
-            auto advance = [&]() {                    // next item with tiles; items without arrive on their slot at once
-                have = false;
-                while (it < it_end) {
-                    im = item_of(nxt_a, nxt_b, lens, fused);
-                    fetch(it + 1);
-                    if (im.tiles > 0) {
-                        have = true;
-                        t = 0;
-                        return;
-                    }
-                    // an item that is nothing but the step's new token: no product to issue; its
-                    // slot is signed off once it has been filled (not before: the slot's previous
-                    // use must be over)
-                    const uint32_t kk = static_cast<uint32_t>(it - it_begin);
-                    if (!mbar_wait(bar(kBarQFull + kk % kQSlots), (kk / kQSlots) & 1u, abort_flag, p.status, limit)) return;
-                    mbar_arrive(bar(kBarQEmpty + kk % kQSlots));
-                    ++it;
-                }
-            };
-            fetch(it_begin);
-            advance();
-            uint64_t t0 = 0;
-            uint32_t spins = 0;
-            while (have || pv_c[0] < qk_c[0] || pv_c[1] < qk_c[1]) {
-                bool did = false;
-#pragma unroll
-                for (int L = 0; L < kLanes; ++L) {
-                    if (pv_c[L] == qk_c[L]) continue;
-                    const uint32_t cc = pv_c[L], b = cc & 1u, u = cc >> 1, inf = b ? info[L][1] : info[L][0];
-                    const bool first = (inf >> 8) & 1u, last = (inf >> 9) & 1u;
-                    if (!mbar_try(lane_bar(L, P_FULL + b), u & 1u)) continue;
-                    if (first && !mbar_try(lane_bar(L, O_EMPTY), ((inf >> 10) & 1u) ^ 1u)) continue;
-                    tc_fence_after();
-                    const uint32_t st = inf & 15u, ksteps = (inf >> 4) & 15u;
-                    const uint32_t vbase = kv_u32 + st * Cfg::kStageBytes + Cfg::kKvTileBytes;
-                    const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + b) * Cfg::kPBufBytes);
-                    const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
-                    for (uint32_t ks = 0; ks < ksteps; ++ks)
-                        umma_bf16(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * 2048, HALF_BYTES, 1024),
-                                  IDESC_PV, (first && ks == 0) ? 0u : 1u);
-                    umma_commit(bar(kBarEmpty + st));
-                    umma_commit(lane_bar(L, P_EMPTY + b));
-                    if (last) umma_commit(lane_bar(L, O_FULL));
-                    ++pv_c[L];
-                    did = true;
-                }
-#pragma unroll
-                for (int L = 0; L < kLanes; ++L) {
-                    const int k = it - it_begin;
-                    if (!have || (k & 1) != L) continue;
-                    const uint32_t cc = qk_c[L], b = cc & 1u, u = cc >> 1;
-                    const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
-                    const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
-                    if (cc - pv_c[L] >= 2u || (t == 0 && !mbar_try(bar(kBarQFull + slot), use & 1u)) ||
-                        !mbar_try(bar(kBarFull + stage), phase) || !mbar_try(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u))
-                        continue;
-                    tc_fence_after();
-                    const uint32_t qb = q_u32 + slot * Cfg::kQSlotBytes;
-                    const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
-                    const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + b * 64u;
+        // ------------------------------------------------------------------ MMA issue, first products
+        // In ring order: a tile's stage has landed, its lane's S buffer has been read out, and for
+        // an item's first tile its queries are there.  The whole warp runs the loop and one
+        // elected lane issues: tcgen05 instructions issued from a converged warp cost a third of
+        // what they cost a lone thread of a diverged one.
+        uint32_t elected;
+        asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(elected));
+        constexpr uint32_t IDESC_QK = umma_idesc(64, kTile, false);
+        uint32_t c[kLanes] = {0, 0};                  // tiles of each lane issued so far
+        uint32_t g = 0;
+        fetch(it_begin);
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const int k = it - it_begin, L = k & 1;
+            const Item im = item_of(nxt_a, nxt_b, lens, fused);
+            fetch(it + 1);
+            const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
+            if (!ok) break;
+            if (im.tiles == 0) {
+                // nothing but the step's new token: no product; the slot is signed off (after it was
+                // filled, not before: its previous use must be over)
+                if (elected) mbar_arrive(bar(kBarQEmpty + slot));
+                continue;
+            }
+            const uint32_t qb = q_u32 + slot * Cfg::kQSlotBytes;
+            for (int t = 0; t < im.tiles; ++t, ++g) {
+                const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
+                const uint32_t cc = L ? c[1] : c[0], b = cc & 1u, u = cc >> 1;
+                bool good = mbar_wait(bar(kBarFull + stage), phase, abort_flag, p.status, limit);
+                if (good) good = mbar_wait(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit);
+                ok = __all_sync(0xFFFFFFFFu, good);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
+                const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + b * 64u;
+                if (elected) {
 #pragma unroll
                     for (int ks = 0; ks < QK_STEPS; ++ks)
                         umma_bf16(t_s, smem_desc(qb + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
                                   smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
                     umma_commit(lane_bar(L, S_FULL + b));
-                    const bool last = t == im.tiles - 1;
-                    if (last) umma_commit(bar(kBarQEmpty + slot));
-                    const uint32_t ksteps = last ? static_cast<uint32_t>((im.n_slab - t * kTile + 15) >> 4) : 4u;
-                    const uint32_t inf = stage | (ksteps << 4) | ((t == 0 ? 1u : 0u) << 8) | ((last ? 1u : 0u) << 9) |
-                                         ((n_items[L] & 1u) << 10);
-                    if (b) info[L][1] = inf; else info[L][0] = inf;
-                    if (t == 0) ++n_items[L];
-                    ++qk_c[L];
-                    ++g;
-                    if (last) {
-                        ++it;
-                        advance();
-                    } else {
-                        ++t;
-                    }
-                    did = true;
+                    if (t == im.tiles - 1) umma_commit(bar(kBarQEmpty + slot));
                 }
-                if (did) {
-                    spins = 0;
-                    t0 = 0;
-                } else if ((++spins & 255u) == 0u) {
-                    if (*abort_flag) break;
-                    const uint64_t now = global_timer_ns();
-                    if (t0 == 0) {
-                        t0 = now;
-                    } else if (static_cast<int64_t>(now - t0) > limit) {
-                        *abort_flag = 1;
-                        atomicOr(p.status, kStatusTimeout);
-                        break;
-                    }
-                }
+                __syncwarp();
+                if (L) ++c[1]; else ++c[0];
             }
-            // nothing may still be running when tensor memory is given back
-            umma_commit(bar(kBarDrain));
         }
+        // nothing may still be running when tensor memory is given back
+        if (elected) umma_commit(bar(kBarDrain));
         __syncwarp();
         mbar_wait_slow(bar(kBarDrain), 0, nullptr, p.status, limit / 4 + 1);
+    } else if (warp == 5 || warp == 6) {
+        // ------------------------------------------------------------------ MMA issue, second products of one lane
+        // A tile's P has been written (and, for an item's first tile, the lane's O of the item
+        // before has been read out); the commits hand the stage back to the producer and the P
+        // buffer to the softmax warp, and after an item's last tile tell it that O is complete.
+        const int L = warp - 5;
+        uint32_t elected;
+        asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(elected));
+        constexpr uint32_t IDESC_PV = umma_idesc(64, D, true);
+        const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
+        uint32_t c = 0, j = 0, g = 0;                 // the lane's tiles and items (with tiles) so far; ring position
+        fetch(it_begin);
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const int k = it - it_begin;
+            const Item im = item_of(nxt_a, nxt_b, lens, fused);
+            fetch(it + 1);
+            const uint32_t g0 = g;
+            g += static_cast<uint32_t>(im.tiles);
+            if ((k & 1) != L || im.tiles == 0) continue;
+            for (int t = 0; t < im.tiles; ++t, ++c) {
+                const uint32_t b = c & 1u, u = c >> 1, st = (g0 + static_cast<uint32_t>(t)) % STAGES;
+                bool good = mbar_wait(lane_bar(L, P_FULL + b), u & 1u, abort_flag, p.status, limit);
+                if (good && t == 0) good = mbar_wait(lane_bar(L, O_EMPTY), (j & 1u) ^ 1u, abort_flag, p.status, limit);
+                ok = __all_sync(0xFFFFFFFFu, good);
+                if (!ok) break;
+                tc_fence_after();
+                const bool last = t == im.tiles - 1;
+                const int ksteps = last ? (im.n_slab - t * kTile + 15) >> 4 : 4;
+                const uint32_t vbase = kv_u32 + st * Cfg::kStageBytes + Cfg::kKvTileBytes;
+                const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + static_cast<int>(b)) * Cfg::kPBufBytes);
+                if (elected) {
+                    for (int ks = 0; ks < ksteps; ++ks)
+                        umma_bf16(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * 2048, HALF_BYTES, 1024), IDESC_PV,
+                                  (t == 0 && ks == 0) ? 0u : 1u);
+                    umma_commit(bar(kBarEmpty + st));
+                    umma_commit(lane_bar(L, P_EMPTY + b));
+                    if (last) umma_commit(lane_bar(L, O_FULL));
+                }
+                __syncwarp();
+            }
+            ++j;
+        }
+        if (elected) umma_commit(bar(kBarDrain + 1 + L));
+        __syncwarp();
+        mbar_wait_slow(bar(kBarDrain + 1 + L), 0, nullptr, p.status, limit / 4 + 1);
     } else if (warp == 0 || warp == 4) {
         // ------------------------------------------------------------------ softmax + finish
         const int L = warp == 0 ? 0 : 1;

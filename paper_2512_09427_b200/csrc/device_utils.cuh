@@ -45,6 +45,20 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
+// Non-blocking form for polling loops (try_wait may suspend the thread for a while when the
+// phase is not complete; test_wait returns at once).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
 // Every wait of the kernels is bounded: when `limit_ns` passes without the barrier completing,
 // the waiter raises the CTA's abort flag and the timeout bit of the status word and gives up;
 // every other waiter of the CTA sees the flag and gives up too.
