@@ -42,6 +42,11 @@ struct odma_pool {
     int64_t rows_per_array = 0;
     int32_t plan_ctas = 148;
     uint32_t* d_counters = nullptr;   // per split stream: pieces delivered (fused combine)
+    // a second scratch set: consecutive layers of one step alternate between the two, so that a
+    // layer's kernel need not wait for the previous layer's
+    float* part_o2 = nullptr;
+    float* part_ml2 = nullptr;
+    uint32_t* d_counters2 = nullptr;
     int64_t slots_max = 0;
     int64_t table_words_max = 0;
     bool has_maps = false;
@@ -152,6 +157,9 @@ void free_device_side(odma_pool* p) {
     cudaFree(p->part_ml);
     cudaFree(p->d_status);
     cudaFree(p->d_counters);
+    cudaFree(p->part_o2);
+    cudaFree(p->part_ml2);
+    cudaFree(p->d_counters2);
     cudaFree(p->d_q);
     cudaFree(p->d_k_new);
     cudaFree(p->d_v_new);
@@ -309,6 +317,7 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->page_table = nullptr;
     p->max_pages = 0;
     p->wait_limit_ns = kDefaultWaitLimitNs;
+    p->chained = 0;
 }
 
 int32_t check_decode_args(const odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
@@ -414,6 +423,9 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
         const size_t qb = static_cast<size_t>(cfg.max_batch) * kv_heads * cfg.max_group * head_dim * esz;
         const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * esz;
         bool ok = cudaMalloc(&p->part_o, po) == cudaSuccess && cudaMalloc(&p->part_ml, pm) == cudaSuccess &&
+                  cudaMalloc(&p->part_o2, po) == cudaSuccess && cudaMalloc(&p->part_ml2, pm) == cudaSuccess &&
+                  cudaMalloc(&p->d_counters2, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
+                  cudaMemset(p->d_counters2, 0, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
                   cudaMalloc(&p->d_status, 4) == cudaSuccess && cudaMalloc(&p->d_q, qb) == cudaSuccess &&
                   cudaMalloc(&p->d_counters, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
                   cudaMemset(p->d_counters, 0, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
@@ -596,7 +608,8 @@ cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, 
 // token (one per request) instead of finding it in the slab.
 int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
                               const odma_tables* tables, void* out, float* lse, void* stream,
-                              const void* k_new, const void* v_new, const InlineLens* lens = nullptr) {
+                              const void* k_new, const void* v_new, const InlineLens* lens = nullptr,
+                              int32_t chain_pos = -1) {
     int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
     if (rc != ODMA_OK) return rc;
     DecodeParams p;
@@ -613,6 +626,16 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
             if (p.stages < 2) return ODMA_ERR_INVALID;
             fused = p.counters != nullptr;
+            if (chain_pos >= 0 && fused && uses_umma(pool, p.group)) {
+                // layer `chain_pos` of a step over several layers: scratch sets alternate, and every
+                // layer but the first runs chained to the one before
+                if (chain_pos & 1) {
+                    p.part_o = pool->part_o2;
+                    p.part_ml = pool->part_ml2;
+                    p.counters = pool->d_counters2;
+                }
+                p.chained = chain_pos > 0 ? 1 : 0;
+            }
             e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens);
         } else if (generic_supported(pool->head_dim)) {
             p.counters = nullptr;
@@ -696,7 +719,8 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
         rc = decode_attention_impl(pool, layer + l, static_cast<const uint8_t*>(d_q) + l * qb, q_heads, &t,
                                    static_cast<uint8_t*>(d_out) + l * qb,
                                    lse ? lse + static_cast<size_t>(l) * n * q_heads : nullptr, stream,
-                                   fuse ? kn : nullptr, fuse ? vn : nullptr, inline_lens ? &lens : nullptr);
+                                   fuse ? kn : nullptr, fuse ? vn : nullptr, inline_lens ? &lens : nullptr,
+                                   fuse && n_layers > 1 ? l : -1);
         if (rc != ODMA_OK) return rc;
     }
     if (tables_out) *tables_out = t;
@@ -773,7 +797,8 @@ int32_t odma_check_status(odma_pool* pool, void* stream) {
     if (word != 0) {
         // a kernel that gave up may have left split streams half counted
         if (cudaMemset(pool->d_status, 0, 4) != cudaSuccess ||
-            cudaMemset(pool->d_counters, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess)
+            cudaMemset(pool->d_counters, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess ||
+            cudaMemset(pool->d_counters2, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess)
             return ODMA_ERR_CUDA;
     }
     return (word & kStatusTimeout) ? ODMA_ERR_TIMEOUT : ODMA_OK;

@@ -57,7 +57,7 @@ namespace {
 using namespace dev;
 
 constexpr int kTile = 64;
-constexpr int kUmmaWarps = 7;
+constexpr int kUmmaWarps = 8;
 constexpr int kUmmaThreads = kUmmaWarps * 32;
 constexpr int kMaxStages = 8;
 constexpr int kQSlots = 8;
@@ -258,11 +258,40 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
     // Programmatic dependent launch: all of the above may run while the previous kernel of the
     // stream drains, and so may the producer's first loads of rows nobody can be writing; the
-    // rest comes after the dependency wait.  The next kernel is let go only after this wait, so
-    // a kernel can overlap with its immediate predecessor only.
-    if (warp != 1) {
+    // rest comes after the dependency wait.  The next kernel is let go only after this wait (by
+    // warp 7, which does nothing else), so a kernel can overlap with its immediate predecessor
+    // only.  A chained launch (layer l > 0 of a step over several layers) follows this kernel on
+    // layer l - 1: other K/V arrays, other outputs, the other scratch set, inputs that were
+    // complete when the step was issued; none of its roles waits, and its CTAs do real work on
+    // every SM the previous layer's CTAs have left.  (Warp 7 still waits before letting the next
+    // launch go: the kernel two launches back, which used the same scratch set, is complete
+    // before any CTA of this one starts.)
+    const bool chained = p.chained != 0;
+    if (warp == 3 && !chained) {
+        // Before the wait nothing may be READ that the previous kernel could still be writing,
+        // but a line may be asked into L2 (the point of coherence: a later write lands in the
+        // same line): the queries and new rows of the CTA's first items, so that the loads after
+        // the wait are L2 hits.
+        for (int it = it_begin + (lane >> 2); it < it_end && it < it_begin + kQSlots; it += 8) {
+            const int4 a = __ldg(p.items + 2 * it), b = __ldg(p.items + 2 * it + 1);
+            const Item im = item_of(a, b, lens, fused);
+            const uint8_t* src = static_cast<const uint8_t*>(p.q) +
+                                 (static_cast<size_t>(im.req) * p.q_heads + static_cast<size_t>(im.head) * p.group) * D * 2;
+            for (int off = (lane & 3) * 128; off < p.group * D * 2; off += 512)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(src + off) : "memory");
+            if (im.has_new && (lane & 3) < 2) {
+                const size_t nrow = (static_cast<size_t>(im.req) * p.kv_heads + im.head) * D * 2;
+                const uint8_t* nsrc = static_cast<const uint8_t*>((lane & 1) ? p.v_new : p.k_new) + nrow;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc) : "memory");
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + 128) : "memory");
+            }
+        }
+    }
+    if (warp == 7) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    } else if (warp != 1 && !chained) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
     }
 
     // item walk shared by the roles: descriptor of item `it`, the next one already on its way
@@ -321,7 +350,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // requested before the dependency wait, so that HBM is already streaming while the
         // previous grid finishes.
         int n_early = 0;
-        if (MODE != kModePaged) {
+        if (MODE != kModePaged && !chained) {
             const int4* r = p.cta + 3 * cta;
             int4 a = __ldg(r + 1), b = __ldg(r + 2);
             for (int it = it_begin; it < it_end && n_early < static_cast<int>(STAGES); ++it) {
@@ -334,8 +363,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     issue_tile(static_cast<uint32_t>(n_early), im, t, 1);
             }
         }
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        if (!chained) asm volatile("griddepcontrol.wait;" ::: "memory");
 
         uint32_t g = 0;                               // tiles issued so far
         fetch(it_begin);
@@ -422,9 +450,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         uint32_t g = 0;
         fetch(it_begin);
         for (int it = it_begin; it < it_end && ok; ++it) {
-            const int k = it - it_begin, L = k & 1;
+            const int k = it - it_begin;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
             fetch(it + 1);
+            const int L = k & 1;
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
             if (!ok) break;
@@ -438,10 +467,14 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             for (int t = 0; t < im.tiles; ++t, ++g) {
                 const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
                 const uint32_t cc = L ? c[1] : c[0], b = cc & 1u, u = cc >> 1;
-                bool good = mbar_wait(bar(kBarFull + stage), phase, abort_flag, p.status, limit);
-                if (good) good = mbar_wait(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit);
-                ok = __all_sync(0xFFFFFFFFu, good);
-                if (!ok) break;
+                // both barriers are looked at before either answer is needed; the slow path only when one is not ready
+                const bool f_ok = mbar_try(bar(kBarFull + stage), phase), e_ok = mbar_try(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u);
+                if (!__all_sync(0xFFFFFFFFu, f_ok && e_ok)) {
+                    bool good = f_ok || mbar_wait_slow(bar(kBarFull + stage), phase, abort_flag, p.status, limit);
+                    if (good && !e_ok) good = mbar_wait_slow(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit);
+                    ok = __all_sync(0xFFFFFFFFu, good);
+                    if (!ok) break;
+                }
                 tc_fence_after();
                 const uint32_t kbase = kv_u32 + stage * Cfg::kStageBytes;
                 const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + b * 64u;
@@ -482,7 +515,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             if ((k & 1) != L || im.tiles == 0) continue;
             for (int t = 0; t < im.tiles; ++t, ++c) {
                 const uint32_t b = c & 1u, u = c >> 1, st = (g0 + static_cast<uint32_t>(t)) % STAGES;
-                bool good = mbar_wait(lane_bar(L, P_FULL + b), u & 1u, abort_flag, p.status, limit);
+                bool good = mbar_wait_spin(lane_bar(L, P_FULL + b), u & 1u, abort_flag, p.status, limit);
                 if (good && t == 0) good = mbar_wait(lane_bar(L, O_EMPTY), (j & 1u) ^ 1u, abort_flag, p.status, limit);
                 ok = __all_sync(0xFFFFFFFFu, good);
                 if (!ok) break;
@@ -571,7 +604,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             }
             for (int t = 0; t < im.tiles; ++t) {
                 const uint32_t b = c & 1u, u = c >> 1;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
                 if (!ok) break;
                 tc_fence_after();
                 uint32_t r[32];
@@ -678,7 +711,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             // ---- the item's result: O from tensor memory, then out / partial / merge
             float oo[NT][D / 4];                          // [rs][2i + e]: head hq + 8 rs, element 8i + kq + e
             if (im.tiles > 0) {
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
@@ -749,8 +782,8 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             }
             if (p.counters == nullptr) continue;           // a combine kernel follows
             // The CTA that delivers a split stream's last piece merges all of them, in slot
-            // order (so the result does not depend on which CTA that is): its own piece from the
-            // registers it still holds, the others read back through L2.
+            // order (so the result does not depend on which CTA that is), reading them back
+            // through L2 (its own included), the next piece's loads in flight while one is folded.
             const int4 cr = __ldg(p.combine + im.comb);   // {request, head, first slot, pieces}
             __syncwarp();
             int is_last = 0;
@@ -770,33 +803,34 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 float fm = -INFINITY, fl = 0.f, fa[D / 4];
 #pragma unroll
                 for (int i = 0; i < D / 4; ++i) fa[i] = 0.f;
-                for (int s = 0; s < cr.w; ++s) {
-                    float m, l, x[D / 4];
-                    if (cr.z + s == im.slot) {
-                        m = m_ref[rs];
-                        l = l_acc[rs];
+                auto load = [&](int s, float2& ml, float2 (&x)[D / 8]) {
+                    const size_t prow = static_cast<size_t>(cr.z + s) * group + h;
+                    ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
+                    const float* po = p.part_o + prow * D + kq;
 #pragma unroll
-                        for (int i = 0; i < D / 4; ++i) x[i] = oo[rs][i];
-                    } else {
-                        const size_t prow = static_cast<size_t>(cr.z + s) * group + h;
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
-                        m = ml.x;
-                        l = ml.y;
-                        const float* po = p.part_o + prow * D + kq;
-#pragma unroll
-                        for (int i = 0; i < D / 8; ++i) {
-                            const float2 v = __ldcg(reinterpret_cast<const float2*>(po + 8 * i));
-                            x[2 * i] = v.x;
-                            x[2 * i + 1] = v.y;
-                        }
-                    }
-                    const float mn = fmaxf(fm, m);
+                    for (int i = 0; i < D / 8; ++i) x[i] = __ldcg(reinterpret_cast<const float2*>(po + 8 * i));
+                };
+                auto fold = [&](const float2& ml, const float2 (&x)[D / 8]) {
+                    const float mn = fmaxf(fm, ml.x);
                     const float e0 = fm == -INFINITY ? 0.f : fast_exp2(fm - mn);
-                    const float e1 = m == -INFINITY ? 0.f : fast_exp2(m - mn);
-                    fl = fmaf(fl, e0, l * e1);
+                    const float e1 = ml.x == -INFINITY ? 0.f : fast_exp2(ml.x - mn);
+                    fl = fmaf(fl, e0, ml.y * e1);
 #pragma unroll
-                    for (int i = 0; i < D / 4; ++i) fa[i] = fmaf(fa[i], e0, x[i] * e1);
+                    for (int i = 0; i < D / 8; ++i) {
+                        fa[2 * i] = fmaf(fa[2 * i], e0, x[i].x * e1);
+                        fa[2 * i + 1] = fmaf(fa[2 * i + 1], e0, x[i].y * e1);
+                    }
                     fm = mn;
+                };
+                float2 ml_a, ml_b, x_a[D / 8], x_b[D / 8];
+                load(0, ml_a, x_a);
+                for (int s = 0; s < cr.w; s += 2) {
+                    if (s + 1 < cr.w) load(s + 1, ml_b, x_b);
+                    fold(ml_a, x_a);
+                    if (s + 1 < cr.w) {
+                        if (s + 2 < cr.w) load(s + 2, ml_a, x_a);
+                        fold(ml_b, x_b);
+                    }
                 }
                 write_out(cr.x, cr.y, rs, fm, fl, fa);
             }

@@ -87,6 +87,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_slow(bar, parity, abort_flag, status, limit_ns);
 }
 
+// For hand-overs on a latency-critical chain: polls with test_wait (a waiter parked in try_wait
+// takes noticeably longer to see the phase complete), then falls back to the bounded wait.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               uint32_t* status, int64_t limit_ns) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+        if (mbar_test(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, limit_ns);
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x,
                                             int32_t y, uint32_t bar) {
     asm volatile(

@@ -39,6 +39,9 @@ struct DecodeParams {
     const int32_t* page_table;  // [n, max_pages]
     int32_t max_pages;
     int64_t wait_limit_ns;
+    int32_t chained;            // tcgen05 kernel: the previous kernel of the stream is this kernel on the
+                                // previous layer of the same step (same plan, other K/V arrays, other
+                                // outputs, the other scratch set): nothing of this launch waits for it
     int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
 };

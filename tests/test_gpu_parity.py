@@ -394,6 +394,56 @@ def test_back_to_back_steps_on_one_layer_without_host_syncs():
         assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
 
 
+@pytest.mark.parametrize("ctas", [0, 5])
+def test_layers_of_one_step_run_chained_without_host_syncs(ctas):
+    """odma_decode_step over six layers, three steps enqueued back to back: the kernel of layer
+    l > 0 does not wait for the kernel of layer l - 1 (other K/V arrays, other outputs, the other
+    scratch set), so kernels of neighbouring layers run side by side.  Every layer of every
+    step against the checker, and every appended row in place."""
+    odma = lib()
+    lens = [0, 40, 64, 129, 700, 1500, 2771]
+    w = qwen_small(lens, layers=6)
+    w = wl.scaled(w, predicted=w.context + 8)
+    s = Session(w, plan_ctas=ctas)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    pre = [r for r in reqs if w.context[r] > 0]
+    s.append(pre, [int(w.context[r]) for r in pre])
+    steps, NL = 3, w.layers
+    qs = [torch.stack([s.queries(l, reqs, w.q_heads, k) for l in range(NL)]).contiguous() for k in range(steps)]
+    kns = [torch.stack([torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]) for l in range(NL)]).contiguous()
+           for k in range(steps)]
+    vns = [torch.stack([torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]) for l in range(NL)]).contiguous()
+           for k in range(steps)]
+    outs = [torch.full_like(qs[0], float("nan")) for _ in range(steps)]
+    lses = [torch.full((NL, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev) for _ in range(steps)]
+    torch.cuda.synchronize()
+    t = odma.Tables()
+    for k in range(steps):                       # no synchronisation inside this loop
+        s.pool.decode_step(0, NL, w.q_heads, reqs, qs[k].data_ptr(), kns[k].data_ptr(), vns[k].data_ptr(),
+                           outs[k].data_ptr(), lses[k].data_ptr(), s.stream, t)
+        s.ls.commit(reqs, 1)
+    torch.cuda.synchronize()
+    assert s.pool.check_status(s.stream) == odma.OK
+    if ctas == 0:
+        assert t.n_combine > 0
+    for k in range(steps):
+        for l in range(NL):
+            for i, r in enumerate(reqs):
+                s.kv.append(r, l, kns[k][l, i:i + 1], vns[k][l, i:i + 1])
+            ref, ref_lse, _ = s.oracle_out(l, reqs, qs[k][l], w.q_heads)
+            assert torch.isfinite(outs[k][l].float()).all()
+            assert_close(outs[k][l], ref, w.dtype, f"step {k} layer {l}")
+            assert np.abs(lses[k][l].double().cpu().numpy() - ref_lse).max() <= 2e-2
+    for r in reqs:
+        s.lens[r] += steps
+        for l in range(NL):
+            k_ref, v_ref = s.kv.gathered(r, l)
+            assert np.array_equal(s.pool_rows(l, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+            assert np.array_equal(s.pool_rows(l, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
 @pytest.mark.parametrize("fused", [1, 0])
 def test_profile_counts_launches(fused):
     odma = lib()
