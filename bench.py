@@ -40,6 +40,7 @@ METRIC = "decode tokens/s (slab-KV attention path: append + split decode + combi
 UNIT = "tokens/s"
 L2_BYTES = 126 * 2**20
 FALLBACK_HBM_GBS = 6650.0
+DECODE_KERNELS = {"auto": 0, "tcgen05": 1, "mma_sync": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum per decode-kernel launch, from the ncu capture
 # summarised under profiles/ (None once the kernel has changed since the capture)
 TRAFFIC = {"config2": 72.79e6 + 1.56e6}
@@ -150,7 +151,7 @@ class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
     def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0,
-                 fused: int = 1):
+                 fused: int = 1, decode_kernel: int = 0):
         from paper_2512_09427_b200 import odma
         self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
         self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
@@ -165,6 +166,7 @@ class SlabDecode:
         cfg.max_batch = max(1024, w.batch)
         cfg.plan_ctas = plan_ctas
         cfg.fused_combine = fused
+        cfg.decode_kernel = decode_kernel
         self.pool_cfg = cfg
         self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
         self.stream = torch.cuda.current_stream().cuda_stream
@@ -453,7 +455,7 @@ def run_ours(args):
     phases = set(args.phases.split(","))
     K, W = args.steps, args.warmup
     w, step_layers, copies = pick_workload(args.workload, rank, args.copies, args.layers)
-    sd = SlabDecode(w, step_layers, dev, fused=args.fused_combine)
+    sd = SlabDecode(w, step_layers, dev, fused=args.fused_combine, decode_kernel=DECODE_KERNELS[args.decode_kernel])
     bounds, epoch = sd.learn_boundaries()
     sd.admit_and_fill()
     q, kn, vn, out = sd.make_inputs()
@@ -649,7 +651,7 @@ def run_config4(args):
         kv_bytes = int((w.context + 1).sum()) * 2 * w.kv_heads * w.head_dim * w.elem_bytes
         copies = max(2, -(-3 * L2_BYTES // kv_bytes))               # rotate over copies: cold L2
         wc = wl.scaled(w, layers=copies, pool_bytes=w.pool_bytes * copies)
-        sd = SlabDecode(wc, 1, dev, fused=args.fused_combine)
+        sd = SlabDecode(wc, 1, dev, fused=args.fused_combine, decode_kernel=DECODE_KERNELS[args.decode_kernel])
         sd.learn_boundaries()
         sd.admit_and_fill()
         q, kn, vn, out = sd.make_inputs()
@@ -705,6 +707,8 @@ def main():
                          "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
                          "paged (page-16 ablation of the decode kernel on the same inputs)")
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
+    ap.add_argument("--decode-kernel", default="auto", choices=list(DECODE_KERNELS),
+                    help="which bf16 decode kernel the pool runs (auto: the library's choice per shape)")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
     ap.add_argument("--layers", type=int, default=0,
                     help="config3/config5: step through this many layers only (0 = all 28; a reduced size for profiler "

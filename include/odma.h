@@ -96,9 +96,10 @@ typedef struct odma_config {
                                 kernel take the step's new token from k_new / v_new and write
                                 it into the slab itself (one launch per layer); 0: they launch
                                 the append kernel first (1) */
-    int32_t decode_kernel;   /* bf16 decode kernel: ODMA_DECODE_AUTO picks per shape,
-                                ODMA_DECODE_TCGEN05 the tcgen05 / tensor-memory kernel,
-                                ODMA_DECODE_MMA_SYNC the mma.sync kernel (0) */
+    int32_t decode_kernel;   /* bf16 decode kernel: ODMA_DECODE_TCGEN05 the tcgen05 / tensor-memory
+                                kernel, ODMA_DECODE_MMA_SYNC the mma.sync kernel, ODMA_DECODE_AUTO
+                                the first for the layers of an odma_decode_step over several
+                                layers and the second for single launches (0) */
 } odma_config;
 
 typedef struct odma_slab {

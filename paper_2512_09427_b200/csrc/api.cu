@@ -592,16 +592,20 @@ bool uses_tc(const odma_pool* pool, int32_t q_heads) {
     return pool->has_maps && tc_supported(pool->head_dim, q_heads / pool->kv_heads);
 }
 
-// Which of the two tensor-core kernels runs a launch: the tcgen05 one unless the pool was
-// configured for mma.sync.
-bool uses_umma(const odma_pool* pool, int32_t group) {
-    return pool->alloc.config().decode_kernel != ODMA_DECODE_MMA_SYNC && umma_supported(pool->head_dim, group);
+// Which of the two tensor-core kernels runs a launch.  ODMA_DECODE_AUTO: the tcgen05 kernel for
+// the layers of a step that spans several layers (its launches chain without dependency waits;
+// measured 3 to 6 % faster on the 28-layer workloads), the mma.sync kernel for single launches
+// (3 to 4 % faster there: its last tile and hand-over are a shorter chain).
+bool uses_umma(const odma_pool* pool, int32_t group, bool part_of_multi_layer_step) {
+    const int32_t want = pool->alloc.config().decode_kernel;
+    if (want == ODMA_DECODE_MMA_SYNC || !umma_supported(pool->head_dim, group)) return false;
+    return want == ODMA_DECODE_TCGEN05 || part_of_multi_layer_step;
 }
 
 cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, const DecodeParams& p, int mode,
-                                 int n_ctas, cudaStream_t stream, const InlineLens* lens) {
-    return uses_umma(pool, p.group) ? launch_decode_umma(maps, p, mode, n_ctas, stream, lens)
-                                    : launch_decode_tc(maps, p, mode, n_ctas, stream, lens);
+                                 int n_ctas, cudaStream_t stream, const InlineLens* lens, bool umma) {
+    return umma ? launch_decode_umma(maps, p, mode, n_ctas, stream, lens)
+                : launch_decode_tc(maps, p, mode, n_ctas, stream, lens);
 }
 
 // odma_decode_attention; with k_new / v_new the tensor-core kernel also appends the step's
@@ -626,7 +630,8 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
             if (p.stages < 2) return ODMA_ERR_INVALID;
             fused = p.counters != nullptr;
-            if (chain_pos >= 0 && fused && uses_umma(pool, p.group)) {
+            const bool umma = uses_umma(pool, p.group, chain_pos >= 0);
+            if (chain_pos >= 0 && fused && umma) {
                 // layer `chain_pos` of a step over several layers: scratch sets alternate, and every
                 // layer but the first runs chained to the one before
                 if (chain_pos & 1) {
@@ -636,7 +641,7 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
                 }
                 p.chained = chain_pos > 0 ? 1 : 0;
             }
-            e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens);
+            e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens, umma);
         } else if (generic_supported(pool->head_dim)) {
             p.counters = nullptr;
             e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
@@ -977,7 +982,8 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
     cudaError_t e;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
-        e = launch_tensor_decode(pool, paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream), nullptr);
+        e = launch_tensor_decode(pool, paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream), nullptr,
+                                 uses_umma(pool, p.group, false));
     }
     if (e != cudaSuccess) return ODMA_ERR_CUDA;
     if (tables->n_combine > 0 && p.counters == nullptr) {

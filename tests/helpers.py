@@ -14,9 +14,15 @@ def lib():
     return odma
 
 
+# configuration fields applied to every pool a test creates (a module's fixture may set, say,
+# the decode kernel to run the same tests on both tensor-core kernels)
+CFG_DEFAULTS = {}
+
+
 def make_cfg(w: wl.Workload, **over):
     odma = lib()
     cfg = odma.config_default()
+    over = {**CFG_DEFAULTS, **over}
     cfg.safety_pct, cfg.max_len, cfg.granule = w.safety_pct, w.max_len, w.granule
     cfg.window, cfg.refresh = w.window, w.refresh
     pn, pd = w.quantiles

@@ -16,6 +16,15 @@ from paper_2512_09427_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=[1, 2], ids=["tcgen05", "mma_sync"])
+def decode_kernel(request):
+    """Every test of this module runs once on each bf16 tensor-core decode kernel."""
+    import helpers
+    helpers.CFG_DEFAULTS["decode_kernel"] = request.param
+    yield request.param
+    helpers.CFG_DEFAULTS.clear()
+
+
 def checker_out(w, layer, reqs, lens, q):
     """fp64 attention of `reqs` (KV lengths `lens`) on `layer` from regenerated inputs."""
     Ks = [wl.kv_rows(w.seed, layer, r, wl.KIND_K, 0, L, w.kv_heads, w.head_dim, w.dtype) for r, L in zip(reqs, lens)]
@@ -174,14 +183,14 @@ def test_config4_drift_stream_attention_at_boundary_epochs():
           "utilisation %.3f" % (st["sum_len_completed"] / st["sum_cap_completed"]))
 
 
-def test_config2_in_the_benchmarks_own_launch_configuration():
+def test_config2_in_the_benchmarks_own_launch_configuration(decode_kernel):
     """bench.py's set-up and step for config 2 (rotating KV copies, odma_decode_step with the
     append and the merge inside the decode kernel, plan reused from step to step): outputs of
     sampled requests on two of the copies against the checker, and the appended rows in place."""
     import bench
     odma = lib()
     w, step_layers, copies = bench.pick_workload("config2")
-    sd = bench.SlabDecode(w, step_layers, torch.device("cuda:0"))
+    sd = bench.SlabDecode(w, step_layers, torch.device("cuda:0"), decode_kernel=decode_kernel)
     bounds, epoch = sd.learn_boundaries()
     assert len(bounds) == 4 and epoch == 10
     sd.admit_and_fill()

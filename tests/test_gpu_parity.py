@@ -9,6 +9,15 @@ from paper_2512_09427_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
+
+@pytest.fixture(autouse=True, params=[1, 2], ids=["tcgen05", "mma_sync"])
+def decode_kernel(request):
+    """Every test of this module runs once on each bf16 tensor-core decode kernel."""
+    import helpers
+    helpers.CFG_DEFAULTS["decode_kernel"] = request.param
+    yield request.param
+    helpers.CFG_DEFAULTS.clear()
+
 RAGGED = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 500, 1000, 2771]
 
 
