@@ -41,9 +41,7 @@ UNIT = "tokens/s"
 L2_BYTES = 126 * 2**20
 FALLBACK_HBM_GBS = 6650.0
 DECODE_KERNELS = {"auto": 0, "tcgen05": 1, "mma_sync": 2}
-# dram__bytes_read.sum + dram__bytes_write.sum per decode-kernel launch, from the ncu capture
-# summarised under profiles/ (None once the kernel has changed since the capture)
-TRAFFIC = {"config2": 72.79e6 + 1.56e6}
+MIN_TIMED_SECONDS = 0.5      # the K-step region is repeated until this much device time has been timed
 
 
 # ---------------------------------------------------------------------------------------------
@@ -426,6 +424,34 @@ def workload_config(w, name, step_layers, copies):
                    if copies > 1 else f"one step streams {step_layers * kv_bytes_layer >> 20} MiB of KV (> L2)")}
 
 
+def kernel_sources_hash() -> str:
+    """sha256 over the CUDA/C++ sources of the library: identifies the kernels a counter capture
+    was taken from."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    base = os.path.join(ROOT, "paper_2512_09427_b200", "csrc")
+    for f in sorted(glob.glob(os.path.join(base, "*"))):
+        h.update(os.path.basename(f).encode())
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, kernel: str):
+    """DRAM bytes (read + written) per launch of the decode kernel from the ncu capture noted in
+    profiles/traffic.json, or None when there is no capture of this kernel on this workload or
+    the kernel sources have changed since it was taken."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            rec = json.load(f)[f"{workload}:{kernel}"]
+    except Exception:
+        return None
+    if rec.get("sources_sha256_16") != kernel_sources_hash():
+        return None
+    return float(rec["dram_bytes_per_launch"])
+
+
 def measured_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -470,27 +496,50 @@ def run_ours(args):
     step_no = 0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    # ---- warm-up, then exactly K timed steps -------------------------------------------------
+    # ---- warm-up, then regions of exactly K timed steps ------------------------------------------
+    # One region = K consecutive steps between two CUDA events on the launch stream.  A region of
+    # the default K lasts a fraction of a millisecond, so regions are enqueued back to back until
+    # MIN_TIMED_SECONDS of device time have been timed (no host synchronisation in between);
+    # `ms_per_step` is the median region, the spread is reported beside it.  Barrier and
+    # synchronize bracket the whole timed part, and the clock sampler covers exactly it.
     for _ in range(W):
         sd.step(step_no, q, kn, vn, out, tables)
         step_no += 1
     barrier()
-    t_wall0 = time.time()
     ev0.record()
-    for _ in range(K):
+    for _ in range(max(W, 3)):
         sd.step(step_no, q, kn, vn, out, tables)
         step_no += 1
     ev1.record()
+    torch.cuda.synchronize()
+    est_ms = max_over_ranks([ev0.elapsed_time(ev1) / max(W, 3)], dist, dev)[0]
+    n_regions = int(min(5000, max(5, -(-MIN_TIMED_SECONDS * 1e3 // max(K * est_ms, 1e-6)))))
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_regions + 1)]
+    barrier()
+    t_wall0 = time.time()
+    marks[0].record()
+    for r in range(n_regions):
+        for _ in range(K):
+            sd.step(step_no, q, kn, vn, out, tables)
+            step_no += 1
+        marks[r + 1].record()
     barrier()
     if clocks:
         clocks.mark(t_wall0, time.time())
-    ms = ev0.elapsed_time(ev1)
+    region_ms = max_over_ranks([marks[r].elapsed_time(marks[r + 1]) for r in range(n_regions)], dist, dev)
+    ms = statistics.median(region_ms)
     assert sd.pool.check_status(sd.stream) == odma.OK
     fused_append = bool(sd.pool_cfg.fused_append) and w.dtype == torch.bfloat16
     launches_per_step = step_layers * (1 + (0 if fused_append else 1) +
                                        (1 if tables.n_combine > 0 and not args.fused_combine else 0))
     kv_bytes_per_launch = tables.kv_tokens * 2 * w.kv_heads * row_bytes
     step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes)
+    if w.dtype != torch.bfloat16:
+        kernel_name = "decode_generic_kernel"
+    elif args.decode_kernel == "tcgen05" or (args.decode_kernel == "auto" and step_layers > 1):
+        kernel_name = "decode_umma_kernel"
+    else:
+        kernel_name = "decode_tc_kernel"
 
     # ---- the same steps with every launch bracketed by CUDA events (per-kernel time) ----------
     roofline, kernels_us = None, None
@@ -514,16 +563,41 @@ def run_ours(args):
         # bracketed one by one are used (each bracket adds the events' own latency).
         bracketed_us = dec_ms / dec_n * 1e3
         if launches_per_step == step_layers:
-            us, how, timed_n = ms / (K * step_layers) * 1e3, "timed region: consecutive launches between two events", K * step_layers
+            us, how, timed_n = ms / (K * step_layers) * 1e3, "median timed region: K steps of consecutive launches between two events", K * step_layers
         else:
             us, how, timed_n = bracketed_us, "each launch bracketed by two events", dec_n
         achieved = kv_bytes_per_launch / (us * 1e-6) / 1e9
-        roofline = {"bound": "hbm", "kernel": "decode_tc_kernel", "achieved": achieved, "peak": peak,
-                    "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": TRAFFIC.get(args.workload),
+        isolated = kv_bytes_per_launch / (bracketed_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                    "traffic": recorded_traffic(args.workload, kernel_name),
                     "bytes_per_launch": kv_bytes_per_launch, "us_per_launch": us, "timing": how,
-                    "launches_timed": timed_n, "us_per_launch_bracketed": bracketed_us}
+                    "launches_timed": timed_n, "us_per_launch_bracketed": bracketed_us,
+                    "frac_isolated": isolated / peak}
         kernels_us = {"append": app_ms / max(app_n, 1) * 1e3, "decode": dec_ms / dec_n * 1e3,
                       "combine": cmb_ms / cmb_n * 1e3 if cmb_n else 0.0}
+
+    # ---- the read probe: the decode kernel's loads and barrier traffic with no arithmetic, launched
+    #      the way the timed steps are (consecutive launches between two events)
+    probe_line = None
+    if "probe" in phases and w.dtype == torch.bfloat16:
+        own_p = torch.empty(sd.pool.tables_bytes(n), dtype=torch.uint8, device=dev)
+        tables_p = sd.pool.build_tables(sd.reqs, own_p.data_ptr(), own_p.numel(), sd.stream)
+        reps = max(20, min(K, 200)) if step_layers == 1 else 2
+        for timed in (False, True):
+            if timed:
+                ev0.record()
+            for i in range(reps * step_layers):
+                sd.pool.read_probe(i % w.layers, w.q_heads, tables_p, sd.stream)
+            if timed:
+                ev1.record()
+            torch.cuda.synchronize()
+        assert sd.pool.check_status(sd.stream) == odma.OK
+        p_us = ev0.elapsed_time(ev1) / (reps * step_layers) * 1e3
+        probe_line = {"us_per_launch": p_us, "GBs": kv_bytes_per_launch / (p_us * 1e-6) / 1e9,
+                      "frac": kv_bytes_per_launch / (p_us * 1e-6) / 1e9 / peak, "launches": reps * step_layers,
+                      "kernel": "decode_tc_kernel<probe>"}
+        del own_p
 
     # ---- contiguity ablation: the same requests re-laid in 16-token pages (shuffled), same kernel
     paged_line = None
@@ -557,7 +631,8 @@ def run_ours(args):
             sd.pool.profile_enable(False)
             res[kind] = {"us_per_launch": t_ms / cnt * 1e3, "GBs": kv_bytes_per_launch / (t_ms / cnt * 1e-3) / 1e9}
         assert sd.pool.check_status(sd.stream) == odma.OK
-        paged_line = {"pages": "16 tokens, ids shuffled", **res}
+        paged_line = {"pages": "16 tokens, ids shuffled", "timing": "each launch bracketed by two events", **res,
+                      "slab_over_paged": res["paged"]["us_per_launch"] / res["slab"]["us_per_launch"]}
         del pages, paged
 
     # ---- end to end from pinned host buffers ---------------------------------------------------
@@ -583,26 +658,17 @@ def run_ours(args):
     else:
         e2e_steps, e2e_ms = 1, float("nan")
 
-    # ---- if the timed passes were too short for the 50 ms sampler, repeat the same step under it
-    clk = None
-    if clocks:
-        if sum(b - a for a, b in clocks.windows) < 1.0:
-            t0w = time.time()
-            while time.time() - t0w < 1.2:
-                for _ in range(20):
-                    sd.step(step_no, q, kn, vn, out, tables)
-                    step_no += 1
-            torch.cuda.synchronize()
-            clocks.mark(t0w, time.time())
-        clk = clocks.stop()
+    clk = clocks.stop() if clocks else None
 
     # ---- max over ranks ------------------------------------------------------------------------
-    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, dev)
+    e2e_ms = max_over_ranks([e2e_ms], dist, dev)[0]
     value = world * n * K / (ms * 1e-3)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
             "config": workload_config(w, args.workload, step_layers, copies),
+            "regions": {"count": n_regions, "steps_each": K, "ms_per_step_min": min(region_ms) / K,
+                        "ms_per_step_max": max(region_ms) / K, "timed_seconds": sum(region_ms) * 1e-3},
             "step_gbs": step_bytes / (ms / K * 1e-3) / 1e9,
             "gpu_launches": int(launches_per_step * K),
             "plan": {"ctas": tables.n_ctas, "items": tables.n_items, "combine": tables.n_combine},
@@ -615,6 +681,9 @@ def run_ours(args):
                        "ms_per_step": e2e_ms / e2e_steps}
     if roofline:
         line["roofline"], line["kernels_us"] = roofline, kernels_us
+    if probe_line:
+        line["read_probe"] = probe_line
+        line["read_probe_gbs"] = probe_line["GBs"]
     if paged_line:
         line["page16_ablation"] = paged_line
     if clk:
@@ -702,10 +771,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--phases", default="timed,kernels,e2e,clocks,cpu",
+    ap.add_argument("--phases", default="",
                     help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
                          "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
-                         "paged (page-16 ablation of the decode kernel on the same inputs)")
+                         "probe (the no-arithmetic read probe), paged (page-16 ablation of the decode kernel on "
+                         "the same inputs); default: all of them on config2, all but paged elsewhere")
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
     ap.add_argument("--decode-kernel", default="auto", choices=list(DECODE_KERNELS),
                     help="which bf16 decode kernel the pool runs (auto: the library's choice per shape)")
@@ -716,6 +786,8 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if not args.phases:
+        args.phases = "timed,kernels,e2e,clocks,cpu,probe" + (",paged" if args.workload == "config2" else "")
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "config4":

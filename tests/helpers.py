@@ -145,6 +145,7 @@ class Session:
         odma = lib()
         self.odma, self.w = odma, w
         self.dev = torch.device("cuda:0")
+        self.gen_dev = self.dev          # where the seeded inputs are generated ("cpu": no generator kernels on the GPU)
         self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
         self.mem = torch.empty(w.pool_bytes, dtype=torch.uint8, device=self.dev)
         if fill is not None:
@@ -175,8 +176,9 @@ class Session:
     # -- data ---------------------------------------------------------------------------------
     def rows(self, layer, req, kind, t0, t1, scale=1.0):
         x = wl.kv_rows(self.w.seed, layer, req, kind, t0, t1, self.w.kv_heads, self.w.head_dim,
-                       self.w.dtype, self.dev)
-        return x if scale == 1.0 else (x.float() * scale).to(self.w.dtype)
+                       self.w.dtype, self.gen_dev)
+        x = x if scale == 1.0 else (x.float() * scale).to(self.w.dtype)
+        return x.to(self.dev)
 
     def append(self, reqs, n_new, layers=None, scale=1.0):
         """Append n_new[i] generated tokens to every request, on all layers; commit lengths."""
@@ -202,8 +204,9 @@ class Session:
 
     def queries(self, layer, reqs, q_heads, step=0, scale=1.0):
         q = torch.stack([wl.q_rows(self.w.seed, layer, int(r), step, q_heads, self.w.head_dim,
-                                   self.w.dtype, self.dev) for r in reqs]).contiguous()
-        return q if scale == 1.0 else (q.float() * scale).to(self.w.dtype)
+                                   self.w.dtype, self.gen_dev) for r in reqs]).contiguous()
+        q = q if scale == 1.0 else (q.float() * scale).to(self.w.dtype)
+        return q.to(self.dev)
 
     def decode_step(self, reqs, q_heads, layers=None, step=0, want_lse=True, scale=1.0):
         """One decode step: ensure room, build tables, then per layer append one token and attend.
