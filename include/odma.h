@@ -20,7 +20,12 @@
  *  - Kernel launchers are asynchronous on the given stream (a cudaStream_t passed as
  *    void*; NULL = the legacy default stream).  All device work of one pool must be
  *    issued on one stream, or be ordered by the caller: a slab released on the host may
- *    be handed out again while an earlier kernel still reads it otherwise.
+ *    be handed out again while an earlier kernel still reads it otherwise.  The decode
+ *    kernels are launched with programmatic stream serialization and read queries, new
+ *    rows and (after another decode launch of this library) slab rows only once the
+ *    kernels ahead of them have completed; a caller that writes pool memory, q, k_new or
+ *    v_new with kernels of its own must not let those signal their dependents early
+ *    (no programmatic launch trigger before the writes are done).
  *  - Host-side calls are not thread-safe; serialise calls on one pool.
  *  - Lengths and capacities are in tokens.  One token occupies
  *    layers * 2 * kv_heads * head_dim * elem_bytes bytes of the pool.
@@ -129,7 +134,8 @@ typedef struct odma_stats {
  *   item    = {request, kv_head, first_token, n_tokens, flags (bit 0: the piece is the whole
  *              stream, written out directly; bit 1: the piece ends its stream), slot,
  *              first row of the piece inside one K/V array, combine record (-1 if direct)};
- *             slots number all pieces in (request, head, token) order
+ *             slots number the pieces in plan order (longest streams first; the pieces of one
+ *             cut stream are consecutive, in token order)
  *   combine = {request, kv_head, first_slot, n_slots}
  * The off_* fields are word offsets of those arrays inside d_table. */
 typedef struct odma_tables {
@@ -200,8 +206,9 @@ int32_t odma_get_stats(const odma_pool* pool, odma_stats* out);
 /* ---- per-step tables -------------------------------------------------------------------
  * Slab table, lengths and the split plan for a batch of n live requests, each about to
  * append n_new[i] tokens (NULL = 1 each; 0 allowed).  Every request must already have room
- * (odma_ensure_capacity).  The plan cuts the batch's KV streams (one per request and KV
- * head) into equal shares of 64-token tiles, one share per persistent CTA.
+ * (odma_ensure_capacity).  The plan deals the batch's KV streams (one per request and KV
+ * head, read in 64-token tiles) to the persistent CTAs in shares of equal cost: streams longer
+ * than a share are cut into pieces, all others go whole, longest first, to the least loaded share.
  * odma_plan_host writes the table to host memory (no CUDA call); odma_build_tables writes
  * it to the caller's device buffer d_table with one asynchronous copy.  table_bytes must be
  * at least odma_tables_bytes(pool, n). */

@@ -41,6 +41,11 @@ struct odma_pool {
     int32_t layers = 0, kv_heads = 0, head_dim = 0, dtype = 0, elem_bytes = 0;
     int64_t rows_per_array = 0;
     int32_t plan_ctas = 148;
+    // The decode kernels start reading slab rows before their dependency wait, on the
+    // assumption that the kernel ahead of them in the stream is a decode kernel (which writes
+    // only the last row of each stream).  True after a decode launch, false after any other
+    // launch of the library that writes the pool (append, migration copy).
+    bool decode_was_last = false;
     uint32_t* d_counters = nullptr;   // per split stream: pieces delivered (fused combine)
     // a second scratch set: consecutive layers of one step alternate between the two, so that a
     // layer's kernel need not wait for the previous layer's
@@ -318,6 +323,7 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->max_pages = 0;
     p->wait_limit_ns = kDefaultWaitLimitNs;
     p->chained = 0;
+    p->early_ok = 0;
 }
 
 int32_t check_decode_args(const odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
@@ -494,6 +500,7 @@ int32_t odma_ensure_capacity(odma_pool* pool, uint64_t req, int32_t needed_len, 
     mp.arrays = pool->layers * 2;
     mp.kv_heads = pool->kv_heads;
     mp.row_vecs = pool->head_dim * pool->elem_bytes / 16;
+    pool->decode_was_last = false;
     ProfScope ps(pool, ODMA_K_MIGRATE, as_stream(stream));
     return launch_migrate(mp, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
@@ -578,6 +585,7 @@ int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables
     ap.n_new_total = tables->n_new_total;
     ap.row_vecs = pool->head_dim * pool->elem_bytes / 16;
     ap.one_new_each = tables->one_new_each;
+    pool->decode_was_last = false;
     ProfScope ps(pool, ODMA_K_APPEND, as_stream(stream));
     return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
@@ -625,6 +633,8 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
     }
     cudaError_t e;
     bool fused = false;
+    p.early_ok = pool->decode_was_last ? 1 : 0;
+    pool->decode_was_last = true;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {

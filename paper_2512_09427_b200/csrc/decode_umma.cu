@@ -124,7 +124,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // 16 lanes x 64 columns of 32 bits: lane t of the warp receives, in register 4i + j, row
 // t/4 + 8 (j/2), column 8i + 2 (t%4) + (j%2) (the accumulator layout of m16n8 tiles, repeated
@@ -239,7 +238,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // rows of the query slots beyond the group stay zero for the whole kernel
     for (int i = tid; i < Cfg::kQBytes / 16; i += kUmmaThreads)
         reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
-    fence_async_smem();
+    fence_proxy_async();
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(static_cast<uint32_t>(kTmemCols))
@@ -350,7 +349,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // requested before the dependency wait, so that HBM is already streaming while the
         // previous grid finishes.
         int n_early = 0;
-        if (MODE != kModePaged && !chained) {
+        if (MODE != kModePaged && !chained && p.early_ok) {
             const int4* r = p.cta + 3 * cta;
             int4 a = __ldg(r + 1), b = __ldg(r + 2);
             for (int it = it_begin; it < it_end && n_early < static_cast<int>(STAGES); ++it) {
@@ -433,7 +432,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                               ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
                 *slab = nv;
             }
-            fence_async_smem();
+            fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQFull + slot));
         }
@@ -701,7 +700,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                             make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
-                fence_async_smem();
+                fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(lane_bar(L, P_FULL + b));
                 ++c;

@@ -50,9 +50,9 @@ using namespace dev;
 // append fused in) the stream's new K and V rows travel through a ring of 4..8 slots so the
 // producer can run several short items ahead of the consumers.
 //
-// Shared memory is handed back (a query slot to the producer, a merge buffer to its group)
-// only behind a USE of the registers loaded from it: a load may still be in flight when a
-// later mbarrier.arrive of the same thread is performed, and the other side refills at once.
+// A query slot is refilled by bulk copies (async proxy) after generic-proxy reads of it: its
+// release (mbarrier arrive) is preceded by fence.proxy.async.  Merge buffers are written and
+// read through the generic proxy only; arrive (release) and wait (acquire) order them.
 //
 // The contraction is arranged with the KEYS on the M side of the MMA tiles and the query heads
 // of the GQA group on the N side (8 heads per n-tile; columns >= group hold whatever the
@@ -305,7 +305,7 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // requested before the dependency wait, so that HBM is already streaming while the
         // previous grid finishes; queries, new tokens and the rows in flux come after it.
         int n_early = 0;
-        if (MODE != kModePaged) {
+        if (MODE != kModePaged && p.early_ok) {
             for (int j = 0; j < 32 && it_begin + j < it_end && n_early < static_cast<int>(STAGES); ++j) {
                 int4 a = first_a, b = first_b;
                 int safe = first_r.safe;
@@ -471,13 +471,6 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                             const float4 x = *reinterpret_cast<const float4*>(bo + (w * ROWS + rr[i]) * MO + dd[i]);
                             lse_fold(acc_m[i], acc_l[i], acc[i], ml.x, ml.y, x);
                         }
-                    }
-                    {   // (the branch needs the folded sums, so the buffer reads are complete before
-                        //  the arrive below lets the group overwrite it; the sums are never negative)
-                        float seen = 0.f;
-#pragma unroll
-                        for (int i = 0; i < CH; ++i) seen += acc_l[i];
-                        if (seen < 0.f) *(abort_flag + 2) = 1;
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(mdone_bar(g));        // the buffer may be refilled
@@ -690,18 +683,10 @@ decode_tc_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 *dst = *reinterpret_cast<const uint4*>(nk + lane * 16);
             }
         }
-        if (MODE != kModeProbe) {
-            // The slot is refilled the moment its last reader lets go of it, and ldmatrix results
-            // may still be on their way to the registers when a later arrive is performed.  A
-            // use of every fragment register (the branch needs them all) keeps the arrive behind
-            // the loads; the store never happens in practice and touches a word nobody reads.
-            uint32_t fold = 0;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) fold ^= qb[nt][kk][0] + 3u * qb[nt][kk][1];
-            if (fold == 0x9E3779B9u) *(abort_flag + 2) = 1;
-        }
+        // The slot is refilled by a bulk copy (async proxy) the moment its last reader lets go of it;
+        // the reads above went through the generic proxy.  The cross-proxy fence orders them
+        // before the arrive that licenses the refill.
+        fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(qempty_bar(qs));
         if (++qs == QSLOTS) {
@@ -1137,16 +1122,20 @@ template <int D, int NT, int MODE>
 cudaError_t launch_tc_inst(const TensorMaps& maps, const DecodeParams& p, int n_ctas, cudaStream_t stream,
                            const InlineLens& lens) {
     using Cfg = TcConfig<D, NT>;
-    static bool configured = false;
+    static bool configured[64] = {false};          // the opt-in to large shared memory is per device
     auto kern = decode_tc_kernel<D, NT, MODE>;
     const int smem = Cfg::smem_bytes(p.stages, p.q_slots);
     if (p.stages < 2 || p.stages > kMaxStages || p.q_slots < kMinQSlots || p.q_slots > kMaxQSlots ||
         smem > kSmemPerCtaMax)
         return cudaErrorInvalidValue;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(static_cast<unsigned>(n_ctas));

@@ -39,6 +39,9 @@ struct DecodeParams {
     const int32_t* page_table;  // [n, max_pages]
     int32_t max_pages;
     int64_t wait_limit_ns;
+    int32_t early_ok;           // the previous kernel of the stream that wrote this pool was a decode kernel (it
+                                // appends one row per stream): rows up to two before a stream's end may be
+                                // requested before the dependency wait; 0: nothing is read before it
     int32_t chained;            // tcgen05 kernel: the previous kernel of the stream is this kernel on the
                                 // previous layer of the same step (same plan, other K/V arrays, other
                                 // outputs, the other scratch set): nothing of this launch waits for it

@@ -1,11 +1,13 @@
-// Split plan for one decode step: cuts the batch's KV streams into equal shares of tiles.
+// Split plan for one decode step: deals the batch's KV streams to the persistent CTAs in shares
+// of equal cost.
 //
-// A "stream" is the keys/values of one (request, KV head): one contiguous run in the slab.
-// All streams of the batch, laid end to end in (request, head) order, form a sequence of
-// 64-token tiles.  The plan gives each persistent CTA a contiguous share of that sequence, so
-// every CTA streams the same number of bytes (+-1 tile) whatever the length mix of the batch.
-// A share that ends inside a stream leaves a partial result (running max, sum, unnormalised
-// output) in a scratch slot; a stream covered by one share is written out directly.
+// A "stream" is the keys/values of one (request, KV head): one contiguous run in the slab, read
+// in 64-token tiles.  Streams longer than a share are cut into pieces that fill one share after
+// the other; all others go whole, longest first, to the share with the least load so far.  A
+// piece of a cut stream leaves a partial result (running max, sum, unnormalised output) in a
+// scratch slot and the CTA that delivers the last piece merges them; a whole stream is written
+// out directly.  Costs are in tiles: a tile 1, a stream's start-up 1, a piece of a cut stream 6
+// more (see plan_batch).
 #include "planner.hpp"
 
 #include <algorithm>
@@ -239,6 +241,9 @@ int32_t plan_batch(const PlanInput& in, int32_t* table, int64_t table_words, odm
         if (worst <= C + kSlackTiles + C / 16) break;
     }
     const int32_t n_items = static_cast<int32_t>(pieces.size());
+    // the table was sized for at most streams + ctas items and min(streams, ctas) cut streams
+    if (static_cast<int64_t>(t.off_items) + 8ll * n_items + static_cast<int64_t>(comb.size()) > table_words)
+        return ODMA_ERR_INVALID;
 
     // Group the pieces by share.  Each CTA works through its pieces of split streams first,
     // then through the whole streams: partial results are delivered early, so the merge of a

@@ -128,6 +128,80 @@ def test_repeated_launches_with_many_items_per_cta_are_bit_identical(ctas):
         assert torch.equal(out, out0) and torch.equal(lse, lse0), f"repeat {rep} differs"
 
 
+@pytest.mark.parametrize("ctas", [1, 3])
+def test_repeated_fused_steps_with_many_items_per_cta_are_bit_identical(ctas):
+    """The same stress through odma_decode_step with the append fused in: the query slots then
+    also carry each stream's new K/V rows.  The step is repeated without committing lengths, so
+    every repeat appends the same rows at the same place and must give the same bits."""
+    odma = lib()
+    w = qwen_small([L - 1 for L in RAGGED])
+    w = wl.scaled(w, predicted=w.context + 8)
+    s = Session(w, plan_ctas=ctas)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    pre = [r for r in reqs if w.context[r] > 0]
+    s.append(pre, [int(w.context[r]) for r in pre])
+    for r in reqs:
+        s.ls.ensure(r, s.lens[r] + 1)
+    q = s.queries(0, reqs, w.q_heads, 0).contiguous()
+    kn = torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+    vn = torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+    out0 = None
+    for rep in range(25):
+        out = torch.full_like(q, float("nan"))
+        s.pool.decode_step(0, 1, w.q_heads, reqs, q.data_ptr(), kn.data_ptr(), vn.data_ptr(), out.data_ptr(), 0, s.stream)
+        torch.cuda.synchronize()
+        assert s.pool.check_status(s.stream) == odma.OK
+        if out0 is None:
+            out0 = out
+            for i, r in enumerate(reqs):
+                s.kv.append(r, 0, kn[i:i + 1], vn[i:i + 1])
+            ref, _, _ = s.oracle_out(0, reqs, q, w.q_heads)
+            assert_close(out0, ref, w.dtype, f"fused step, many items per CTA, ctas={ctas}")
+        else:
+            assert torch.equal(out, out0), f"repeat {rep} differs"
+    s.ls.commit(reqs, 1)
+    for r in reqs:
+        s.lens[r] += 1
+        k_ref, v_ref = s.kv.gathered(r, 0)
+        assert np.array_equal(s.pool_rows(0, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+        assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+
+
+def test_migration_copy_then_fused_step_without_a_host_sync():
+    """A request outgrows its slab: the migration copy and the decode step that reads the
+    copied rows are enqueued back to back.  The decode kernel must not read slab rows before the
+    copy kernel ahead of it has completed (it may only do so behind another decode kernel)."""
+    odma = lib()
+    lens = [63, 64, 200, 1024]
+    w = qwen_small(lens)
+    w = wl.scaled(w, predicted=w.context)            # slabs exactly full: 64 and 1024 overflow on the next token
+    s = Session(w, plan_ctas=4)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    s.append(reqs, [int(c) for c in w.context])
+    q = s.queries(0, reqs, w.q_heads, 0).contiguous()
+    kn = torch.cat([s.rows(0, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+    vn = torch.cat([s.rows(0, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]).contiguous()
+    out = torch.full_like(q, float("nan"))
+    torch.cuda.synchronize()
+    migrated = sum(s.ls.ensure(r, s.lens[r] + 1)[1] for r in reqs)     # launches the copies, no sync
+    s.pool.decode_step(0, 1, w.q_heads, reqs, q.data_ptr(), kn.data_ptr(), vn.data_ptr(), out.data_ptr(), 0, s.stream)
+    torch.cuda.synchronize()
+    assert migrated == 2 and s.pool.check_status(s.stream) == odma.OK
+    s.ls.commit(reqs, 1)
+    for i, r in enumerate(reqs):
+        s.kv.append(r, 0, kn[i:i + 1], vn[i:i + 1])
+        s.lens[r] += 1
+    ref, _, _ = s.oracle_out(0, reqs, q, w.q_heads)
+    assert_close(out, ref, w.dtype, "migration then fused step")
+    for r in reqs:
+        k_ref, v_ref = s.kv.gathered(r, 0)
+        assert np.array_equal(s.pool_rows(0, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+
+
 def test_fused_and_separate_combine_agree_bit_for_bit():
     w = qwen_small([L - 1 for L in RAGGED] + [4000])
     outs = []

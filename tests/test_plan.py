@@ -169,3 +169,32 @@ def test_a_decode_step_plan_is_reused_while_the_batch_only_grows_a_little():
     items = cover(t, np.array(words, dtype=np.int64), cur)
     row0 = items[(items[:, 0] == 0) & (items[:, 1] == 0) & (items[:, 2] == 0)][0, 6]
     assert row0 == slab2[0] * hkv
+
+
+def test_plan_never_outgrows_the_table_it_was_sized_for():
+    """Random length mixes and CTA counts: the words a plan writes stay within
+    odma_tables_bytes (items <= streams + ctas, cut streams <= min(streams, ctas))."""
+    rng = np.random.default_rng(5)
+    odma = lib()
+    for trial in range(300):
+        n = int(rng.integers(1, 40))
+        ctas = int(rng.integers(1, 200))
+        kind = trial % 3
+        if kind == 0:
+            lens = rng.integers(1, 200, size=n)
+        elif kind == 1:
+            lens = np.clip(np.rint(np.exp(rng.normal(6, 1.2, size=n))), 1, 16000).astype(int)
+        else:
+            lens = rng.choice([1, 63, 64, 65, 4096, 16000], size=n)
+        w = wl.scaled(wl.config1("a"), pool_bytes=1 << 30, max_len=16384, context=np.asarray(lens, dtype=np.int64),
+                      predicted=np.asarray(lens, dtype=np.int64) + 1)
+        pool = host_pool(w, plan_ctas=ctas, max_batch=64)
+        assert pool.set_buckets([16384]) == 0
+        reqs = list(range(n))
+        for r in reqs:
+            assert pool.alloc(r, int(lens[r]) + 1)[0] == 0
+            assert pool.commit_step([r], [int(lens[r])]) == 0
+        rc, t, words = pool.plan_host(reqs)
+        assert rc == 0
+        assert t.words * 4 <= pool.tables_bytes(n)
+        assert t.n_items <= n * w.kv_heads + ctas and t.n_combine <= min(n * w.kv_heads, ctas)
