@@ -316,6 +316,47 @@ int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const o
 int32_t odma_profile_enable(odma_pool* pool, int32_t on);
 int32_t odma_profile_read(odma_pool* pool, int32_t kernel, double* total_ms, int64_t* launches);
 
+/* ---- admission / serving simulator (the paper's evaluation protocol, Section V: Poisson
+ *      arrivals into one KV pool; KV-cache utilisation = actual / reserved; throughput in
+ *      output tokens per second) ----------------------------------------------------------------
+ * Host only.  One model replica decodes in lock step over the pool; `reqs` (host, n entries,
+ * arrival times non-decreasing) are admitted first come first served under one of three
+ * reservation policies: ODMA_SIM_STATIC reserves max_len tokens per request (the static
+ * worst-case baseline), ODMA_SIM_PAGED16 takes 16-token pages on demand (PagedAttention
+ * accounting), ODMA_SIM_ODMA drives this pool's own allocator (odma_alloc, or
+ * odma_alloc_uncertain when u_permille >= 0; odma_ensure_capacity with allocate-and-copy
+ * migration; odma_free with boundary recalibration).  `pool` must be a pool without live
+ * requests; a bookkeeping-only pool (dev_base NULL) is enough, no kernel is launched.
+ * Rules: time in integer nanoseconds; the prompt is in place at admission; a decode step lasts
+ * layers * (base_ns + kv_tokens * ps_per_token / 1000) with kv_tokens the keys attended by the
+ * requests that generate in that step (fit base_ns and ps_per_token to measured launches);
+ * admission stops at the first request that does not fit, at max_batch live requests, or at
+ * one that has not arrived (with nobody live the clock jumps to the next arrival); a request
+ * without room for its next token stalls for the step; when all stall, the youngest is
+ * preempted (progress lost, back to the head of the queue) and nothing is admitted until a
+ * live request completes; a request that cannot be placed in an empty pool, or stalls alone,
+ * is dropped (failed).  Results are sums; utilisation = sum_actual / sum_reserved (capacity
+ * held at completion), time-averaged utilisation = used_time / reserved_time, mean
+ * concurrency = conc_time / makespan_ns, tokens per second = tokens_out / makespan_ns * 1e9. */
+enum { ODMA_SIM_STATIC = 0, ODMA_SIM_PAGED16 = 1, ODMA_SIM_ODMA = 2 };
+typedef struct odma_sim_request {
+    int64_t arrival_ns;
+    int32_t prompt;      /* KV tokens present at admission (>= 1) */
+    int32_t total;       /* KV tokens at completion (> prompt) */
+    int32_t predicted;   /* predicted total, as given to the allocator */
+    int32_t u_permille;  /* predictor uncertainty in thousandths, -1: none */
+} odma_sim_request;
+typedef struct odma_sim_params {
+    int32_t policy, max_batch, layers, reserved;
+    int64_t base_ns, ps_per_token;
+} odma_sim_params;
+typedef struct odma_sim_result {
+    int64_t completed, failed, tokens_out, tokens_lost, steps, makespan_ns, sum_actual, sum_reserved,
+        conc_time, reserved_time, used_time, migrations, preemptions, stalls, deferred;
+} odma_sim_result;
+int32_t odma_sim_run(odma_pool* pool, const odma_sim_params* params, const odma_sim_request* reqs,
+                     int32_t n, odma_sim_result* out);
+
 /* ---- page-16 ablation (paging is the layout the paper argues against, Sections I, II-A) --
  * The same requests re-laid in 16-token pages: page p of (array a, head) is 16 rows at
  * ((a*n_pages + p)*kv_heads + head)*16 of the caller's buffer d_pages.  odma_paged_build

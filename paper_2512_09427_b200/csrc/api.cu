@@ -15,6 +15,11 @@
 
 using namespace odma;
 
+namespace odma {
+int32_t simulate(Allocator& alloc, const odma_sim_params& prm, const odma_sim_request* reqs, int32_t n,
+                 odma_sim_result* out);      // simulator.cpp
+}
+
 namespace {
 
 constexpr int kStagingSlots = 4;
@@ -1005,6 +1010,16 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
         if (e != cudaSuccess) return ODMA_ERR_CUDA;
     }
     return ODMA_OK;
+}
+
+int32_t odma_sim_run(odma_pool* pool, const odma_sim_params* params, const odma_sim_request* reqs, int32_t n,
+                     odma_sim_result* out) {
+    if (!pool || !params) return ODMA_ERR_INVALID;
+    odma_stats st;
+    pool->alloc.stats(&st);
+    if (st.live != 0) return ODMA_ERR_INVALID;
+    pool->plan_cache.valid = false;
+    return simulate(pool->alloc, *params, reqs, n, out);
 }
 
 }  // extern "C"

@@ -62,6 +62,27 @@ class Tables(C.Structure):
                [("kv_tokens", C.c_int64), ("epoch", C.c_uint64)]
 
 
+class SimRequest(C.Structure):
+    _fields_ = [("arrival_ns", C.c_int64), ("prompt", C.c_int32), ("total", C.c_int32), ("predicted", C.c_int32),
+                ("u_permille", C.c_int32)]
+
+
+class SimParams(C.Structure):
+    _fields_ = [("policy", C.c_int32), ("max_batch", C.c_int32), ("layers", C.c_int32), ("reserved", C.c_int32),
+                ("base_ns", C.c_int64), ("ps_per_token", C.c_int64)]
+
+
+class SimResult(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in
+                ("completed", "failed", "tokens_out", "tokens_lost", "steps", "makespan_ns", "sum_actual", "sum_reserved",
+                 "conc_time", "reserved_time", "used_time", "migrations", "preemptions", "stalls", "deferred")]
+
+    def asdict(self):
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+SIM_STATIC, SIM_PAGED16, SIM_ODMA = 0, 1, 2
+
 _vp, _i32, _u64, _i64 = C.c_void_p, C.c_int32, C.c_uint64, C.c_int64
 _i32p, _u64p = C.POINTER(C.c_int32), C.POINTER(C.c_uint64)
 
@@ -93,6 +114,7 @@ _SIGS = {
     "odma_read_probe": (_i32, [_vp, _i32, _i32, C.POINTER(Tables), _vp]),
     "odma_profile_enable": (_i32, [_vp, _i32]),
     "odma_profile_read": (_i32, [_vp, _i32, C.POINTER(C.c_double), C.POINTER(_i64)]),
+    "odma_sim_run": (_i32, [_vp, C.POINTER(SimParams), C.POINTER(SimRequest), _i32, C.POINTER(SimResult)]),
     "odma_paged_create": (_i32, [_vp, _vp, _u64, C.POINTER(_vp)]),
     "odma_paged_destroy": (_i32, [_vp]),
     "odma_paged_build": (_i32, [_vp, C.POINTER(Tables), _i32p, _u64, _vp, _i32, _vp]),
@@ -257,6 +279,14 @@ class Pool:
 
     def selftest_timeout(self, limit_ms: int, stream: int = 0) -> int:
         return _lib.odma_selftest_timeout(self._h, limit_ms, stream or None)
+
+    def sim_run(self, policy: int, requests, max_batch: int, layers: int, base_ns: int, ps_per_token: int) -> dict:
+        """requests: sequence of (arrival_ns, prompt, total, predicted, u_permille)."""
+        arr = (SimRequest * len(requests))(*[SimRequest(*[int(x) for x in r]) for r in requests])
+        prm = SimParams(policy, max_batch, layers, 0, base_ns, ps_per_token)
+        res = SimResult()
+        _check(_lib.odma_sim_run(self._h, C.byref(prm), arr, len(requests), C.byref(res)), "odma_sim_run")
+        return res.asdict()
 
     def read_probe(self, layer: int, q_heads: int, tables: Tables, stream: int = 0) -> None:
         _check(_lib.odma_read_probe(self._h, layer, q_heads, C.byref(tables), stream or None),

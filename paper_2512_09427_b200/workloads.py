@@ -434,3 +434,37 @@ def run_closed_loop(alloc, total_len: np.ndarray, predicted: np.ndarray, concurr
                     on_epoch(e, list(live), np.asarray(cur, dtype=np.int64))
             admit()
     return res
+
+
+# ---------------------------------------------------------------------------
+# arrival trace for the admission simulator
+# ---------------------------------------------------------------------------
+
+
+def poisson_trace(seed: int, n: int, rate_per_s: float, law: str = "lognormal", noise_sigma: float = 0.3,
+                  max_len: int = 16384, with_uncertainty: bool = False):
+    """n requests arriving by a Poisson process of `rate_per_s`: rows of (arrival_ns, prompt,
+    total, predicted, u_permille).  Totals follow the named length law (the stand-in for the
+    request mix of the paper's evaluation, Section V), the prompt is a quarter of the total,
+    the prediction is the total times a lognormal(0, noise_sigma) error.  With
+    `with_uncertainty` the synthetic predictor also reports an uncertainty u in [0, 1] that
+    grows with its (absolute, relative) error plus noise, so that a large u really does mark
+    the requests whose prediction is poor; otherwise u = -1 (none)."""
+    rng = _rng(seed)
+    if law == "lognormal":
+        total = lognormal_lengths(rng, n, 512, 0.8, 16, min(8192, max_len))
+    elif law == "pareto":
+        total = pareto_lengths(rng, n, 1.5, 32, max_len)
+    else:
+        raise ValueError(law)
+    total = np.maximum(total, 2)
+    prompt = np.clip(total // 4, 1, total - 1)
+    predicted = np.minimum(noisy_prediction(rng, total, noise_sigma), max_len)
+    arrival = np.cumsum(rng.exponential(1e9 / rate_per_s, size=n)).astype(np.int64)
+    if with_uncertainty:
+        rel = np.abs(predicted - total) / total
+        u = np.clip(rel / (3 * noise_sigma) + rng.normal(0, 0.1, size=n), 0, 1)
+        u_pm = np.rint(u * 1000).astype(np.int64)
+    else:
+        u_pm = np.full(n, -1, dtype=np.int64)
+    return [(int(a), int(p), int(t), int(q), int(u)) for a, p, t, q, u in zip(arrival, prompt, total, predicted, u_pm)]
