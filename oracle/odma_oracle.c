@@ -12,6 +12,11 @@
  *   reading KV head h div (Hq/Hkv).
  *   Pins: fp64 library attention, closed forms, invariants, a high-precision
  *   evaluation on tiny inputs (tests/test_oracle_attention.py).
+ *   K and V may also be held as E4M3 codes with a dequantisation scale per layer (an
+ *   8-bit slab): the format is written out from its definition, rounding is a search for
+ *   the nearest code.  Pins: the format's published special values, an independent
+ *   library's widening of all 256 codes and its rounding on 200,000 numbers and every
+ *   midpoint, attention over the dequantised values (tests/test_oracle_e4m3.py).
  *
  * Part 2 - allocator.  One owner entry per token of the pool; every placement is
  *   found by scanning that array.  Steps follow Section III (B: uncertainty
@@ -39,24 +44,85 @@
 /* Part 1: attention                                                          */
 /* ------------------------------------------------------------------------- */
 
-enum { ORA_F32 = 0, ORA_BF16 = 1 };
+enum { ORA_F32 = 0, ORA_BF16 = 1, ORA_E4M3 = 2 };
+
+/*
+ * The 8-bit floating-point format E4M3 (OCP 8-bit floating point specification, the "fn"
+ * variant: no infinities): bit 7 sign, bits 6..3 exponent E (bias 7), bits 2..0 mantissa M.
+ *   E = 0:            value = M * 2^-9                (subnormal; M = 0 is zero)
+ *   E = 15 and M = 7: NaN
+ *   otherwise:        value = (1 + M/8) * 2^(E - 7)   (largest: E = 15, M = 6: 448)
+ */
+static double e4m3_value(uint8_t code) {
+    int e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    v = e == 0 ? ldexp((double)m, -9) : ldexp(1.0 + m / 8.0, e - 7);
+    return (code & 0x80) ? -v : v;
+}
+
+/*
+ * Nearest E4M3 code of a finite fp32 number by the definition of rounding: of all finite
+ * codes, the one whose value is closest (distances are exact in fp64); of two equally
+ * close ones the one with an even code (round to nearest even: neighbouring magnitudes are
+ * consecutive codes); anything beyond +-448 saturates to +-448.  NaN gives the NaN code.
+ */
+static uint8_t e4m3_nearest(float y) {
+    double a = fabs((double)y), best_d = INFINITY;
+    int best = 0;
+    uint8_t sign = signbit(y) ? 0x80 : 0;
+    if (isnan(y)) return (uint8_t)(sign | 0x7F);
+    for (int c = 0; c <= 0x7E; ++c) {
+        double d = fabs(a - e4m3_value((uint8_t)c));
+        if (d < best_d || (d == best_d && (c & 1) == 0)) {
+            best_d = d;
+            best = c;
+        }
+    }
+    return (uint8_t)(sign | best);
+}
 
 /* Widen one stored element to fp64.  bf16 is the upper half of an fp32. */
 static double widen(const void* p, size_t i, int dtype) {
     if (dtype == ORA_F32) return (double)((const float*)p)[i];
+    if (dtype == ORA_E4M3) return e4m3_value(((const uint8_t*)p)[i]);
     uint32_t bits = (uint32_t)((const uint16_t*)p)[i] << 16;
     float f;
     memcpy(&f, &bits, sizeof f);
     return (double)f;
 }
 
+void oracle_e4m3_widen(const uint8_t* codes, size_t n, double* out) {
+    for (size_t i = 0; i < n; ++i) out[i] = e4m3_value(codes[i]);
+}
+
+void oracle_e4m3_round(const float* x, size_t n, uint8_t* codes) {
+    for (size_t i = 0; i < n; ++i) codes[i] = e4m3_nearest(x[i]);
+}
+
 /*
- * One (request, query head).  q: [Hq][D].  K, V: [L][Hkv][D], token-major (the
- * checker's own store; it never sees the device layout).  out: [D].  weights (may
- * be NULL): [L] softmax weights.  Returns the log-sum-exp of the scaled scores.
+ * What an append into an E4M3 slab stores: the row's elements (fp32 or bf16, as given)
+ * widened to fp32, multiplied IN FP32 by inv_scale (the caller's fp32 reciprocal of the
+ * dequantisation scale; one rounding, the precision the GPU path takes the same decision
+ * in), rounded to the nearest code.
  */
-static double attention_head(const void* q, const void* K, const void* V, int L, int h, int Hq,
-                             int Hkv, int D, int dtype, double* out, double* weights) {
+void oracle_e4m3_quantize(const void* x, int dtype, size_t n, float inv_scale, uint8_t* codes) {
+    for (size_t i = 0; i < n; ++i) {
+        volatile float y = (float)widen(x, i, dtype) * inv_scale;
+        codes[i] = e4m3_nearest(y);
+    }
+}
+
+/*
+ * One (request, query head).  q: [Hq][D] of type qdtype.  K, V: [L][Hkv][D] of type kvdtype,
+ * token-major (the checker's own store; it never sees the device layout); a stored key
+ * element stands for widen(K) * k_scale, a value element for widen(V) * v_scale (both 1 for
+ * fp32 and bf16 stores; the per-layer dequantisation scales of an E4M3 store).  out: [D].
+ * weights (may be NULL): [L] softmax weights.  Returns the log-sum-exp of the scaled scores.
+ */
+static double attention_head(const void* q, int qdtype, const void* K, const void* V, int kvdtype,
+                             double k_scale, double v_scale, int L, int h, int Hq, int Hkv, int D,
+                             double* out, double* weights) {
     int group = Hq / Hkv;
     int kappa = h / group;
     double* s = (double*)malloc(sizeof(double) * (size_t)L);
@@ -64,8 +130,8 @@ static double attention_head(const void* q, const void* K, const void* V, int L,
     for (int j = 0; j < L; ++j) {
         double dot = 0.0;
         for (int d = 0; d < D; ++d)
-            dot += widen(q, (size_t)h * D + d, dtype) *
-                   widen(K, ((size_t)j * Hkv + kappa) * D + d, dtype);
+            dot += widen(q, (size_t)h * D + d, qdtype) *
+                   (widen(K, ((size_t)j * Hkv + kappa) * D + d, kvdtype) * k_scale);
         s[j] = dot / sqrt((double)D);
         if (s[j] > mx) mx = s[j];
     }
@@ -75,7 +141,8 @@ static double attention_head(const void* q, const void* K, const void* V, int L,
     for (int j = 0; j < L; ++j) {
         double p = exp(s[j] - mx) / sum;
         if (weights) weights[j] = p;
-        for (int d = 0; d < D; ++d) out[d] += p * widen(V, ((size_t)j * Hkv + kappa) * D + d, dtype);
+        for (int d = 0; d < D; ++d)
+            out[d] += p * (widen(V, ((size_t)j * Hkv + kappa) * D + d, kvdtype) * v_scale);
     }
     free(s);
     return mx + log(sum);
@@ -86,10 +153,10 @@ static double attention_head(const void* q, const void* K, const void* V, int L,
  * out: [n][Hq][D] fp64; lse: [n][Hq] fp64 or NULL.  Work is spread over
  * (request, head) pairs; returns the number of threads used.
  */
-int oracle_decode_attention(int n, const void* q, const void* const* K, const void* const* V,
-                            const int32_t* L, int Hq, int Hkv, int D, int dtype, double* out,
-                            double* lse, int threads) {
-    size_t esz = dtype == ORA_F32 ? 4 : 2;
+static int attention_batch(int n, const void* q, int qdtype, const void* const* K, const void* const* V,
+                           int kvdtype, double k_scale, double v_scale, const int32_t* L, int Hq, int Hkv,
+                           int D, double* out, double* lse, int threads) {
+    size_t esz = qdtype == ORA_F32 ? 4 : 2;
     int used = 1;
 #ifdef _OPENMP
     if (threads > 0) omp_set_num_threads(threads);
@@ -103,17 +170,31 @@ int oracle_decode_attention(int n, const void* q, const void* const* K, const vo
     for (int w = 0; w < n * Hq; ++w) {
         int i = w / Hq, h = w % Hq;
         const char* qi = (const char*)q + (size_t)i * Hq * D * esz;
-        double l = attention_head(qi, K[i], V[i], L[i], h, Hq, Hkv, D, dtype,
+        double l = attention_head(qi, qdtype, K[i], V[i], kvdtype, k_scale, v_scale, L[i], h, Hq, Hkv, D,
                                   out + ((size_t)i * Hq + h) * D, NULL);
         if (lse) lse[(size_t)i * Hq + h] = l;
     }
     return used;
 }
 
+int oracle_decode_attention(int n, const void* q, const void* const* K, const void* const* V,
+                            const int32_t* L, int Hq, int Hkv, int D, int dtype, double* out,
+                            double* lse, int threads) {
+    return attention_batch(n, q, dtype, K, V, dtype, 1.0, 1.0, L, Hq, Hkv, D, out, lse, threads);
+}
+
+/* The same with K and V held as E4M3 codes (one byte per element) and their scales. */
+int oracle_decode_attention_e4m3(int n, const void* q, int qdtype, const void* const* K,
+                                 const void* const* V, float k_scale, float v_scale, const int32_t* L,
+                                 int Hq, int Hkv, int D, double* out, double* lse, int threads) {
+    return attention_batch(n, q, qdtype, K, V, ORA_E4M3, (double)k_scale, (double)v_scale, L, Hq, Hkv, D,
+                           out, lse, threads);
+}
+
 /* Softmax weights of one (request, head), for the invariants tests. */
 double oracle_attention_weights(const void* q, const void* K, const void* V, int L, int h, int Hq,
                                 int Hkv, int D, int dtype, double* out, double* weights) {
-    return attention_head(q, K, V, L, h, Hq, Hkv, D, dtype, out, weights);
+    return attention_head(q, dtype, K, V, dtype, 1.0, 1.0, L, h, Hq, Hkv, D, out, weights);
 }
 
 /*

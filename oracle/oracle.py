@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "odma_oracle.c")
 _LIB = os.path.join(_HERE, "libodma_oracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, E4M3 = 0, 1, 2
 
 OK, ERR_INVALID, ERR_NOMEM, ERR_UNKNOWN_REQ, ERR_DUP_REQ, ERR_OVERFLOW = range(6)
 
@@ -52,6 +52,16 @@ def lib():
         L.oracle_attention_chunked.restype = None
         L.oracle_attention_chunked.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                                C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, dp]
+        L.oracle_decode_attention_e4m3.restype = C.c_int
+        L.oracle_decode_attention_e4m3.argtypes = [C.c_int, C.c_void_p, C.c_int, C.POINTER(C.c_void_p),
+                                                   C.POINTER(C.c_void_p), C.c_float, C.c_float, i32p, C.c_int,
+                                                   C.c_int, C.c_int, dp, dp, C.c_int]
+        L.oracle_e4m3_widen.restype = None
+        L.oracle_e4m3_widen.argtypes = [C.c_void_p, C.c_size_t, dp]
+        L.oracle_e4m3_round.restype = None
+        L.oracle_e4m3_round.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+        L.oracle_e4m3_quantize.restype = None
+        L.oracle_e4m3_quantize.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_float, C.c_void_p]
         L.ora_create.restype = C.c_void_p
         L.ora_create.argtypes = [C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64,
                                  C.c_int64, C.c_int64, C.c_int64, C.c_int, i32p, C.c_int32, C.c_int,
@@ -125,6 +135,56 @@ def decode_attention(q, K: Sequence, V: Sequence, q_heads: int, kv_heads: int, h
     return out, lse, used
 
 
+def e4m3_widen(codes) -> np.ndarray:
+    """The values (float64) of an array of E4M3 codes (uint8)."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(c.shape, dtype=np.float64)
+    lib().oracle_e4m3_widen(c.ctypes.data, c.size, out.ctypes.data_as(C.POINTER(C.c_double)))
+    return out
+
+
+def e4m3_round(x) -> np.ndarray:
+    """Nearest E4M3 code (ties to even, saturating at +-448) of each float32."""
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(a.shape, dtype=np.uint8)
+    lib().oracle_e4m3_round(a.ctypes.data, a.size, out.ctypes.data)
+    return out
+
+
+def inv_scale(scale: float) -> np.float32:
+    """The fp32 reciprocal an append multiplies by: 1 / scale, both in fp32, correctly rounded."""
+    return np.float32(1.0) / np.float32(scale)
+
+
+def e4m3_quantize(x, dtype: int, scale: float) -> np.ndarray:
+    """Codes an append of `x` (fp32 / bf16 rows) stores in an E4M3 slab with dequantisation scale `scale`."""
+    a = _as_store(x, dtype)
+    out = np.empty(a.shape, dtype=np.uint8)
+    lib().oracle_e4m3_quantize(a.ctypes.data, dtype, a.size, C.c_float(float(inv_scale(scale))), out.ctypes.data)
+    return out
+
+
+def decode_attention_e4m3(q, qdtype: int, K: Sequence, V: Sequence, k_scale: float, v_scale: float,
+                          q_heads: int, kv_heads: int, head_dim: int, threads: int = 0, want_lse: bool = False):
+    """Dense fp64 attention with K[i], V[i] as E4M3 code arrays [L_i, Hkv, D] (uint8) and their scales."""
+    L = lib()
+    qa = _as_store(q, qdtype)
+    n = qa.shape[0]
+    Ks = [np.ascontiguousarray(k, dtype=np.uint8) for k in K]
+    Vs = [np.ascontiguousarray(v, dtype=np.uint8) for v in V]
+    lens = np.array([k.shape[0] for k in Ks], dtype=np.int32)
+    kp = (C.c_void_p * n)(*[k.ctypes.data for k in Ks])
+    vp = (C.c_void_p * n)(*[v.ctypes.data for v in Vs])
+    out = np.empty((n, q_heads, head_dim), dtype=np.float64)
+    lse = np.empty((n, q_heads), dtype=np.float64) if want_lse else None
+    used = L.oracle_decode_attention_e4m3(
+        n, qa.ctypes.data, qdtype, kp, vp, C.c_float(float(np.float32(k_scale))), C.c_float(float(np.float32(v_scale))),
+        lens.ctypes.data_as(C.POINTER(C.c_int32)), q_heads, kv_heads, head_dim,
+        out.ctypes.data_as(C.POINTER(C.c_double)), lse.ctypes.data_as(C.POINTER(C.c_double)) if want_lse else None,
+        threads)
+    return out, lse, used
+
+
 def attention_weights(q, K, V, h: int, q_heads: int, kv_heads: int, head_dim: int, dtype: int):
     """(out [D], weights [L], lse) of one request and one query head."""
     L = lib()
@@ -153,13 +213,23 @@ def attention_chunked(q, K, V, h: int, q_heads: int, kv_heads: int, head_dim: in
 class KVStore:
     """The checker's own KV cache: per (request, layer) the rows appended so far, in order."""
 
-    def __init__(self, layers: int, kv_heads: int, head_dim: int, dtype: int):
+    def __init__(self, layers: int, kv_heads: int, head_dim: int, dtype: int, kv_e4m3: bool = False,
+                 k_scale: Optional[Sequence[float]] = None, v_scale: Optional[Sequence[float]] = None):
+        """`dtype`: the type of q and of the rows given to append.  With `kv_e4m3` the store holds
+        E4M3 codes, quantised at append with the layer's scale (k_scale[l], v_scale[l]; default 1)."""
         self.layers, self.kv_heads, self.head_dim, self.dtype = layers, kv_heads, head_dim, dtype
+        self.kv_e4m3 = kv_e4m3
+        self.k_scale = [float(x) for x in (k_scale if k_scale is not None else [1.0] * layers)]
+        self.v_scale = [float(x) for x in (v_scale if v_scale is not None else [1.0] * layers)]
         self.k: Dict[Tuple[int, int], List[np.ndarray]] = {}
         self.v: Dict[Tuple[int, int], List[np.ndarray]] = {}
 
     def append(self, req: int, layer: int, k_rows, v_rows) -> None:
         """k_rows, v_rows: [n_tok, Hkv, D]."""
+        if self.kv_e4m3:
+            self.k.setdefault((req, layer), []).append(e4m3_quantize(k_rows, self.dtype, self.k_scale[layer]))
+            self.v.setdefault((req, layer), []).append(e4m3_quantize(v_rows, self.dtype, self.v_scale[layer]))
+            return
         self.k.setdefault((req, layer), []).append(_as_store(k_rows, self.dtype).copy())
         self.v.setdefault((req, layer), []).append(_as_store(v_rows, self.dtype).copy())
 
@@ -180,6 +250,9 @@ class KVStore:
     def decode_attention(self, layer: int, reqs: Sequence[int], q, q_heads: int, threads: int = 0,
                          want_lse: bool = False):
         Ks, Vs = zip(*[self.gathered(r, layer) for r in reqs])
+        if self.kv_e4m3:
+            return decode_attention_e4m3(q, self.dtype, Ks, Vs, self.k_scale[layer], self.v_scale[layer], q_heads,
+                                         self.kv_heads, self.head_dim, threads, want_lse)
         return decode_attention(q, Ks, Vs, q_heads, self.kv_heads, self.head_dim, self.dtype,
                                 threads, want_lse)
 
