@@ -48,18 +48,20 @@ MIN_TIMED_SECONDS = 0.5      # the K-step region is repeated until this much dev
 # workload set-up through the C ABI (no checker code on this path)
 # ---------------------------------------------------------------------------------------------
 
-def pick_workload(name: str, rank: int = 0, copies_override: int = 0, layers_override: int = 0):
+def pick_workload(name: str, rank: int = 0, copies_override: int = 0, layers_override: int = 0, kv_dtype: str = "bf16"):
     """Returns (workload, layers stepped per step, number of rotating KV copies).
 
     config2 is one layer; the pool is given several `layers`, each an independent copy of the
     single-layer cache, and consecutive steps rotate over them so that no step finds its KV in
     L2 (one copy is ~90 MB, L2 is 126 MB).  config3/config5 step through all their layers,
     which together are far larger than L2; `layers_override` keeps only that many of them (same
-    per-layer sizes, pool shrunk in proportion) for captures that must stay small."""
+    per-layer sizes, pool shrunk in proportion) for captures that must stay small.
+    `kv_dtype` "e4m3": the same requests on 8-bit slabs (half the KV bytes per token)."""
     seed_off = 1000 * rank
+    esz = 1 if kv_dtype == "e4m3" else 2
     if name == "config2":
         base = wl.config2(seed=950902 + seed_off)
-        kv_bytes = int((base.context + 1).sum()) * 2 * base.kv_heads * base.head_dim * 2
+        kv_bytes = int((base.context + 1).sum()) * 2 * base.kv_heads * base.head_dim * esz
         copies = copies_override or max(4, -(-3 * L2_BYTES // kv_bytes))
         w = wl.config2(layers=copies, seed=950902 + seed_off)
         step_layers = 1
@@ -74,6 +76,8 @@ def pick_workload(name: str, rank: int = 0, copies_override: int = 0, layers_ove
     if layers_override and name != "config2" and layers_override < w.layers:
         w = wl.scaled(w, layers=layers_override, pool_bytes=w.pool_bytes * layers_override // w.layers)
         step_layers = layers_override
+    if kv_dtype == "e4m3":
+        w = wl.with_e4m3(w)
     return w, step_layers, copies
 
 
@@ -152,7 +156,8 @@ class SlabDecode:
                  fused: int = 1, decode_kernel: int = 0):
         from paper_2512_09427_b200 import odma
         self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
-        self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
+        self.dt = (odma.DTYPE_FP8_E4M3 if w.kv_dtype == "e4m3" else
+                   odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32)
         cfg = odma.config_default()
         cfg.safety_pct, cfg.max_len, cfg.granule = w.safety_pct, w.max_len, w.granule
         cfg.window, cfg.refresh = w.window, w.refresh
@@ -170,6 +175,8 @@ class SlabDecode:
         self.stream = torch.cuda.current_stream().cuda_stream
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
                               self.dt, cfg)
+        if w.kv_dtype == "e4m3":
+            self.pool.set_kv_scales(*wl.e4m3_scales(w.layers))
         self.reqs = list(range(w.batch))
         self.reqs_c = (C.c_uint64 * w.batch)(*self.reqs)
         self.zeros_c = (C.c_int32 * w.batch)()
@@ -366,7 +373,8 @@ def checker_time_step(w: wl.Workload, m: int, step_layers: int):
     code = ora.dtype_code(w.dtype)
     reqs = list(range(m))
     q, Ks, Vs = _host_batch(w, reqs)
-    store = ora.KVStore(1, w.kv_heads, w.head_dim, code)
+    ks, vs = wl.e4m3_scales(1)
+    store = ora.KVStore(1, w.kv_heads, w.head_dim, code, kv_e4m3=w.kv_dtype == "e4m3", k_scale=ks, v_scale=vs)
     for r, k, v in zip(reqs, Ks, Vs):
         store.append(r, 0, k[:-1], v[:-1])
         store.gathered(r, 0)
@@ -384,7 +392,7 @@ def run_reference(args):
     if rank != 0:
         return
     total = args.steps + args.warmup
-    w, step_layers, copies = pick_workload(args.workload)
+    w, step_layers, copies = pick_workload(args.workload, kv_dtype=args.kv_dtype)
     per_step_budget = max(0.02, min(15.0, 150.0 / max(total, 1)))
     m, _ = checker_sample(w, step_layers, per_step_budget)
     times, threads = [], 0
@@ -418,6 +426,8 @@ def workload_config(w, name, step_layers, copies):
                        "noisy predictions, 10% safety pool",
             "config5": "configs[4]: long-reasoning decode, batch 32, contexts U[16384,32768], 28 layers"}[name]
     kv_bytes_layer = int((w.context + 1).sum()) * 2 * w.kv_heads * w.head_dim * w.elem_bytes
+    if w.kv_dtype == "e4m3":
+        desc += "; K/V slabs held as E4M3 codes with per-layer scales (q, new rows and output bf16)"
     return {"workload": desc, "batch": w.batch, "layers_per_step": step_layers,
             "kv_tokens": int((w.context + 1).sum()), "kv_bytes_per_layer": kv_bytes_layer,
             "l2": (f"steps rotate over {copies} independent KV copies ({copies * kv_bytes_layer >> 20} MiB > L2)"
@@ -480,7 +490,9 @@ def run_ours(args):
 
     phases = set(args.phases.split(","))
     K, W = args.steps, args.warmup
-    w, step_layers, copies = pick_workload(args.workload, rank, args.copies, args.layers)
+    w, step_layers, copies = pick_workload(args.workload, rank, args.copies, args.layers, args.kv_dtype)
+    if w.kv_dtype == "e4m3":
+        phases -= {"probe", "paged"}          # both exist for 16-bit slabs only
     sd = SlabDecode(w, step_layers, dev, fused=args.fused_combine, decode_kernel=DECODE_KERNELS[args.decode_kernel])
     bounds, epoch = sd.learn_boundaries()
     sd.admit_and_fill()
@@ -491,7 +503,8 @@ def run_ours(args):
     tables = odma.Tables()
     clocks = ClockSampler(local) if "clocks" in phases else None
     peak, peak_kind = measured_peak()
-    row_bytes = w.head_dim * w.elem_bytes
+    row_bytes = w.head_dim * w.elem_bytes             # of a stored K/V row
+    io_row_bytes = w.head_dim * (4 if w.dtype == torch.float32 else 2)
     n = w.batch
     step_no = 0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -533,10 +546,10 @@ def run_ours(args):
     launches_per_step = step_layers * (1 + (0 if fused_append else 1) +
                                        (1 if tables.n_combine > 0 and not args.fused_combine else 0))
     kv_bytes_per_launch = tables.kv_tokens * 2 * w.kv_heads * row_bytes
-    step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes)
+    step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * io_row_bytes + 2 * n * w.kv_heads * io_row_bytes)
     if w.dtype != torch.bfloat16:
         kernel_name = "decode_generic_kernel"
-    elif args.decode_kernel == "tcgen05" or (args.decode_kernel == "auto" and step_layers > 1):
+    elif args.decode_kernel == "tcgen05" or (args.decode_kernel == "auto" and step_layers > 1) or w.kv_dtype == "e4m3":
         kernel_name = "decode_umma_kernel"
     else:
         kernel_name = "decode_tc_kernel"
@@ -665,7 +678,7 @@ def run_ours(args):
     value = world * n * K / (ms * 1e-3)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+            "dtype": "e4m3" if w.kv_dtype == "e4m3" else "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
             "config": workload_config(w, args.workload, step_layers, copies),
             "regions": {"count": n_regions, "steps_each": K, "ms_per_step_min": min(region_ms) / K,
                         "ms_per_step_max": max(region_ms) / K, "timed_seconds": sum(region_ms) * 1e-3},
@@ -674,8 +687,8 @@ def run_ours(args):
             "plan": {"ctas": tables.n_ctas, "items": tables.n_items, "combine": tables.n_combine},
             "buckets": list(bounds), "migrations_at_fill": sd.migrations_at_fill}
     if e2e_ms == e2e_ms:
-        h2d = step_layers * (n * w.q_heads * row_bytes + 2 * n * w.kv_heads * row_bytes + tables.words * 4)
-        d2h = step_layers * n * w.q_heads * row_bytes
+        h2d = step_layers * (n * w.q_heads * io_row_bytes + 2 * n * w.kv_heads * io_row_bytes + tables.words * 4)
+        d2h = step_layers * n * w.q_heads * io_row_bytes
         line["e2e"] = {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                        "ms_per_step": e2e_ms / e2e_steps}
@@ -866,6 +879,8 @@ def main():
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
     ap.add_argument("--decode-kernel", default="auto", choices=list(DECODE_KERNELS),
                     help="which bf16 decode kernel the pool runs (auto: the library's choice per shape)")
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "e4m3"],
+                    help="element type of the slabs: bf16 (the configs as stated) or E4M3 codes with per-layer scales")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
     ap.add_argument("--layers", type=int, default=0,
                     help="config3/config5: step through this many layers only (0 = all 28; a reduced size for profiler "

@@ -62,7 +62,13 @@ enum {
     ODMA_ERR_TOO_LARGE = 8    /* odma_decode_attention_static: batch beyond its fixed scratch */
 };
 
-enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1 };
+/* Element type of the pool's K/V rows.  ODMA_DTYPE_FP8_E4M3: one byte per element in the OCP
+ * 8-bit floating-point format E4M3 (no infinities, largest value 448) with one fp32
+ * dequantisation scale per layer for K and one for V (odma_set_kv_scales); queries, the rows
+ * given to an append and the output are bf16 ("io type": bf16 for BF16 and FP8_E4M3 pools,
+ * fp32 for F32 pools).  An 8-bit pool needs head_dim 128 and at most 8 query heads per KV
+ * head; its decode runs on the tcgen05 kernel only. */
+enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1, ODMA_DTYPE_FP8_E4M3 = 2 };
 
 /* which tensor-core decode kernel a bf16 pool runs (odma_config.decode_kernel) */
 enum { ODMA_DECODE_AUTO = 0, ODMA_DECODE_TCGEN05 = 1, ODMA_DECODE_MMA_SYNC = 2 };
@@ -165,6 +171,15 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
                          int32_t head_dim, int32_t dtype, const odma_config* cfg, odma_pool** out);
 int32_t odma_pool_destroy(odma_pool* pool);
 
+/* Dequantisation scales of an ODMA_DTYPE_FP8_E4M3 pool (the 8-bit variant of the slab layout;
+ * the paper's slabs hold the serving stack's 16-bit cache, Section IV-A): k_scale, v_scale:
+ * host, [layers] fp32, finite and > 0.  A stored code c of layer l stands for value(c) *
+ * scale[l]; an append stores the code nearest (ties to even, saturating at +-448) to
+ * fp32(x) * (1.0f / scale[l]), product and reciprocal taken in fp32.  Default 1 for every
+ * layer.  Takes effect for launches issued after the call; rows already stored keep their
+ * codes.  ODMA_ERR_INVALID for another pool type or a bad scale. */
+int32_t odma_set_kv_scales(odma_pool* pool, const float* k_scale, const float* v_scale);
+
 /* ---- bucket boundaries (Section III-C, Eq. 2) ------------------------------------------
  * Static / initial boundaries: n in [1, ODMA_MAX_BUCKETS], strictly increasing multiples of
  * the granule, none above max_len.  They hold until the next recalibration. */
@@ -221,15 +236,15 @@ int32_t odma_build_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* 
 /* ---- KV append (the per-step growth of each request's cache, Section II-A) --------------
  * Writes the step's new K and V rows of `layer` behind each request's existing tokens:
  * token j of request i goes to slab position len[i] - n_new[i] + j.  k_new, v_new: device,
- * [n_new_total, kv_heads, head_dim] in the pool dtype, requests in table order, 16-byte
- * aligned. */
+ * [n_new_total, kv_heads, head_dim] in the pool's io type, requests in table order, 16-byte
+ * aligned.  An 8-bit pool quantises the rows as odma_set_kv_scales describes. */
 int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables,
                        const void* k_new, const void* v_new, void* stream);
 
 /* ---- decode attention over the slabs (the bandwidth consumer, Sections III-A and V-B) ---
  * out[i][h] = softmax_j(q[i][h] . K_i[h div g][j] / sqrt(head_dim)) V_i[h div g], j < len[i],
- * g = q_heads / kv_heads.  q, out: device, [n, q_heads, head_dim] in the pool dtype, 16-byte
- * aligned; lse: device fp32 [n, q_heads] or NULL (natural-log sum of exp of the scaled
+ * g = q_heads / kv_heads (K_i, V_i of an 8-bit pool: the dequantised values).  q, out: device,
+ * [n, q_heads, head_dim] in the pool's io type, 16-byte aligned; lse: device fp32 [n, q_heads] or NULL (natural-log sum of exp of the scaled
  * scores).  Accumulation and softmax are fp32.  Launches the split kernel and, when some
  * stream was split, the combine kernel. */
 int32_t odma_decode_attention(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,

@@ -62,22 +62,28 @@ static double e4m3_value(uint8_t code) {
 }
 
 /*
- * Nearest E4M3 code of a finite fp32 number by the definition of rounding: of all finite
- * codes, the one whose value is closest (distances are exact in fp64); of two equally
- * close ones the one with an even code (round to nearest even: neighbouring magnitudes are
- * consecutive codes); anything beyond +-448 saturates to +-448.  NaN gives the NaN code.
+ * Nearest E4M3 code of an fp32 number by the definition of rounding.  The magnitudes of
+ * codes 0x00..0x7E increase with the code, so the nearest finite value is one of the two
+ * that enclose |y|: lo = the largest code whose value is <= |y| (found by bisection) and
+ * lo + 1.  Distances are exact in fp64; of two equally close values the one with the even
+ * code (round to nearest even: neighbours are consecutive codes); anything beyond +-448
+ * saturates to +-448.  NaN gives the NaN code.
  */
 static uint8_t e4m3_nearest(float y) {
-    double a = fabs((double)y), best_d = INFINITY;
-    int best = 0;
+    double a = fabs((double)y);
     uint8_t sign = signbit(y) ? 0x80 : 0;
+    int lo = 0, hi = 0x7E, best;
     if (isnan(y)) return (uint8_t)(sign | 0x7F);
-    for (int c = 0; c <= 0x7E; ++c) {
-        double d = fabs(a - e4m3_value((uint8_t)c));
-        if (d < best_d || (d == best_d && (c & 1) == 0)) {
-            best_d = d;
-            best = c;
-        }
+    if (a >= e4m3_value(0x7E)) return (uint8_t)(sign | 0x7E);
+    while (hi - lo > 1) {               /* invariant: value(lo) <= a < value(hi) */
+        int mid = (lo + hi) / 2;
+        if (e4m3_value((uint8_t)mid) <= a) lo = mid; else hi = mid;
+    }
+    {
+        double d_lo = a - e4m3_value((uint8_t)lo), d_hi = e4m3_value((uint8_t)hi) - a;
+        if (d_lo < d_hi) best = lo;
+        else if (d_hi < d_lo) best = hi;
+        else best = (lo & 1) == 0 ? lo : hi;
     }
     return (uint8_t)(sign | best);
 }
@@ -107,8 +113,11 @@ void oracle_e4m3_round(const float* x, size_t n, uint8_t* codes) {
  * in), rounded to the nearest code.
  */
 void oracle_e4m3_quantize(const void* x, int dtype, size_t n, float inv_scale, uint8_t* codes) {
-    for (size_t i = 0; i < n; ++i) {
-        volatile float y = (float)widen(x, i, dtype) * inv_scale;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static)
+#endif
+    for (long long i = 0; i < (long long)n; ++i) {
+        volatile float y = (float)widen(x, (size_t)i, dtype) * inv_scale;
         codes[i] = e4m3_nearest(y);
     }
 }

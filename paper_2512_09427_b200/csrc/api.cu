@@ -43,7 +43,11 @@ struct odma_pool {
     Allocator alloc;
     void* dev_base = nullptr;
     uint64_t bytes = 0;
-    int32_t layers = 0, kv_heads = 0, head_dim = 0, dtype = 0, elem_bytes = 0;
+    int32_t layers = 0, kv_heads = 0, head_dim = 0, dtype = 0;
+    int32_t elem_bytes = 0;     // of a stored K/V element
+    int32_t io_bytes = 0;       // of an element of q, out and the rows given to an append
+    int32_t io_dtype = 0;       // ODMA_DTYPE_F32 or ODMA_DTYPE_BF16
+    std::vector<float> k_scale, v_scale;   // 8-bit pools: dequantisation scale per layer
     int64_t rows_per_array = 0;
     int32_t plan_ctas = 148;
     // The decode kernels start reading slab rows before their dependency wait, on the
@@ -114,9 +118,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
-// Four views of a [rows x head_dim] bf16 row array: boxes of 16, 32, 48 and 64 rows by 64
-// elements (128 bytes, the widest inner extent the 128-byte swizzle allows).
-int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, TensorMaps* out) {
+// Four views of a [rows x head_dim] row array of 2-byte (bf16) or 1-byte (E4M3) elements: boxes of
+// 16, 32, 48 and 64 rows by 128 bytes (the widest inner extent the 128-byte swizzle allows).
+int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, int32_t elem_bytes, TensorMaps* out) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
@@ -124,11 +128,12 @@ int32_t make_tensor_maps(void* base, int64_t rows, int32_t head_dim, TensorMaps*
         return ODMA_ERR_CUDA;
     auto encode = reinterpret_cast<EncodeTiledFn>(fn);
     const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(head_dim) * 2};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(head_dim) * elem_bytes};
     const cuuint32_t estride[2] = {1, 1};
+    const CUtensorMapDataType type = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     for (int k = 0; k < 4; ++k) {
-        const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(16 * (k + 1))};
-        if (encode(&out->box[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estride,
+        const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(16 * (k + 1))};
+        if (encode(&out->box[k], type, 2, base, gdim, gstride, box, estride,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return ODMA_ERR_CUDA;
@@ -329,6 +334,14 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->wait_limit_ns = kDefaultWaitLimitNs;
     p->chained = 0;
     p->early_ok = 0;
+    p->kv_fp8 = pool->dtype == ODMA_DTYPE_FP8_E4M3 ? 1 : 0;
+    p->k_scale = p->v_scale = p->k_inv = p->v_inv = 1.f;
+    if (p->kv_fp8) {
+        p->k_scale = pool->k_scale[layer];
+        p->v_scale = pool->v_scale[layer];
+        p->k_inv = 1.0f / p->k_scale;
+        p->v_inv = 1.0f / p->v_scale;
+    }
 }
 
 int32_t check_decode_args(const odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
@@ -338,6 +351,8 @@ int32_t check_decode_args(const odma_pool* pool, int32_t layer, const void* q, i
         return ODMA_ERR_INVALID;
     if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
     if (q_heads / pool->kv_heads > pool->alloc.config().max_group) return ODMA_ERR_INVALID;
+    if (pool->dtype == ODMA_DTYPE_FP8_E4M3 && !umma_supported(pool->head_dim, q_heads / pool->kv_heads, true))
+        return ODMA_ERR_INVALID;
     return check_tables(pool, t);
 }
 
@@ -387,15 +402,20 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
                          int32_t head_dim, int32_t dtype, const odma_config* cfg_in, odma_pool** out) {
     if (!out) return ODMA_ERR_INVALID;
     *out = nullptr;
-    if (dtype != ODMA_DTYPE_F32 && dtype != ODMA_DTYPE_BF16) return ODMA_ERR_INVALID;
+    if (dtype != ODMA_DTYPE_F32 && dtype != ODMA_DTYPE_BF16 && dtype != ODMA_DTYPE_FP8_E4M3) return ODMA_ERR_INVALID;
     odma_config cfg;
     if (cfg_in) cfg = *cfg_in; else odma_config_default(&cfg);
-    const int32_t esz = dtype == ODMA_DTYPE_F32 ? 4 : 2;
+    const int32_t esz = dtype == ODMA_DTYPE_F32 ? 4 : dtype == ODMA_DTYPE_BF16 ? 2 : 1;
+    const int32_t iosz = dtype == ODMA_DTYPE_F32 ? 4 : 2;
     if (layers < 1 || kv_heads < 1 || head_dim < 1 || (static_cast<int64_t>(head_dim) * esz) % 16 != 0)
         return ODMA_ERR_INVALID;
     if (cfg.max_batch < 1 || cfg.max_group < 1 || cfg.plan_ctas < 0) return ODMA_ERR_INVALID;
     if (cfg.decode_kernel < ODMA_DECODE_AUTO || cfg.decode_kernel > ODMA_DECODE_MMA_SYNC) return ODMA_ERR_INVALID;
     if (dev_base && (reinterpret_cast<uintptr_t>(dev_base) & 255u) != 0) return ODMA_ERR_INVALID;
+    // an 8-bit pool is served by the tcgen05 kernel alone
+    if (dtype == ODMA_DTYPE_FP8_E4M3 &&
+        (!umma_supported(head_dim, 1, true) || cfg.decode_kernel == ODMA_DECODE_MMA_SYNC || cfg.max_group > 8))
+        return ODMA_ERR_INVALID;
 
     odma_pool* p = new (std::nothrow) odma_pool();
     if (!p) return ODMA_ERR_NOMEM;
@@ -411,6 +431,10 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
     p->head_dim = head_dim;
     p->dtype = dtype;
     p->elem_bytes = esz;
+    p->io_bytes = iosz;
+    p->io_dtype = dtype == ODMA_DTYPE_F32 ? ODMA_DTYPE_F32 : ODMA_DTYPE_BF16;
+    p->k_scale.assign(layers, 1.f);
+    p->v_scale.assign(layers, 1.f);
     p->rows_per_array = p->alloc.T() * kv_heads;
     if (p->rows_per_array * layers * 2 >= (int64_t(1) << 31)) {
         delete p;
@@ -431,8 +455,8 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
     if (dev_base) {
         const size_t po = static_cast<size_t>(p->slots_max) * cfg.max_group * head_dim * 4;
         const size_t pm = static_cast<size_t>(p->slots_max) * cfg.max_group * 2 * 4;
-        const size_t qb = static_cast<size_t>(cfg.max_batch) * kv_heads * cfg.max_group * head_dim * esz;
-        const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * esz;
+        const size_t qb = static_cast<size_t>(cfg.max_batch) * kv_heads * cfg.max_group * head_dim * iosz;
+        const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * iosz;
         bool ok = cudaMalloc(&p->part_o, po) == cudaSuccess && cudaMalloc(&p->part_ml, pm) == cudaSuccess &&
                   cudaMalloc(&p->part_o2, po) == cudaSuccess && cudaMalloc(&p->part_ml2, pm) == cudaSuccess &&
                   cudaMalloc(&p->d_counters2, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
@@ -448,8 +472,8 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
             ok = ok && cudaMallocHost(&s.host, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
                  cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) == cudaSuccess;
         }
-        if (ok && dtype == ODMA_DTYPE_BF16 && tc_supported(head_dim, 1)) {
-            ok = make_tensor_maps(dev_base, p->rows_per_array * layers * 2, head_dim, &p->maps) == ODMA_OK;
+        if (ok && ((dtype == ODMA_DTYPE_BF16 && tc_supported(head_dim, 1)) || dtype == ODMA_DTYPE_FP8_E4M3)) {
+            ok = make_tensor_maps(dev_base, p->rows_per_array * layers * 2, head_dim, esz, &p->maps) == ODMA_OK;
             p->has_maps = ok;
         }
         if (!ok) {
@@ -466,6 +490,16 @@ int32_t odma_pool_destroy(odma_pool* pool) {
     if (!pool) return ODMA_ERR_INVALID;
     if (pool->dev_base) free_device_side(pool);
     delete pool;
+    return ODMA_OK;
+}
+
+int32_t odma_set_kv_scales(odma_pool* pool, const float* k_scale, const float* v_scale) {
+    if (!pool || !k_scale || !v_scale || pool->dtype != ODMA_DTYPE_FP8_E4M3) return ODMA_ERR_INVALID;
+    for (int32_t l = 0; l < pool->layers; ++l)
+        if (!(k_scale[l] > 0.f) || !(v_scale[l] > 0.f) || !std::isfinite(k_scale[l]) || !std::isfinite(v_scale[l]))
+            return ODMA_ERR_INVALID;
+    pool->k_scale.assign(k_scale, k_scale + pool->layers);
+    pool->v_scale.assign(v_scale, v_scale + pool->layers);
     return ODMA_OK;
 }
 
@@ -590,6 +624,9 @@ int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables
     ap.n_new_total = tables->n_new_total;
     ap.row_vecs = pool->head_dim * pool->elem_bytes / 16;
     ap.one_new_each = tables->one_new_each;
+    ap.quantize = pool->dtype == ODMA_DTYPE_FP8_E4M3 ? 1 : 0;
+    ap.k_inv = ap.quantize ? 1.0f / pool->k_scale[layer] : 1.f;
+    ap.v_inv = ap.quantize ? 1.0f / pool->v_scale[layer] : 1.f;
     pool->decode_was_last = false;
     ProfScope ps(pool, ODMA_K_APPEND, as_stream(stream));
     return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
@@ -611,7 +648,8 @@ bool uses_tc(const odma_pool* pool, int32_t q_heads) {
 // (3 to 4 % faster there: its last tile and hand-over are a shorter chain).
 bool uses_umma(const odma_pool* pool, int32_t group, bool part_of_multi_layer_step) {
     const int32_t want = pool->alloc.config().decode_kernel;
-    if (want == ODMA_DECODE_MMA_SYNC || !umma_supported(pool->head_dim, group)) return false;
+    if (pool->dtype == ODMA_DTYPE_FP8_E4M3) return true;
+    if (want == ODMA_DECODE_MMA_SYNC || !umma_supported(pool->head_dim, group, false)) return false;
     return want == ODMA_DECODE_TCGEN05 || part_of_multi_layer_step;
 }
 
@@ -670,7 +708,7 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
         e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,
                            pool->part_o, pool->part_ml, out, lse, p.group, pool->head_dim, q_heads,
-                           pool->dtype, as_stream(stream));
+                           pool->io_dtype, as_stream(stream));
         if (e != cudaSuccess) return ODMA_ERR_CUDA;
     }
     return ODMA_OK;
@@ -692,8 +730,8 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
     if (!pool || !pool->dev_base || !d_q || !d_k_new || !d_v_new || !d_out) return ODMA_ERR_INVALID;
     if (n_layers < 1 || layer < 0 || layer + n_layers > pool->layers) return ODMA_ERR_INVALID;
     if (!reqs || n < 1 || n > pool->alloc.config().max_batch) return ODMA_ERR_INVALID;
-    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
-    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->io_bytes;
+    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->io_bytes;
     // on the tensor-core path the append rides in the decode kernel: one launch per layer
     const bool fuse = pool->alloc.config().fused_append && q_heads >= pool->kv_heads &&
                       q_heads % pool->kv_heads == 0 && uses_tc(pool, q_heads) && aligned16(d_k_new) && aligned16(d_v_new);
@@ -755,8 +793,8 @@ int32_t odma_decode_step_host(odma_pool* pool, int32_t layer, int32_t q_heads, c
     if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0 ||
         q_heads / pool->kv_heads > pool->alloc.config().max_group)
         return ODMA_ERR_INVALID;
-    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->elem_bytes;
-    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->elem_bytes;
+    const size_t qb = static_cast<size_t>(n) * q_heads * pool->head_dim * pool->io_bytes;
+    const size_t kb = static_cast<size_t>(n) * pool->kv_heads * pool->head_dim * pool->io_bytes;
     cudaStream_t s = as_stream(stream);
     // Page-locked buffers are addressable from the device: the kernel then takes the queries
     // and the new rows straight from host memory (one bulk copy per stream, issued by the
@@ -794,7 +832,7 @@ int32_t odma_decode_attention_static(const odma_pool* pool, const void* dev_base
     if (layer < 0 || layer >= pool->layers) return ODMA_ERR_INVALID;
     if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
     if (tables->n < 1 || tables->n_items < 1 || tables->n_ctas < 1) return ODMA_ERR_INVALID;
-    if (!generic_supported(pool->head_dim)) return ODMA_ERR_INVALID;
+    if (!generic_supported(pool->head_dim) || pool->dtype == ODMA_DTYPE_FP8_E4M3) return ODMA_ERR_INVALID;
     const int32_t group = q_heads / pool->kv_heads;
     if (tables->n_items > kStaticSlots || group > kStaticGroup || pool->head_dim > kStaticHeadDim)
         return ODMA_ERR_TOO_LARGE;
@@ -828,6 +866,7 @@ int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const o
                         void* stream) {
     if (!pool || !pool->dev_base || !pool->has_maps || layer < 0 || layer >= pool->layers)
         return ODMA_ERR_INVALID;
+    if (pool->dtype != ODMA_DTYPE_BF16) return ODMA_ERR_INVALID;      // the probe is the mma.sync kernel's
     if (q_heads < pool->kv_heads || q_heads % pool->kv_heads != 0) return ODMA_ERR_INVALID;
     int32_t rc = check_tables(pool, tables);
     if (rc != ODMA_OK) return rc;
@@ -887,6 +926,7 @@ int32_t odma_paged_create(odma_pool* pool, void* d_pages, uint64_t bytes, odma_p
     *out = nullptr;
     if (!pool || !pool->dev_base || !d_pages || (reinterpret_cast<uintptr_t>(d_pages) & 255u) != 0)
         return ODMA_ERR_INVALID;
+    if (pool->dtype == ODMA_DTYPE_FP8_E4M3) return ODMA_ERR_INVALID;  // the ablation exists for 16- and 32-bit pools
     const uint64_t page_bytes = static_cast<uint64_t>(pool->layers) * 2u * pool->kv_heads * 16u *
                                 pool->head_dim * pool->elem_bytes;
     const int64_t n_pages = static_cast<int64_t>(bytes / page_bytes);
@@ -899,7 +939,7 @@ int32_t odma_paged_create(odma_pool* pool, void* d_pages, uint64_t bytes, odma_p
     pg->n_pages = n_pages;
     if (pool->has_maps) {
         if (make_tensor_maps(d_pages, n_pages * pool->kv_heads * 16 * pool->layers * 2, pool->head_dim,
-                             &pg->maps) != ODMA_OK) {
+                             pool->elem_bytes, &pg->maps) != ODMA_OK) {
             delete pg;
             return ODMA_ERR_CUDA;
         }
@@ -1006,7 +1046,7 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
         const int32_t* tab = static_cast<const int32_t*>(tables->d_table);
         e = launch_combine(reinterpret_cast<const int4*>(tab + tables->off_combine), tables->n_combine,
                            pool->part_o, pool->part_ml, out, lse, p.group, pool->head_dim, q_heads,
-                           pool->dtype, as_stream(stream));
+                           pool->io_dtype, as_stream(stream));
         if (e != cudaSuccess) return ODMA_ERR_CUDA;
     }
     return ODMA_OK;

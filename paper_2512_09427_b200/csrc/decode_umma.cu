@@ -1,4 +1,5 @@
-// Split decode attention on the fifth-generation tensor cores (tcgen05 / tensor memory), bf16.
+// Split decode attention on the fifth-generation tensor cores (tcgen05 / tensor memory): bf16
+// slabs, and slabs of E4M3 codes (one byte per element) with bf16 queries and output.
 //
 // Same contract as decode_tc_kernel (kernels.cu): persistent CTAs walk the items of the
 // host-built plan; an item is a run of tokens of one (request, KV head) stream; K and V tiles
@@ -46,6 +47,20 @@
 // bf16 and the fp32 accumulator hold without loss, and the accumulator in tensor memory is
 // rescaled (read, multiplied, written back) only on that rare path.  (m, l, O) with such a
 // reference is a valid partial result for the log-sum-exp merge.
+//
+// 8-bit slabs (F8): K and V tiles are E4M3 codes, 128 bytes per row, and both products are
+// kind::f8f6f4 instructions (E4M3 x E4M3, fp32 accumulation, K = 32), so the A operands must be
+// E4M3 as well.  Neither the queries nor the probabilities are rounded to 3 mantissa bits for
+// that: each is split into two E4M3 terms, x = hi + lo / 16, which occupy rows h and h + 8 of
+// the A operand (at most 8 heads per group), and the two result rows are added when they are
+// read from tensor memory (one thread holds rows h and h + 8 of its columns).  A bf16 query
+// times a power of two that brings its row's largest element into [128, 256) splits exactly
+// (8 significant bits = 4 + 4); a probability splits with a relative error of 2^-8, what
+// rounding it to bf16 costs the 16-bit kernel.  Probabilities are kept below 16 (reference
+// raised when a tile's maximum passes it by 2^4) and multiplied by 16 before the split, so
+// that the small ones stay normal numbers.  The key scale goes into the score factor, the
+// value scale onto the result; the step's new token is quantised by the query loader (codes to
+// the slab and to the side buffer) and used, like every other token, as its code's value.
 #include <algorithm>
 
 #include "device_utils.cuh"
@@ -59,36 +74,44 @@ using namespace dev;
 constexpr int kTile = 64;
 constexpr int kUmmaWarps = 8;
 constexpr int kUmmaThreads = kUmmaWarps * 32;
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr int kQSlots = 8;
 constexpr int kLanes = 2;
-constexpr float kRescaleAbove = 8.f;      // log2 units a tile's maximum may pass the reference by
+constexpr int kBothTiles = 4;             // 8-bit slabs: items of this many tiles or more are worked on by both lanes
+constexpr float kRescaleAbove = 8.f;      // log2 units a tile's maximum may pass the reference by (16-bit slabs)
+constexpr float kRescaleAbove8 = 4.f;     // 8-bit slabs: P < 16
+constexpr int kMaxStages16 = 8;           // stage-ring depth limits: 16-bit slabs / 8-bit slabs (kMaxStages)
 
 // barrier indices
 constexpr int kBarFull = 0, kBarEmpty = kMaxStages;
 constexpr int kBarQFull = 2 * kMaxStages, kBarQEmpty = kBarQFull + kQSlots;
 constexpr int kBarLane0 = kBarQEmpty + kQSlots;
-constexpr int kBarPerLane = 10;           // s_full[2] s_empty[2] p_full[2] p_empty[2] o_full o_empty
+constexpr int kBarPerLane = 12;           // s_full[2] s_empty[2] p_full[2] p_empty[2] o_full o_empty x_full x_empty
 constexpr int kBarDrain = kBarLane0 + kLanes * kBarPerLane;
 constexpr int kNumBars = kBarDrain + 3;
 
 constexpr int kTmemCols = 512;            // all of it: one CTA per SM
 constexpr int kTmemLaneCols = 256;        // per lane: S0 at +0, S1 at +64, O at +128
 
-template <int D, int NT>
+template <int D, int NT, bool F8>
 struct UmmaConfig {
-    static constexpr int kHalves = D / 64;                 // 128-byte column blocks per row
-    static constexpr int kKvTileBytes = kTile * D * 2;
+    static constexpr int kElem = F8 ? 1 : 2;               // bytes of a stored K/V element
+    static constexpr int kRowGroups = F8 ? 2 : NT;         // groups of 8 rows of the A operands (F8: hi and lo terms)
+    static constexpr int kHalves = D * kElem / 128;        // 128-byte column blocks per row
+    static constexpr int kKvTileBytes = kTile * D * kElem;
     static constexpr int kStageBytes = 2 * kKvTileBytes;
-    static constexpr int kQHalfBytes = NT * 1024;          // 8 NT rows of 128 bytes
+    static constexpr int kQHalfBytes = kRowGroups * 1024;  // rows of 128 bytes
     static constexpr int kQSlotBytes = kHalves * kQHalfBytes;
-    static constexpr int kPBufBytes = NT * 1024;           // 8 NT rows of 64 keys
+    static constexpr int kPBufBytes = kRowGroups * 1024;   // rows of 64 keys (F8: 64 of a row's 128 bytes used)
     static constexpr int kPBytes = kLanes * 2 * kPBufBytes;
     static constexpr int kQBytes = kQSlots * kQSlotBytes;
-    static constexpr int kNewBytes = 2 * D * 2;            // the step's new K row and V row of an item's stream
+    // the step's new K row and V row of an item's stream (as stored); F8: and the score factor of each head
+    static constexpr int kNewBytes = 2 * D * kElem + (F8 ? 64 : 0);
     static constexpr int kNewBufBytes = ((kQSlots * kNewBytes + 1023) / 1024) * 1024;
-    static constexpr int kTailBytes = kNumBars * 8 + 64;
+    static constexpr int kXchgBytes = kLanes * 16 * 2 * 4;  // per lane and head: (reference maximum, sum) of a helper lane
+    static constexpr int kTailBytes = kNumBars * 8 + 64 + kXchgBytes;
     static constexpr int kAlignSlack = 1024;
+    static constexpr int kStagesMax = F8 ? kMaxStages : kMaxStages16;
     static int smem_bytes(int stages) {
         return kNewBufBytes + kPBytes + kQBytes + stages * kStageBytes + kTailBytes + kAlignSlack;
     }
@@ -109,12 +132,26 @@ __host__ __device__ constexpr uint32_t umma_idesc(int m, int n, bool b_mn_major)
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
-        "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
+// Instruction descriptor of kind::f8f6f4: fp32 accumulator, E4M3 A and B (format 0), A K-major.
+__host__ __device__ constexpr uint32_t umma_idesc8(int m, int n, bool b_mn_major) {
+    return (1u << 4) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+template <bool F8>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    if (F8)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
+            "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
+            "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
 }
 
 // The barrier receives one arrival once every tcgen05.mma this thread has issued is complete.
@@ -194,15 +231,20 @@ __device__ __forceinline__ Item item_of(const int4& a, const int4& b, const Inli
     return it;
 }
 
-template <int D, int NT, int MODE>
+template <int D, int NT, int MODE, bool F8>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                    const __grid_constant__ InlineLens lens) {
-    using Cfg = UmmaConfig<D, NT>;
+    using Cfg = UmmaConfig<D, NT, F8>;
+    static_assert(!F8 || (D == 128 && NT == 1 && MODE == kModeSlab), "8-bit slabs: head_dim 128, group <= 8, slab mode");
+    constexpr int ES = Cfg::kElem;
     constexpr int HALVES = Cfg::kHalves;
     constexpr int HALF_BYTES = kTile * 128;           // one 128-byte column block of a K or V tile
-    constexpr int ROW_CHUNKS = D * 2 / 16;            // 16-byte chunks per row
-    constexpr int QK_STEPS = D / 16;                  // K = 16 per instruction
+    constexpr int ROW_CHUNKS = D * 2 / 16;            // 16-byte chunks per row of q, k_new, v_new (bf16)
+    constexpr int KV_CHUNKS = D * ES / 16;            // 16-byte chunks per stored row
+    constexpr int QK_STEPS = D * ES / 32;             // 32 bytes of a row per instruction (K = 16 or 32)
+    constexpr int PV_KEYS = 16 * (2 / ES);            // keys per instruction of the second product
+    constexpr float RESCALE_ABOVE = F8 ? kRescaleAbove8 : kRescaleAbove;
     const uint32_t STAGES = static_cast<uint32_t>(p.stages);
 
     extern __shared__ uint8_t smem_raw[];
@@ -217,11 +259,15 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     uint64_t* bars = reinterpret_cast<uint64_t*>(kv + STAGES * Cfg::kStageBytes);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(abort_flag) + 1);
+    float* xchg = reinterpret_cast<float*>(const_cast<int*>(abort_flag) + 16);   // [lane][head][2]
 
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int idx) { return bar0 + 8u * static_cast<uint32_t>(idx); };
     auto lane_bar = [&](int L, int idx) { return bar0 + 8u * static_cast<uint32_t>(kBarLane0 + L * kBarPerLane + idx); };
-    enum { S_FULL = 0, S_EMPTY = 2, P_FULL = 4, P_EMPTY = 6, O_FULL = 8, O_EMPTY = 9 };
+    enum { S_FULL = 0, S_EMPTY = 2, P_FULL = 4, P_EMPTY = 6, O_FULL = 8, O_EMPTY = 9, X_FULL = 10, X_EMPTY = 11 };
+    // 8-bit slabs: the softmax warp is the slowest role (a tile arrives in half the time), so an item of
+    // kBothTiles tiles or more is worked on by both lanes, its tiles going to them in turn
+    constexpr bool BOTH = F8;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -229,8 +275,9 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     const int cta = blockIdx.x;
     const bool fused = p.k_new != nullptr;
 
-    // a query slot is handed back by two parties: the MMA thread and the lane's softmax warp
-    if (tid < kNumBars) mbar_init(bar(tid), (tid >= kBarQEmpty && tid < kBarQEmpty + kQSlots) ? 2u : 1u);
+    // a query slot is handed back by the MMA thread and the lane's softmax warp (BOTH: and the other lane's,
+    // which takes the heads' score factors from it when it helps with the item)
+    if (tid < kNumBars) mbar_init(bar(tid), (tid >= kBarQEmpty && tid < kBarQEmpty + kQSlots) ? (BOTH ? 3u : 2u) : 1u);
     if (tid == 0) {
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -320,7 +367,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             const int ge = min(nb, max(im.safe - r0, 0) >> 4);
             const int g0 = part == 2 ? ge : 0, g1 = part == 1 ? ge : nb;
             if (part != 2) {
-                if (lane == 0) mbar_expect_tx(bar(kBarFull + stage), static_cast<uint32_t>(nb) * 16u * D * 2u * 2u);
+                if (lane == 0) mbar_expect_tx(bar(kBarFull + stage), static_cast<uint32_t>(nb) * 16u * D * ES * 2u);
                 issued_any |= 1u << stage;
                 issued_odd ^= 1u << stage;
                 __syncwarp();
@@ -405,6 +452,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 #pragma unroll
             for (int i = 0; i < Q_LOADS; ++i) {
                 const int idx = lane + 32 * i;
+                v[i] = make_uint4(0u, 0u, 0u, 0u);
                 if (idx < p.group * ROW_CHUNKS) v[i] = __ldg(reinterpret_cast<const uint4*>(src) + idx);
             }
             uint4 nv = make_uint4(0u, 0u, 0u, 0u);
@@ -417,20 +465,64 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQEmpty + slot), (use & 1u) ^ 1u, abort_flag, p.status, limit));
             if (!ok) break;
             uint8_t* dst = qbuf + slot * Cfg::kQSlotBytes;
+            if (F8) {
+                // A row of D bf16 numbers is 16 chunks: lanes 0..15 hold row 2i, lanes 16..31 row 2i + 1
+                // of load i.  Per row: the power of two that brings the largest element into [128, 256),
+                // then x * 2^e = hi + lo / 16 in E4M3 (exact for all but elements 2^13 below the largest),
+                // hi to row r, lo to row r + 8 of the slot; the score factor 2^-e * k_scale * log2(e) /
+                // sqrt(D) of the row goes to the side buffer.
+                float* qf = reinterpret_cast<float*>(newbuf + slot * Cfg::kNewBytes + 2 * D);
 #pragma unroll
-            for (int i = 0; i < Q_LOADS; ++i) {
-                const int idx = lane + 32 * i;
-                if (idx < p.group * ROW_CHUNKS) {
-                    const int r = idx / ROW_CHUNKS, c = idx - r * ROW_CHUNKS;
-                    *reinterpret_cast<uint4*>(dst + (c >> 3) * Cfg::kQHalfBytes + (r >> 3) * 1024 + (r & 7) * 128 +
-                                              (((c & 7) ^ (r & 7)) << 4)) = v[i];
+                for (int i = 0; i < Q_LOADS; ++i) {
+                    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                    uint32_t amax = 0;                   // as bits: the order of non-negative floats
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) amax = max(amax, max((w[j] << 16) & 0x7FFFFFFFu, w[j] & 0x7FFF0000u));
+#pragma unroll
+                    for (int sh = 1; sh < 16; sh <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sh));
+                    const int ex = static_cast<int>(amax >> 23);                 // biased exponent of the largest element
+                    const int e = (ex == 0 || ex == 255) ? 0 : min(134 - ex, 120);  // 2^e * largest in [128, 256)
+                    const float up = __uint_as_float(static_cast<uint32_t>(e + 127) << 23);
+                    const int r = (lane + 32 * i) / ROW_CHUNKS, c = (lane + 32 * i) % ROW_CHUNKS;
+                    if (r < p.group) {
+                        uint32_t hi[4], lo[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float x0 = __uint_as_float(w[j] << 16) * up, x1 = __uint_as_float(w[j] & 0xFFFF0000u) * up;
+                            hi[j] = pack_e4m3(x0, x1);
+                            const float2 h = unpack_e4m3(hi[j]);
+                            lo[j] = pack_e4m3((x0 - h.x) * 16.f, (x1 - h.y) * 16.f);
+                        }
+                        uint8_t* row = dst + r * 128 + ((((c >> 1) ^ r) & 7) << 4) + (c & 1) * 8;
+                        *reinterpret_cast<uint2*>(row) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+                        *reinterpret_cast<uint2*>(row + 1024) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+                        if (c == 0) qf[r] = __uint_as_float(static_cast<uint32_t>(127 - e) << 23) * (p.k_scale * p.scale_log2);
+                    }
                 }
-            }
-            if (mine) {
-                *reinterpret_cast<uint4*>(newbuf + slot * Cfg::kNewBytes + lane * 16) = nv;
-                uint4* slab = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
-                              ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
-                *slab = nv;
+                if (mine) {
+                    // the new rows as the slab will hold them: eight codes from this lane's eight numbers
+                    const uint2 codes = quantize8_e4m3(nv, kvsel ? p.v_inv : p.k_inv);
+                    *reinterpret_cast<uint2*>(newbuf + slot * Cfg::kNewBytes + lane * 8) = codes;
+                    uint2* slab = reinterpret_cast<uint2*>(const_cast<void*>(p.pool)) +
+                                  ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * (D / 8) + c_new;
+                    *slab = codes;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < Q_LOADS; ++i) {
+                    const int idx = lane + 32 * i;
+                    if (idx < p.group * ROW_CHUNKS) {
+                        const int r = idx / ROW_CHUNKS, c = idx - r * ROW_CHUNKS;
+                        *reinterpret_cast<uint4*>(dst + (c >> 3) * Cfg::kQHalfBytes + (r >> 3) * 1024 + (r & 7) * 128 +
+                                                  (((c & 7) ^ (r & 7)) << 4)) = v[i];
+                    }
+                }
+                if (mine) {
+                    *reinterpret_cast<uint4*>(newbuf + slot * Cfg::kNewBytes + lane * 16) = nv;
+                    uint4* slab = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
+                                  ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
+                    *slab = nv;
+                }
             }
             fence_proxy_async();
             __syncwarp();
@@ -444,7 +536,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // what they cost a lone thread of a diverged one.
         uint32_t elected;
         asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(elected));
-        constexpr uint32_t IDESC_QK = umma_idesc(64, kTile, false);
+        constexpr uint32_t IDESC_QK = F8 ? umma_idesc8(64, kTile, false) : umma_idesc(64, kTile, false);
         uint32_t c[kLanes] = {0, 0};                  // tiles of each lane issued so far
         uint32_t g = 0;
         fetch(it_begin);
@@ -452,7 +544,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             const int k = it - it_begin;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
             fetch(it + 1);
-            const int L = k & 1;
+            const bool both = BOTH && im.tiles >= kBothTiles;
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
             if (!ok) break;
@@ -465,6 +557,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             const uint32_t qb = q_u32 + slot * Cfg::kQSlotBytes;
             for (int t = 0; t < im.tiles; ++t, ++g) {
                 const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
+                const int L = (both ? k + t : k) & 1;
                 const uint32_t cc = L ? c[1] : c[0], b = cc & 1u, u = cc >> 1;
                 // both barriers are looked at before either answer is needed; the slow path only when one is not ready
                 const bool f_ok = mbar_try(bar(kBarFull + stage), phase), e_ok = mbar_try(lane_bar(L, S_EMPTY + b), (u & 1u) ^ 1u);
@@ -480,7 +573,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if (elected) {
 #pragma unroll
                     for (int ks = 0; ks < QK_STEPS; ++ks)
-                        umma_bf16(t_s, smem_desc(qb + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
+                        umma<F8>(t_s, smem_desc(qb + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
                                   smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
                     umma_commit(lane_bar(L, S_FULL + b));
                     if (t == im.tiles - 1) umma_commit(bar(kBarQEmpty + slot));
@@ -501,7 +594,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const int L = warp - 5;
         uint32_t elected;
         asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(elected));
-        constexpr uint32_t IDESC_PV = umma_idesc(64, D, true);
+        constexpr uint32_t IDESC_PV = F8 ? umma_idesc8(64, D, true) : umma_idesc(64, D, true);
         const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
         uint32_t c = 0, j = 0, g = 0;                 // the lane's tiles and items (with tiles) so far; ring position
         fetch(it_begin);
@@ -511,22 +604,25 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             fetch(it + 1);
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
-            if ((k & 1) != L || im.tiles == 0) continue;
-            for (int t = 0; t < im.tiles; ++t, ++c) {
+            // the lane's tiles of the item: all of them, or every second one when both lanes work on it
+            const bool both = BOTH && im.tiles >= kBothTiles;
+            if ((!both && (k & 1) != L) || im.tiles == 0) continue;
+            const int t_first = both ? (L ^ k) & 1 : 0, t_step = both ? 2 : 1;
+            for (int t = t_first; t < im.tiles; t += t_step, ++c) {
                 const uint32_t b = c & 1u, u = c >> 1, st = (g0 + static_cast<uint32_t>(t)) % STAGES;
                 bool good = mbar_wait_spin(lane_bar(L, P_FULL + b), u & 1u, abort_flag, p.status, limit);
-                if (good && t == 0) good = mbar_wait(lane_bar(L, O_EMPTY), (j & 1u) ^ 1u, abort_flag, p.status, limit);
+                if (good && t == t_first) good = mbar_wait(lane_bar(L, O_EMPTY), (j & 1u) ^ 1u, abort_flag, p.status, limit);
                 ok = __all_sync(0xFFFFFFFFu, good);
                 if (!ok) break;
                 tc_fence_after();
-                const bool last = t == im.tiles - 1;
-                const int ksteps = last ? (im.n_slab - t * kTile + 15) >> 4 : 4;
+                const bool last = t + t_step >= im.tiles;                      // the lane's last tile of the item
+                const int ksteps = (t == im.tiles - 1 ? im.n_slab - t * kTile + PV_KEYS - 1 : kTile) / PV_KEYS;
                 const uint32_t vbase = kv_u32 + st * Cfg::kStageBytes + Cfg::kKvTileBytes;
                 const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + static_cast<int>(b)) * Cfg::kPBufBytes);
                 if (elected) {
                     for (int ks = 0; ks < ksteps; ++ks)
-                        umma_bf16(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * 2048, HALF_BYTES, 1024), IDESC_PV,
-                                  (t == 0 && ks == 0) ? 0u : 1u);
+                        umma<F8>(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * (PV_KEYS * 128), HALF_BYTES, 1024), IDESC_PV,
+                                  (t == t_first && ks == 0) ? 0u : 1u);
                     umma_commit(bar(kBarEmpty + st));
                     umma_commit(lane_bar(L, P_EMPTY + b));
                     if (last) umma_commit(lane_bar(L, O_FULL));
@@ -548,6 +644,9 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const int group = p.group;
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
         uint32_t c = 0, j = 0, g = 0;                       // the lane's tiles and items so far; ring position
+        uint32_t n_helped = 0, n_merged = 0;                // items this lane helped with / merged the other lane's part of
+        float* x_mine = xchg + L * 32;                      // where this lane leaves (m, l) per head as a helper
+        const float* x_other = xchg + (L ^ 1) * 32;
         fetch(it_begin);
         for (int it = it_begin; it < it_end && ok; ++it) {
             const int k = it - it_begin;
@@ -555,10 +654,23 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             fetch(it + 1);
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
-            if ((k & 1) != L) continue;
+            // BOTH: an item of kBothTiles tiles or more is worked on by both lanes, its tiles going to
+            // them in turn from its home lane (item number mod 2).  The other lane is the helper: it
+            // leaves its accumulator in tensor memory and its (m, l) in shared memory, and the home
+            // lane merges the two parts and finishes the item.  Every item's query slot is visited by
+            // both softmax warps (each sees every phase of the slot's barriers, and a helper takes the
+            // heads' score factors from it).
+            const bool both = BOTH && im.tiles >= kBothTiles, home = (k & 1) == L;
+            if (!BOTH && !home) continue;
+            const int t_first = both ? (L ^ k) & 1 : 0, t_step = both ? 2 : 1;
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
             if (!ok) break;
+            if (!both && !home) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
+                continue;
+            }
             // The token appended this step: its scaled score per head from the query rows and the
             // new K row in shared memory (each thread adds up the elements it will also hold of the
             // output, the quad completes the sum); its value row, packed, for when the item ends.
@@ -566,7 +678,27 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             uint32_t v_new[D / 8];
 #pragma unroll
             for (int rs = 0; rs < NT; ++rs) s_new[rs] = -INFINITY;
-            if (im.has_new) {
+            float qfac = scale;                            // F8: the head's score factor (query power of two, key scale)
+            if (F8) qfac = reinterpret_cast<const float*>(newbuf + slot * Cfg::kNewBytes + 2 * D)[hq];
+            if (im.has_new && home && F8) {
+                // queries as hi + lo / 16 from rows hq and hq + 8 of the slot, the new rows as codes
+                const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes + hq * 128;
+                const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
+                float dot = 0.f;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) {
+                    const float2 kk = unpack_e4m3(*reinterpret_cast<const uint16_t*>(nk + 8 * i + kq));
+                    v_new[i] = *reinterpret_cast<const uint16_t*>(nk + D + 8 * i + kq);
+                    const int off = (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
+                    const float2 qh = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + off));
+                    const float2 ql = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + 1024 + off));
+                    dot = fmaf(fmaf(ql.x, 0.0625f, qh.x), kk.x, dot);
+                    dot = fmaf(fmaf(ql.y, 0.0625f, qh.y), kk.y, dot);
+                }
+                dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 1);
+                dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 2);
+                s_new[0] = dot * qfac;
+            } else if (im.has_new && home) {
                 const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes;
                 const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
                 const uint8_t* nvp = nk + D * 2;
@@ -601,7 +733,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 m_ref[rs] = s_new[rs];
                 l_acc[rs] = 0.f;
             }
-            for (int t = 0; t < im.tiles; ++t) {
+            for (int t = t_first; t < im.tiles; t += t_step) {
                 const uint32_t b = c & 1u, u = c >> 1;
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
                 if (!ok) break;
@@ -622,7 +754,8 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     for (int i = 0; i < 8; ++i)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            float s = __uint_as_float(r[4 * i + 2 * rs + e]) * scale;
+                            float s = F8 ? fmaf(__uint_as_float(r[4 * i + 2 + e]), 0.0625f, __uint_as_float(r[4 * i + e])) * qfac
+                                         : __uint_as_float(r[4 * i + 2 * rs + e]) * scale;
                             if (8 * i + kq + e >= valid) s = -INFINITY;
                             sc[rs][2 * i + e] = s;
                             mx[rs] = fmaxf(mx[rs], s);
@@ -630,13 +763,13 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 1));
                     mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 2));
                 }
-                if (t == 0) {
+                if (t == t_first) {
 #pragma unroll
                     for (int rs = 0; rs < NT; ++rs) m_ref[rs] = fmaxf(m_ref[rs], mx[rs]);
                 } else {
                     bool grow = false;
 #pragma unroll
-                    for (int rs = 0; rs < NT; ++rs) grow = grow || mx[rs] > m_ref[rs] + kRescaleAbove;
+                    for (int rs = 0; rs < NT; ++rs) grow = grow || mx[rs] > m_ref[rs] + RESCALE_ABOVE;
                     if (__any_sync(0xFFFFFFFFu, grow)) {
                         // Rare: raise the reference of the heads that need it and rescale their
                         // rows of the accumulator.  Every second product issued so far must be
@@ -650,11 +783,12 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                         float f[2] = {1.f, 1.f};
 #pragma unroll
                         for (int rs = 0; rs < NT; ++rs) {
-                            const float mn = mx[rs] > m_ref[rs] + kRescaleAbove ? mx[rs] : m_ref[rs];
+                            const float mn = mx[rs] > m_ref[rs] + RESCALE_ABOVE ? mx[rs] : m_ref[rs];
                             f[rs] = fast_exp2(m_ref[rs] - mn);
                             l_acc[rs] *= f[rs];
                             m_ref[rs] = mn;
                         }
+                        if (F8) f[1] = f[0];             // rows h and h + 8 are the two terms of one head
 #pragma unroll
                         for (int blk = 0; blk < D / 32; ++blk) {
                             uint32_t o[16];
@@ -684,18 +818,29 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     for (int i = 0; i < 8; ++i) {
                         const float p0 = fast_exp2(sc[rs][2 * i] - m_ref[rs]), p1 = fast_exp2(sc[rs][2 * i + 1] - m_ref[rs]);
                         sum += p0 + p1;
-                        *reinterpret_cast<uint32_t*>(pb + rs * 1024 + hq * 128 + ((i ^ hq) << 4) + kq * 2) = pack_bf16(p0, p1);
+                        if (F8) {
+                            // 16 P = hi + lo / 16: hi to row hq, lo to row hq + 8; keys 8i + kq, + 1 are bytes of the row
+                            const float y0 = p0 * 16.f, y1 = p1 * 16.f;
+                            const uint32_t hi = pack_e4m3(y0, y1);
+                            const float2 h = unpack_e4m3(hi);
+                            const uint32_t lo = pack_e4m3((y0 - h.x) * 16.f, (y1 - h.y) * 16.f);
+                            uint8_t* dst = pb + hq * 128 + (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
+                            *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(hi);
+                            *reinterpret_cast<uint16_t*>(dst + 1024) = static_cast<uint16_t>(lo);
+                        } else {
+                            *reinterpret_cast<uint32_t*>(pb + rs * 1024 + hq * 128 + ((i ^ hq) << 4) + kq * 2) = pack_bf16(p0, p1);
+                        }
                     }
                     l_acc[rs] += sum;
                 }
-                if (valid & 15) {
-                    // the second product takes whole groups of 16 keys: value rows between the item's
-                    // end and the end of its last group are zeroed (P is zero there; the rows hold
-                    // whatever the slab does, which may not be a finite number)
+                if (valid & (PV_KEYS - 1)) {
+                    // the second product takes whole groups of 16 (8-bit slabs: 32) keys: value rows between
+                    // the item's end and the end of its last group are zeroed (P is zero there; the rows hold
+                    // whatever the slab or the stage did, which may not be a finite number)
                     uint8_t* vt = kv + ((g0 + static_cast<uint32_t>(t)) % STAGES) * Cfg::kStageBytes + Cfg::kKvTileBytes;
-                    const int zero_rows = 16 - (valid & 15);
-                    for (int idx = lane; idx < zero_rows * ROW_CHUNKS; idx += 32) {
-                        const int zr = valid + idx / ROW_CHUNKS, cc = idx % ROW_CHUNKS;
+                    const int zero_rows = PV_KEYS - (valid & (PV_KEYS - 1));
+                    for (int idx = lane; idx < zero_rows * KV_CHUNKS; idx += 32) {
+                        const int zr = valid + idx / KV_CHUNKS, cc = idx % KV_CHUNKS;
                         *reinterpret_cast<uint4*>(vt + (cc >> 3) * HALF_BYTES + zr * 128 + (((cc & 7) ^ (zr & 7)) << 4)) =
                             make_uint4(0u, 0u, 0u, 0u);
                     }
@@ -706,6 +851,21 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 ++c;
             }
             if (!ok) break;
+            if (BOTH && !home) {
+                // helper: once its accumulator is complete, (m, l) per head goes to shared memory;
+                // the home lane reads the accumulator itself and signs it off
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
+                if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, X_EMPTY), (n_helped & 1u) ^ 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                ++j;
+                ++n_helped;
+                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 1);
+                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 2);
+                if ((lane & 3) == 0) *reinterpret_cast<float2*>(x_mine + hq * 2) = make_float2(m_ref[0], l_acc[0]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, X_FULL));
+                continue;
+            }
 
             // ---- the item's result: O from tensor memory, then out / partial / merge
             float oo[NT][D / 4];                          // [rs][2i + e]: head hq + 8 rs, element 8i + kq + e
@@ -722,8 +882,14 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     for (int i = 0; i < 8; ++i)
 #pragma unroll
                         for (int rs = 0; rs < NT; ++rs) {
-                            oo[rs][2 * (8 * blk + i)] = __uint_as_float(r[4 * i + 2 * rs]);
-                            oo[rs][2 * (8 * blk + i) + 1] = __uint_as_float(r[4 * i + 2 * rs + 1]);
+                            if (F8) {                     // (hi row + lo row / 16) / 16: P went in times 16
+                                oo[0][2 * (8 * blk + i)] = fmaf(__uint_as_float(r[4 * i + 2]), 0.0625f, __uint_as_float(r[4 * i])) * 0.0625f;
+                                oo[0][2 * (8 * blk + i) + 1] =
+                                    fmaf(__uint_as_float(r[4 * i + 3]), 0.0625f, __uint_as_float(r[4 * i + 1])) * 0.0625f;
+                            } else {
+                                oo[rs][2 * (8 * blk + i)] = __uint_as_float(r[4 * i + 2 * rs]);
+                                oo[rs][2 * (8 * blk + i) + 1] = __uint_as_float(r[4 * i + 2 * rs + 1]);
+                            }
                         }
                 }
                 tc_fence_before();
@@ -741,6 +907,41 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 l_acc[rs] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[rs], 1);
                 l_acc[rs] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[rs], 2);
             }
+            if (BOTH && both) {
+                // the helper lane's part: its (m, l) from shared memory, its accumulator from its
+                // columns of tensor memory; both are signed off on its behalf
+                const int LO = L ^ 1;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(LO, X_FULL), n_merged & 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                ++n_merged;
+                tc_fence_after();
+                const float2 ml = *reinterpret_cast<const float2*>(x_other + hq * 2);
+                const float mn = fmaxf(m_ref[0], ml.x);
+                const float e_mine = fast_exp2(m_ref[0] - mn), w_other = fast_exp2(ml.x - mn);
+                const float e_other = w_other * 0.0625f;     // its accumulator still carries the factor 16 of P
+                l_acc[0] = fmaf(l_acc[0], e_mine, ml.y * w_other);
+                m_ref[0] = mn;
+                const uint32_t t_o_other = tmem + static_cast<uint32_t>(LO * kTmemLaneCols) + 128u;
+#pragma unroll
+                for (int blk = 0; blk < D / 64; ++blk) {
+                    uint32_t r[32];
+                    tmem_ld_x8(t_o_other + blk * 64u, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {          // (hi row + lo row / 16) / 16, as in the lane's own read-out
+                        float& a0 = oo[0][2 * (8 * blk + i)];
+                        float& a1 = oo[0][2 * (8 * blk + i) + 1];
+                        a0 = fmaf(a0, e_mine, fmaf(__uint_as_float(r[4 * i + 2]), 0.0625f, __uint_as_float(r[4 * i])) * e_other);
+                        a1 = fmaf(a1, e_mine, fmaf(__uint_as_float(r[4 * i + 3]), 0.0625f, __uint_as_float(r[4 * i + 1])) * e_other);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(lane_bar(LO, O_EMPTY));
+                    mbar_arrive(lane_bar(LO, X_EMPTY));
+                }
+            }
             if (im.has_new) {
 #pragma unroll
                 for (int rs = 0; rs < NT; ++rs) {
@@ -748,10 +949,16 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                     l_acc[rs] += pn;
 #pragma unroll
                     for (int i = 0; i < D / 8; ++i) {
-                        oo[rs][2 * i] = fmaf(pn, __uint_as_float(v_new[i] << 16), oo[rs][2 * i]);
-                        oo[rs][2 * i + 1] = fmaf(pn, __uint_as_float(v_new[i] & 0xFFFF0000u), oo[rs][2 * i + 1]);
+                        const float2 vv = F8 ? unpack_e4m3(v_new[i])
+                                             : make_float2(__uint_as_float(v_new[i] << 16), __uint_as_float(v_new[i] & 0xFFFF0000u));
+                        oo[rs][2 * i] = fmaf(pn, vv.x, oo[rs][2 * i]);
+                        oo[rs][2 * i + 1] = fmaf(pn, vv.y, oo[rs][2 * i + 1]);
                     }
                 }
+            }
+            if (F8) {                                      // codes to values
+#pragma unroll
+                for (int i = 0; i < D / 4; ++i) oo[0][i] *= p.v_scale;
             }
             auto write_out = [&](int req, int head, int rs, float M, float Lsum, const float (&x)[D / 4]) {
                 const int h = hq + 8 * rs;
@@ -854,20 +1061,20 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 constexpr int kSmemPerCtaMax = 232448;    // most dynamic shared memory one CTA may ask for
 constexpr int kMaxDevices = 64;
 
-template <int D, int NT>
+template <int D, int NT, bool F8>
 int umma_stages() {
-    using Cfg = UmmaConfig<D, NT>;
+    using Cfg = UmmaConfig<D, NT, F8>;
     const int n = (kSmemPerCtaMax - Cfg::smem_bytes(0)) / Cfg::kStageBytes;
-    return std::min(n, kMaxStages);
+    return std::min(n, Cfg::kStagesMax);
 }
 
-template <int D, int NT, int MODE>
+template <int D, int NT, int MODE, bool F8>
 cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas, cudaStream_t stream,
                              const InlineLens& lens) {
-    using Cfg = UmmaConfig<D, NT>;
+    using Cfg = UmmaConfig<D, NT, F8>;
     static bool configured[kMaxDevices] = {false};     // the opt-in to large shared memory is per device
-    auto kern = decode_umma_kernel<D, NT, MODE>;
-    p.stages = umma_stages<D, NT>();
+    auto kern = decode_umma_kernel<D, NT, MODE, F8>;
+    p.stages = umma_stages<D, NT, F8>();
     if (p.stages < 2) return cudaErrorInvalidValue;
     const int smem = Cfg::smem_bytes(p.stages);
     int dev = 0;
@@ -896,15 +1103,16 @@ template <int D, int NT>
 cudaError_t launch_umma_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s,
                              const InlineLens& lens) {
     switch (mode) {
-        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab>(maps, p, n_ctas, s, lens);
-        case kModePaged: return launch_umma_inst<D, NT, kModePaged>(maps, p, n_ctas, s, lens);
+        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab, false>(maps, p, n_ctas, s, lens);
+        case kModePaged: return launch_umma_inst<D, NT, kModePaged, false>(maps, p, n_ctas, s, lens);
     }
     return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
-bool umma_supported(int32_t head_dim, int32_t group) {
+bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8) {
+    if (kv_fp8) return head_dim == 128 && group >= 1 && group <= 8;
     return (head_dim == 64 || head_dim == 128) && group >= 1 && group <= 16;
 }
 
@@ -912,6 +1120,10 @@ cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, in
                                cudaStream_t stream, const InlineLens* lens_in) {
     static const InlineLens no_lens{};                 // n = 0: lengths as planned
     const InlineLens& lens = lens_in ? *lens_in : no_lens;
+    if (p.kv_fp8) {
+        if (!umma_supported(p.head_dim, p.group, true) || mode != kModeSlab) return cudaErrorInvalidValue;
+        return launch_umma_inst<128, 1, kModeSlab, true>(maps, p, n_ctas, stream, lens);
+    }
     const bool two = p.group > 8;
     if (p.head_dim == 128)
         return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens)

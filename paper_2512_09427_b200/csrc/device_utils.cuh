@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "kernels.hpp"
 
@@ -163,6 +164,29 @@ __device__ __forceinline__ float fast_rcp(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// E4M3 (8-bit float: 4 exponent bits, 3 mantissa bits, no infinities, largest value 448).
+// Two fp32 numbers to two codes, round to nearest even, saturating: `lo` in the low byte.
+__device__ __forceinline__ uint32_t pack_e4m3(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// Two codes (low 16 bits of `codes`) to two fp32 numbers (every code is exact in fp16).
+__device__ __forceinline__ float2 unpack_e4m3(uint32_t codes) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(static_cast<uint16_t>(codes)));
+    return __half22float2(*reinterpret_cast<__half2*>(&h2));
+}
+// Eight bf16 numbers (one 16-byte vector) times `inv` in fp32, rounded to eight codes.
+__device__ __forceinline__ uint2 quantize8_e4m3(const uint4& v, float inv) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        c[i] = pack_e4m3(__fmul_rn(__uint_as_float(w[i] << 16), inv), __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), inv));
+    return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
 }
 
 __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }

@@ -1,6 +1,7 @@
 // CUDA kernels of libodma for sm_100a.
 //
-//  append_kv_kernel        writes the step's new K/V rows behind each request's tokens
+//  append_kv_kernel        writes the step's new K/V rows behind each request's tokens (an 8-bit
+//                          pool: quantised to E4M3 on the way)
 //  migrate_copy_kernel     slab -> slab copy of one request (allocate-and-copy migration)
 //  decode_tc_kernel        split decode attention, bf16: TMA-staged slab streams, keys on the M
 //                          side and the GQA group's heads on the N side of mma.sync tiles, fp32
@@ -1035,6 +1036,7 @@ combine_kernel(const int4* __restrict__ combine, const float* __restrict__ part_
 // append / migrate / page scatter: 16-byte vector copies
 // =============================================================================================
 
+template <bool QUANT>
 __global__ void __launch_bounds__(256) append_kv_kernel(const AppendParams p) {
     const int64_t vecs_per_tok = static_cast<int64_t>(p.kv_heads) * p.row_vecs;
     const int64_t total = static_cast<int64_t>(p.n_new_total) * vecs_per_tok * 2;
@@ -1063,7 +1065,14 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const AppendParams p) {
                             static_cast<int64_t>(head) * p.cap[req] + pos;
         const int64_t array = static_cast<int64_t>(p.layer) * 2 + kv;
         const uint4* src = static_cast<const uint4*>(kv ? p.v_new : p.k_new);
-        pool[(array * p.rows_per_array + row) * p.row_vecs + vec] = src[rem];
+        if (QUANT) {
+            // a stored vector of 16 codes comes from two vectors of eight bf16 numbers
+            const float inv = kv ? p.v_inv : p.k_inv;
+            const uint2 a = quantize8_e4m3(src[2 * rem], inv), b = quantize8_e4m3(src[2 * rem + 1], inv);
+            pool[(array * p.rows_per_array + row) * p.row_vecs + vec] = make_uint4(a.x, a.y, b.x, b.y);
+        } else {
+            pool[(array * p.rows_per_array + row) * p.row_vecs + vec] = src[rem];
+        }
     }
 }
 
@@ -1247,7 +1256,10 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t stream) {
     const int64_t total = static_cast<int64_t>(p.n_new_total) * p.kv_heads * p.row_vecs * 2;
     const int64_t blocks = (total + 255) / 256;
     const int grid = static_cast<int>(blocks < 148 * 16 ? blocks : 148 * 16);
-    append_kv_kernel<<<grid, 256, 0, stream>>>(p);
+    if (p.quantize)
+        append_kv_kernel<true><<<grid, 256, 0, stream>>>(p);
+    else
+        append_kv_kernel<false><<<grid, 256, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

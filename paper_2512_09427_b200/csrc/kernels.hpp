@@ -45,6 +45,9 @@ struct DecodeParams {
     int32_t chained;            // tcgen05 kernel: the previous kernel of the stream is this kernel on the
                                 // previous layer of the same step (same plan, other K/V arrays, other
                                 // outputs, the other scratch set): nothing of this launch waits for it
+    int32_t kv_fp8;             // the pool holds E4M3 codes (one byte per element); q, the new rows and out are bf16
+    float k_scale, v_scale;     // 8-bit pool: a stored code stands for value * scale (this layer's scales)
+    float k_inv, v_inv;         // fp32 reciprocals: what an appended element is multiplied by before rounding
     int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
 };
@@ -58,7 +61,7 @@ struct InlineLens {
 };
 
 struct TensorMaps {
-    CUtensorMap box[4];   // boxes of 16, 32, 48 and 64 rows x 64 elements (box[k]: 16 (k+1) rows)
+    CUtensorMap box[4];   // boxes of 16, 32, 48 and 64 rows x 128 bytes (box[k]: 16 (k+1) rows)
 };
 
 enum DecodeMode { kModeSlab = 0, kModePaged = 1, kModeProbe = 2 };
@@ -72,7 +75,8 @@ cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int 
                              cudaStream_t stream, const InlineLens* lens = nullptr);
 // The same decode step on the tcgen05 tensor cores (decode_umma.cu): slab and paged modes;
 // `stages` and `q_slots` of the parameter block are ignored (the kernel sizes its own rings).
-bool umma_supported(int32_t head_dim, int32_t group);
+// An 8-bit (E4M3) pool: head_dim 128, group <= 8, slab mode.
+bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8);
 cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
                                cudaStream_t stream, const InlineLens* lens = nullptr);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
@@ -94,6 +98,8 @@ struct AppendParams {
     int32_t layer, n, kv_heads, n_new_total;
     int32_t row_vecs;           // 16-byte vectors per row
     int32_t one_new_each;       // every request appends exactly one token: token index = request
+    int32_t quantize;           // the pool holds E4M3 codes: the bf16 rows are multiplied by k_inv / v_inv in
+    float k_inv, v_inv;         // fp32 and rounded to the nearest code (row_vecs counts the stored row)
 };
 cudaError_t launch_append(const AppendParams& p, cudaStream_t stream);
 

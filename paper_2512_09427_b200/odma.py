@@ -21,7 +21,7 @@ _lib = C.CDLL(LIB_PATH)
 
 MAX_BUCKETS = 8
 OK, ERR_INVALID, ERR_NOMEM, ERR_UNKNOWN_REQ, ERR_DUP_REQ, ERR_OVERFLOW, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(9)
-DTYPE_F32, DTYPE_BF16 = 0, 1
+DTYPE_F32, DTYPE_BF16, DTYPE_FP8_E4M3 = 0, 1, 2
 DECODE_AUTO, DECODE_TCGEN05, DECODE_MMA_SYNC = 0, 1, 2
 K_APPEND, K_DECODE, K_COMBINE, K_MIGRATE, K_PROBE = range(5)
 
@@ -91,6 +91,7 @@ _SIGS = {
     "odma_strerror": (C.c_char_p, [_i32]),
     "odma_pool_create": (_i32, [_vp, _u64, _i32, _i32, _i32, _i32, C.POINTER(Config), C.POINTER(_vp)]),
     "odma_pool_destroy": (_i32, [_vp]),
+    "odma_set_kv_scales": (_i32, [_vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]),
     "odma_set_buckets": (_i32, [_vp, _i32p, _i32]),
     "odma_get_buckets": (_i32, [_vp, _i32p, _i32p, _u64p]),
     "odma_alloc": (_i32, [_vp, _u64, _i32, C.POINTER(Slab)]),
@@ -178,6 +179,12 @@ class Pool:
             self.destroy()
         except Exception:
             pass
+
+    def set_kv_scales(self, k_scale: Sequence[float], v_scale: Sequence[float]) -> None:
+        """Per-layer dequantisation scales of an 8-bit (E4M3) pool."""
+        assert len(k_scale) == self.layers and len(v_scale) == self.layers
+        _check(_lib.odma_set_kv_scales(self._h, (C.c_float * self.layers)(*k_scale), (C.c_float * self.layers)(*v_scale)),
+               "odma_set_kv_scales")
 
     # -- boundaries --------------------------------------------------------------------------
     def set_buckets(self, b: Sequence[int]) -> int:

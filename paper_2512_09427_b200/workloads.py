@@ -19,7 +19,7 @@ none of which are available offline.
 from __future__ import annotations
 
 import math
-from dataclasses import dataclass, field
+from dataclasses import dataclass, field, replace
 from typing import Callable, Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
@@ -208,6 +208,7 @@ class Workload:
     refresh: int = 1000
     granule: int = 16
     extra: dict = field(default_factory=dict)
+    kv_dtype: str = ""                        # "": K/V stored as `dtype`; "e4m3": one byte per element
 
     @property
     def batch(self) -> int:
@@ -215,11 +216,26 @@ class Workload:
 
     @property
     def elem_bytes(self) -> int:
+        """Bytes of a stored K/V element."""
+        if self.kv_dtype == "e4m3":
+            return 1
         return 2 if self.dtype == torch.bfloat16 else 4
 
     @property
     def bytes_per_token(self) -> int:
         return self.layers * 2 * self.kv_heads * self.head_dim * self.elem_bytes
+
+
+def with_e4m3(w: Workload) -> Workload:
+    """The same workload on 8-bit slabs: the pool holds the same number of tokens in half the bytes."""
+    assert w.dtype == torch.bfloat16
+    return replace(w, name=w.name + "-e4m3", kv_dtype="e4m3", pool_bytes=w.pool_bytes // 2)
+
+
+def e4m3_scales(layers: int):
+    """Per-layer dequantisation scales the tests and the benchmark use with N(0,1) rows: the format's
+    largest value (448) then stands for 5.6 to 7 standard deviations."""
+    return [0.0125 + 0.0005 * (l % 7) for l in range(layers)], [0.015 + 0.0005 * (l % 5) for l in range(layers)]
 
 
 def config1(variant: str = "a") -> Workload:

@@ -43,10 +43,17 @@ def oracle_allocator(w: wl.Workload, **over) -> ora.Allocator:
     return ora.Allocator(w.pool_bytes, w.layers, w.kv_heads, w.head_dim, w.elem_bytes, **args)
 
 
+def pool_dtype(w: wl.Workload) -> int:
+    odma = lib()
+    if w.kv_dtype == "e4m3":
+        return odma.DTYPE_FP8_E4M3
+    return odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
+
+
 def host_pool(w: wl.Workload, **over):
     """A bookkeeping-only pool (no device memory)."""
     odma = lib()
-    dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
+    dt = pool_dtype(w)
     return odma.Pool(0, w.pool_bytes, w.layers, w.kv_heads, w.head_dim, dt, make_cfg(w, **over))
 
 
@@ -146,7 +153,8 @@ class Session:
         self.odma, self.w = odma, w
         self.dev = torch.device("cuda:0")
         self.gen_dev = self.dev          # where the seeded inputs are generated ("cpu": no generator kernels on the GPU)
-        self.dt = odma.DTYPE_BF16 if w.dtype == torch.bfloat16 else odma.DTYPE_F32
+        self.dt = pool_dtype(w)
+        self.e4m3 = w.kv_dtype == "e4m3"
         self.mem = torch.empty(w.pool_bytes, dtype=torch.uint8, device=self.dev)
         if fill is not None:
             self.mem.view(torch.int16).fill_(fill)
@@ -157,7 +165,11 @@ class Session:
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
                               self.dt, self.cfg)
         self.ls = LockStep(self.pool, oracle_allocator(w), self.stream)
-        self.kv = ora.KVStore(w.layers, w.kv_heads, w.head_dim, ora.dtype_code(w.dtype)) if mirror_kv else None
+        self.k_scale, self.v_scale = wl.e4m3_scales(w.layers) if self.e4m3 else (None, None)
+        if self.e4m3:
+            self.pool.set_kv_scales(self.k_scale, self.v_scale)
+        self.kv = ora.KVStore(w.layers, w.kv_heads, w.head_dim, ora.dtype_code(w.dtype), kv_e4m3=self.e4m3,
+                              k_scale=self.k_scale, v_scale=self.v_scale) if mirror_kv else None
         self.table = torch.empty(self.pool.tables_bytes(self.cfg.max_batch), dtype=torch.uint8, device=self.dev)
         self.lens = {}
         st = self.pool.get_stats()
@@ -244,13 +256,13 @@ class Session:
 
     def pool_rows(self, layer, kv, req, head=None):
         """The request's rows read back from the device pool through the documented formula:
-        [len, kv_heads, head_dim] in token-major order."""
+        [len, kv_heads, head_dim] in token-major order (8-bit pools: the codes, uint8)."""
         rc, slab, ln = self.pool.get_slab(int(req))
         assert rc == 0
         base, cap = slab[0], slab[1]
         w = self.w
         n_elems = w.layers * 2 * self.T * w.kv_heads * w.head_dim
-        arr = self.mem.view(w.dtype)[:n_elems].view(w.layers * 2, self.T * w.kv_heads, w.head_dim)[layer * 2 + kv]
+        arr = self.mem.view(torch.uint8 if self.e4m3 else w.dtype)[:n_elems].view(w.layers * 2, self.T * w.kv_heads, w.head_dim)[layer * 2 + kv]
         heads = [arr[base * w.kv_heads + h * cap: base * w.kv_heads + h * cap + ln] for h in range(w.kv_heads)]
         return torch.stack(heads, dim=1)
 
