@@ -111,6 +111,16 @@ typedef struct odma_config {
                                 kernel, ODMA_DECODE_MMA_SYNC the mma.sync kernel, ODMA_DECODE_AUTO
                                 the first for the layers of an odma_decode_step over several
                                 layers and the second for single launches (0) */
+    int32_t async_recal;     /* 1: a background thread owns the length window: odma_free only logs the
+                                realised length, the thread applies the log in order and refreshes the
+                                boundaries off the critical path (Sections III-E, IV-C); boundaries at
+                                any moment are those of a prefix of the log, after odma_recal_flush
+                                those of the whole log.  0: the refresh runs inside odma_free (0) */
+    int32_t cluster_observe; /* 1: a completion's length goes only to the outbox read by
+                                odma_drain_observations and enters the window through odma_observe
+                                (every replica then feeds the same merged sequence and derives the
+                                same boundaries: the bucket configuration a cluster manager keeps
+                                consistent, Section III-E); 0: it enters the window at once (0) */
 } odma_config;
 
 typedef struct odma_slab {
@@ -170,6 +180,20 @@ const char* odma_strerror(int32_t code);
 int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t kv_heads,
                          int32_t head_dim, int32_t dtype, const odma_config* cfg, odma_pool** out);
 int32_t odma_pool_destroy(odma_pool* pool);
+
+/* ---- boundary refresh off the critical path and across replicas (Sections III-E, IV-C) ------
+ * odma_recal_flush: returns once the background thread (async_recal) has applied every length
+ * logged so far; a no-op otherwise.
+ * odma_drain_observations: copies to `out` (host, room for `cap` values) the lengths of the
+ * requests completed on this pool since the last drain, oldest first (at most `window` are
+ * kept), and forgets them; *n = how many.
+ * odma_observe: feeds `n` realised lengths (host; 0 <= length <= max_len) into the window as if
+ * they had completed here, in the given order; every `refresh`-th observation re-derives the
+ * boundaries (Eq. 2).  Replicas that exchange their drained lengths and observe the
+ * concatenation in rank order hold identical windows and so identical boundaries. */
+int32_t odma_recal_flush(odma_pool* pool);
+int32_t odma_drain_observations(odma_pool* pool, int32_t* out, int32_t cap, int32_t* n);
+int32_t odma_observe(odma_pool* pool, const int32_t* lengths, int32_t n);
 
 /* Dequantisation scales of an ODMA_DTYPE_FP8_E4M3 pool (the 8-bit variant of the slab layout;
  * the paper's slabs hold the serving stack's 16-bit cache, Section IV-A): k_scale, v_scale:
@@ -232,6 +256,22 @@ int32_t odma_plan_host(odma_pool* pool, const uint64_t* reqs, const int32_t* n_n
                        int32_t* host_table, uint64_t table_bytes, odma_tables* out);
 int32_t odma_build_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
                           void* d_table, uint64_t table_bytes, void* stream, odma_tables* out);
+
+/* ---- chunked prefill over the slabs (Section II-A: the prefill phase fills the cache with the
+ *      prompt's keys and values before decoding starts) --------------------------------------
+ * A chunk of n_new[i] >= 1 prompt tokens per request is appended with the ordinary calls
+ * (odma_build_tables with n_new, odma_append_kv); its causal attention is then the decode
+ * attention of one stream PER NEW TOKEN over the owner's slab: token j of request i attends
+ * keys [0, len[i] + j] (len[i] = the committed length, the chunk not yet committed).  This
+ * call plans those sum(n_new) streams (at most max_batch of them; ODMA_ERR_INVALID beyond)
+ * and writes their table to d_table (device, table_bytes >= odma_tables_bytes(pool,
+ * sum(n_new))); odma_decode_attention with the returned descriptor, q and out of shape
+ * [sum(n_new), q_heads, head_dim] (tokens in request order, then position order), computes
+ *   out[t][h] = softmax_{k <= pos(t)}(q[t][h] . K[h div g][k] / sqrt(head_dim)) V[h div g].
+ * The descriptor appends nothing (n_new_total = 0).  A slab is read once per new token, from
+ * L2 after the first; packing several tokens of a chunk into one tensor-core tile is not done. */
+int32_t odma_build_prefill_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                                  void* d_table, uint64_t table_bytes, void* stream, odma_tables* out);
 
 /* ---- KV append (the per-step growth of each request's cache, Section II-A) --------------
  * Writes the step's new K and V rows of `layer` behind each request's existing tokens:

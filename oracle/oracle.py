@@ -257,6 +257,27 @@ class KVStore:
                                 threads, want_lse)
 
 
+def prefill_attention(store: "KVStore", layer: int, reqs: Sequence[int], n_new: Sequence[int], q, q_heads: int,
+                      threads: int = 0):
+    """Causal attention of a prefill chunk, by its definition: the store already holds the chunk;
+    new token j of request i (its n_new[i] last tokens) attends keys [0, its own position].  q:
+    [sum(n_new), Hq, D], tokens in request order then position order.  Each token is one dense
+    fp64 attention over a prefix of the request's rows.  Returns (out [sum(n_new), Hq, D], lse)."""
+    Ks, Vs = [], []
+    for r, k in zip(reqs, n_new):
+        K, V = store.gathered(r, layer)
+        L = K.shape[0]
+        for j in range(k):
+            Ks.append(K[: L - k + j + 1])
+            Vs.append(V[: L - k + j + 1])
+    if store.kv_e4m3:
+        out, lse, _ = decode_attention_e4m3(q, store.dtype, Ks, Vs, store.k_scale[layer], store.v_scale[layer], q_heads,
+                                            store.kv_heads, store.head_dim, threads, True)
+    else:
+        out, lse, _ = decode_attention(q, Ks, Vs, q_heads, store.kv_heads, store.head_dim, store.dtype, threads, True)
+    return out, lse
+
+
 # ---------------------------------------------------------------------------
 # allocator
 # ---------------------------------------------------------------------------

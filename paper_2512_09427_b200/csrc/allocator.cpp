@@ -125,9 +125,99 @@ int32_t Allocator::init(uint64_t bytes, int32_t layers, int32_t kv_heads, int32_
     n_bounds_ = 1;
     bounds_[0] = cfg.max_len;
     epoch_ = 0;
+    applied_ = 0;
+    outbox_.clear();
+    if (cfg.async_recal < 0 || cfg.async_recal > 1 || cfg.cluster_observe < 0 || cfg.cluster_observe > 1)
+        return ODMA_ERR_INVALID;
+    if (cfg.async_recal) {
+        async_.reset(new Async());
+        async_->th = std::thread([this] { worker(); });
+    }
     observed_ = completed_ = sum_len_ = sum_cap_ = migrations_ = nomem_ = routed_large_ = 0;
     safety_peak_ = reserved_live_ = used_live_ = 0;
     return ODMA_OK;
+}
+
+Allocator::~Allocator() {
+    if (async_) {
+        {
+            std::lock_guard<std::mutex> g(async_->mu);
+            async_->stop = true;
+        }
+        async_->work.notify_all();
+        if (async_->th.joinable()) async_->th.join();
+    }
+}
+
+// Background refresh (Sections III-E and IV-C: histogram updates and boundary refreshes run off
+// the critical path; new boundaries reach newly admitted requests only, which holds by
+// construction: a slab is sized once, at admission).  The thread applies the logged lengths in
+// order, so at quiescence the boundaries are those the synchronous path would have.
+void Allocator::worker() {
+    Async& a = *async_;
+    std::unique_lock<std::mutex> lk(a.mu);
+    for (;;) {
+        a.work.wait(lk, [&] { return a.stop || !a.log.empty(); });
+        if (a.log.empty()) {
+            if (a.stop) return;
+            continue;
+        }
+        const int32_t len = a.log.front();
+        a.log.pop_front();
+        a.busy = true;
+        lk.unlock();
+        apply_observation(len);
+        lk.lock();
+        a.busy = false;
+        if (a.log.empty()) a.idle.notify_all();
+    }
+}
+
+void Allocator::flush() {
+    if (!async_) return;
+    std::unique_lock<std::mutex> lk(async_->mu);
+    async_->idle.wait(lk, [&] { return async_->log.empty() && !async_->busy; });
+}
+
+void Allocator::apply_observation(int32_t len) {
+    window_.push(len);
+    applied_ += 1;
+    if (applied_ % cfg_.refresh == 0) recalibrate();
+}
+
+void Allocator::note_observation(int32_t len) {
+    observed_ += 1;
+    if (async_) {
+        {
+            std::lock_guard<std::mutex> g(async_->mu);
+            async_->log.push_back(len);
+        }
+        async_->work.notify_one();
+    } else {
+        apply_observation(len);
+    }
+}
+
+int32_t Allocator::observe(const int32_t* lengths, int32_t n) {
+    if (n < 0 || (n > 0 && !lengths)) return ODMA_ERR_INVALID;
+    for (int32_t i = 0; i < n; ++i)
+        if (lengths[i] < 0 || lengths[i] > cfg_.max_len) return ODMA_ERR_INVALID;
+    for (int32_t i = 0; i < n; ++i) note_observation(lengths[i]);
+    return ODMA_OK;
+}
+
+int32_t Allocator::drain(int32_t* out, int32_t cap, int32_t* n) {
+    if (!n || cap < 0 || (cap > 0 && !out)) return ODMA_ERR_INVALID;
+    const int32_t k = static_cast<int32_t>(std::min<size_t>(outbox_.size(), static_cast<size_t>(cap)));
+    std::copy(outbox_.begin(), outbox_.begin() + k, out);
+    outbox_.erase(outbox_.begin(), outbox_.begin() + k);
+    *n = k;
+    return ODMA_OK;
+}
+
+uint64_t Allocator::epoch() const {
+    std::lock_guard<std::mutex> g(bounds_mu_);
+    return epoch_;
 }
 
 int32_t Allocator::set_buckets(const int32_t* b, int32_t n) {
@@ -136,6 +226,7 @@ int32_t Allocator::set_buckets(const int32_t* b, int32_t n) {
         if (b[i] < 1 || b[i] % G_ != 0 || b[i] > cfg_.max_len) return ODMA_ERR_INVALID;
         if (i > 0 && b[i] <= b[i - 1]) return ODMA_ERR_INVALID;
     }
+    std::lock_guard<std::mutex> g(bounds_mu_);
     for (int i = 0; i < n; ++i) bounds_[i] = b[i];
     n_bounds_ = n;
     epoch_ += 1;
@@ -144,6 +235,7 @@ int32_t Allocator::set_buckets(const int32_t* b, int32_t n) {
 
 int32_t Allocator::get_buckets(int32_t* b, int32_t* n, uint64_t* epoch) const {
     if (!b || !n) return ODMA_ERR_INVALID;
+    std::lock_guard<std::mutex> g(bounds_mu_);
     for (int i = 0; i < n_bounds_; ++i) b[i] = static_cast<int32_t>(bounds_[i]);
     *n = n_bounds_;
     if (epoch) *epoch = epoch_;
@@ -161,7 +253,7 @@ void Allocator::fill(const Request& r, odma_slab* out) const {
     out->cap_tok = static_cast<int32_t>(r.cap);
     out->pool_id = r.pool;
     out->bucket_id = r.bucket;
-    out->epoch = epoch_;
+    out->epoch = epoch();
 }
 
 void Allocator::note_safety_peak() {
@@ -190,7 +282,7 @@ int32_t Allocator::reserve_large(uint64_t req, int64_t need, odma_slab* out) {
     r.cap = cap;
     r.pool = 1;
     r.bucket = -1;
-    r.epoch = epoch_;
+    r.epoch = epoch();
     live_[req] = r;
     reserved_live_ += cap;
     routed_large_ += 1;
@@ -202,11 +294,21 @@ int32_t Allocator::reserve_large(uint64_t req, int64_t need, odma_slab* out) {
 int32_t Allocator::reserve(uint64_t req, int64_t predicted, odma_slab* out) {
     if (predicted < 1) return ODMA_ERR_INVALID;
     if (live_.count(req)) return ODMA_ERR_DUP_REQ;
-    if (predicted > bounds_[n_bounds_ - 1] || predicted > cfg_.max_len)
+    // one consistent view of the boundaries (a background refresh may replace them at any moment)
+    int64_t bnd[ODMA_MAX_BUCKETS];
+    int32_t nb;
+    uint64_t ep;
+    {
+        std::lock_guard<std::mutex> g(bounds_mu_);
+        nb = n_bounds_;
+        for (int i = 0; i < nb; ++i) bnd[i] = bounds_[i];
+        ep = epoch_;
+    }
+    if (predicted > bnd[nb - 1] || predicted > cfg_.max_len)
         return reserve_large(req, std::min<int64_t>(predicted, cfg_.max_len), out);
     int bi = 0;
-    while (bounds_[bi] < predicted) ++bi;      // first boundary that holds the request
-    const int64_t cap = bounds_[bi];
+    while (bnd[bi] < predicted) ++bi;          // first boundary that holds the request
+    const int64_t cap = bnd[bi];
     const int64_t base = main_.take(cap);
     if (base < 0) {
         nomem_ += 1;
@@ -217,7 +319,7 @@ int32_t Allocator::reserve(uint64_t req, int64_t predicted, odma_slab* out) {
     r.cap = cap;
     r.pool = 0;
     r.bucket = bi;
-    r.epoch = epoch_;
+    r.epoch = ep;
     live_[req] = r;
     reserved_live_ += cap;
     fill(r, out);
@@ -287,12 +389,15 @@ int32_t Allocator::commit(const uint64_t* reqs, int32_t n, const int32_t* n_new)
 
 void Allocator::recalibrate() {
     const int64_t n = window_.count();
+    int64_t fresh[ODMA_MAX_BUCKETS];
     for (int i = 0; i < cfg_.n_levels; ++i) {
         int64_t rank = (static_cast<int64_t>(cfg_.p_num[i]) * n + cfg_.p_den - 1) / cfg_.p_den;
         rank = std::min(std::max<int64_t>(rank, 1), n);
         const int64_t b = ceil_g(window_.order_statistic(rank), G_);
-        bounds_[i] = std::min<int64_t>(b, cfg_.max_len);
+        fresh[i] = std::min<int64_t>(b, cfg_.max_len);
     }
+    std::lock_guard<std::mutex> g(bounds_mu_);
+    for (int i = 0; i < cfg_.n_levels; ++i) bounds_[i] = fresh[i];
     n_bounds_ = cfg_.n_levels;
     epoch_ += 1;
 }
@@ -308,9 +413,11 @@ int32_t Allocator::release(uint64_t req) {
     completed_ += 1;
     sum_len_ += r.len;
     sum_cap_ += r.cap;
-    window_.push(static_cast<int32_t>(r.len));
-    observed_ += 1;
-    if (observed_ % cfg_.refresh == 0) recalibrate();
+    // the realised length: into the window here, or (cluster_observe) only into the outbox, from
+    // where the cluster's exchange brings every replica's lengths into every window in one order
+    outbox_.push_back(static_cast<int32_t>(r.len));
+    if (outbox_.size() > static_cast<size_t>(cfg_.window)) outbox_.erase(outbox_.begin());
+    if (!cfg_.cluster_observe) note_observation(static_cast<int32_t>(r.len));
     return ODMA_OK;
 }
 
@@ -330,7 +437,7 @@ void Allocator::stats(odma_stats* out) const {
     out->safety_live = S_ - safety_.free_tokens();
     out->safety_peak = safety_peak_;
     out->observed = observed_;
-    out->epoch = epoch_;
+    out->epoch = epoch();
 }
 
 }  // namespace odma

@@ -381,6 +381,8 @@ void odma_config_default(odma_config* cfg) {
     cfg->fused_combine = 1;
     cfg->fused_append = 1;
     cfg->decode_kernel = ODMA_DECODE_AUTO;
+    cfg->async_recal = 0;
+    cfg->cluster_observe = 0;
 }
 
 const char* odma_strerror(int32_t code) {
@@ -493,6 +495,20 @@ int32_t odma_pool_destroy(odma_pool* pool) {
     return ODMA_OK;
 }
 
+int32_t odma_recal_flush(odma_pool* pool) {
+    if (!pool) return ODMA_ERR_INVALID;
+    pool->alloc.flush();
+    return ODMA_OK;
+}
+
+int32_t odma_drain_observations(odma_pool* pool, int32_t* out, int32_t cap, int32_t* n) {
+    return pool ? pool->alloc.drain(out, cap, n) : ODMA_ERR_INVALID;
+}
+
+int32_t odma_observe(odma_pool* pool, const int32_t* lengths, int32_t n) {
+    return pool ? pool->alloc.observe(lengths, n) : ODMA_ERR_INVALID;
+}
+
 int32_t odma_set_kv_scales(odma_pool* pool, const float* k_scale, const float* v_scale) {
     if (!pool || !k_scale || !v_scale || pool->dtype != ODMA_DTYPE_FP8_E4M3) return ODMA_ERR_INVALID;
     for (int32_t l = 0; l < pool->layers; ++l)
@@ -593,6 +609,58 @@ int32_t odma_build_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* 
     st.in_flight = false;
     int32_t rc = plan_into(pool, reqs, n_new, n, st.host, static_cast<uint64_t>(pool->table_words_max) * 4, out);
     if (rc != ODMA_OK) return rc;
+    if (cudaMemcpyAsync(d_table, st.host, static_cast<size_t>(out->words) * 4, cudaMemcpyHostToDevice,
+                        as_stream(stream)) != cudaSuccess ||
+        cudaEventRecord(st.done, as_stream(stream)) != cudaSuccess)
+        return ODMA_ERR_CUDA;
+    st.in_flight = true;
+    out->d_table = d_table;
+    return ODMA_OK;
+}
+
+int32_t odma_build_prefill_tables(odma_pool* pool, const uint64_t* reqs, const int32_t* n_new, int32_t n,
+                                  void* d_table, uint64_t table_bytes, void* stream, odma_tables* out) {
+    if (!pool || !pool->dev_base || !d_table || !aligned16(d_table) || !reqs || !n_new || !out || n < 1)
+        return ODMA_ERR_INVALID;
+    // one stream per new token: the owner's slab, read up to and including the token itself
+    int64_t total = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        if (n_new[i] < 1) return ODMA_ERR_INVALID;
+        total += n_new[i];
+    }
+    if (total > pool->alloc.config().max_batch || table_bytes < odma_tables_bytes(pool, static_cast<int32_t>(total)))
+        return ODMA_ERR_INVALID;
+    pool->v_base.clear();
+    pool->v_cap.clear();
+    pool->v_len.clear();
+    for (int32_t i = 0; i < n; ++i) {
+        const Request* r = pool->alloc.find(reqs[i]);
+        if (!r) return ODMA_ERR_UNKNOWN_REQ;
+        if (r->len + n_new[i] > r->cap) return ODMA_ERR_OVERFLOW;
+        for (int32_t j = 0; j < n_new[i]; ++j) {
+            pool->v_base.push_back(static_cast<int32_t>(r->base));
+            pool->v_cap.push_back(static_cast<int32_t>(r->cap));
+            pool->v_len.push_back(static_cast<int32_t>(r->len + j + 1));
+        }
+    }
+    Staging& st = pool->staging[pool->staging_next];
+    pool->staging_next = (pool->staging_next + 1) % kStagingSlots;
+    if (st.in_flight && cudaEventSynchronize(st.done) != cudaSuccess) return ODMA_ERR_CUDA;
+    st.in_flight = false;
+    PlanInput in;
+    in.n = static_cast<int32_t>(total);
+    in.kv_heads = pool->kv_heads;
+    in.n_ctas = pool->plan_ctas;
+    in.base = pool->v_base.data();
+    in.cap = pool->v_cap.data();
+    in.len = pool->v_len.data();
+    in.n_new = nullptr;
+    pool->plan_cache.valid = false;                  // the scratch vectors no longer describe the cached batch
+    int32_t rc = plan_batch(in, st.host, pool->table_words_max, out);
+    if (rc != ODMA_OK) return rc;
+    out->epoch = pool->alloc.epoch();
+    out->n_new_total = 0;                            // nothing to append through this descriptor
+    out->one_new_each = 0;
     if (cudaMemcpyAsync(d_table, st.host, static_cast<size_t>(out->words) * 4, cudaMemcpyHostToDevice,
                         as_stream(stream)) != cudaSuccess ||
         cudaEventRecord(st.done, as_stream(stream)) != cudaSuccess)

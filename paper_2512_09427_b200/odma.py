@@ -33,7 +33,7 @@ class Config(C.Structure):
                 ("gamma_permille", C.c_int32), ("tau_permille", C.c_int32), ("growth", C.c_int32),
                 ("large_fixed", C.c_int32), ("max_batch", C.c_int32), ("max_group", C.c_int32),
                 ("plan_ctas", C.c_int32), ("fused_combine", C.c_int32), ("fused_append", C.c_int32),
-                ("decode_kernel", C.c_int32)]
+                ("decode_kernel", C.c_int32), ("async_recal", C.c_int32), ("cluster_observe", C.c_int32)]
 
 
 class Slab(C.Structure):
@@ -91,6 +91,9 @@ _SIGS = {
     "odma_strerror": (C.c_char_p, [_i32]),
     "odma_pool_create": (_i32, [_vp, _u64, _i32, _i32, _i32, _i32, C.POINTER(Config), C.POINTER(_vp)]),
     "odma_pool_destroy": (_i32, [_vp]),
+    "odma_recal_flush": (_i32, [_vp]),
+    "odma_drain_observations": (_i32, [_vp, _i32p, _i32, _i32p]),
+    "odma_observe": (_i32, [_vp, _i32p, _i32]),
     "odma_set_kv_scales": (_i32, [_vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]),
     "odma_set_buckets": (_i32, [_vp, _i32p, _i32]),
     "odma_get_buckets": (_i32, [_vp, _i32p, _i32p, _u64p]),
@@ -104,6 +107,7 @@ _SIGS = {
     "odma_tables_bytes": (_u64, [_vp, _i32]),
     "odma_plan_host": (_i32, [_vp, _u64p, _i32p, _i32, _i32p, _u64, C.POINTER(Tables)]),
     "odma_build_tables": (_i32, [_vp, _u64p, _i32p, _i32, _vp, _u64, _vp, C.POINTER(Tables)]),
+    "odma_build_prefill_tables": (_i32, [_vp, _u64p, _i32p, _i32, _vp, _u64, _vp, C.POINTER(Tables)]),
     "odma_append_kv": (_i32, [_vp, _i32, C.POINTER(Tables), _vp, _vp, _vp]),
     "odma_decode_attention": (_i32, [_vp, _i32, _vp, _i32, C.POINTER(Tables), _vp, _vp, _vp]),
     "odma_decode_step_host": (_i32, [_vp, _i32, _i32, _u64p, _i32, _vp, _vp, _vp, _vp, _vp]),
@@ -180,6 +184,19 @@ class Pool:
         except Exception:
             pass
 
+    def recal_flush(self) -> None:
+        _check(_lib.odma_recal_flush(self._h), "odma_recal_flush")
+
+    def drain_observations(self, cap: int = 1 << 20) -> list:
+        """Lengths of the requests completed here since the last drain (oldest first)."""
+        buf = (C.c_int32 * cap)()
+        n = C.c_int32()
+        _check(_lib.odma_drain_observations(self._h, buf, cap, C.byref(n)), "odma_drain_observations")
+        return list(buf[: n.value])
+
+    def observe(self, lengths: Sequence[int]) -> None:
+        _check(_lib.odma_observe(self._h, _i32arr(list(lengths)), len(lengths)), "odma_observe")
+
     def set_kv_scales(self, k_scale: Sequence[float], v_scale: Sequence[float]) -> None:
         """Per-layer dequantisation scales of an 8-bit (E4M3) pool."""
         assert len(k_scale) == self.layers and len(v_scale) == self.layers
@@ -247,6 +264,14 @@ class Pool:
         t = Tables()
         _check(_lib.odma_build_tables(self._h, _u64arr(reqs), _i32arr(n_new), len(reqs), d_table,
                                       table_bytes, stream or None, C.byref(t)), "odma_build_tables")
+        return t
+
+    def build_prefill_tables(self, reqs: Sequence[int], n_new: Sequence[int], d_table: int, table_bytes: int,
+                             stream: int = 0) -> Tables:
+        """Plan of the causal attention of a prefill chunk: one stream per new token."""
+        t = Tables()
+        _check(_lib.odma_build_prefill_tables(self._h, _u64arr(reqs), _i32arr(n_new), len(reqs), d_table,
+                                              table_bytes, stream or None, C.byref(t)), "odma_build_prefill_tables")
         return t
 
     # -- kernels -----------------------------------------------------------------------------

@@ -219,3 +219,29 @@ def test_kv_store_keeps_append_order():
     k, v = st.gathered(5, 0)
     assert st.length(5) == 4
     assert np.array_equal(k, torch.cat([a, b]).numpy()) and np.array_equal(v, 2 * torch.cat([a, b]).numpy())
+
+
+def test_prefill_chunk_is_causal_attention():
+    """The chunk form against an independent library's masked attention in fp64: token j of the
+    chunk sees the context and the chunk's tokens up to itself."""
+    rng = np.random.default_rng(21)
+    Hq, Hkv, D, ctx, chunk = 4, 2, 16, 11, 7
+    K = rng.standard_normal((ctx + chunk, Hkv, D)).astype(np.float32)
+    V = rng.standard_normal((ctx + chunk, Hkv, D)).astype(np.float32)
+    q = rng.standard_normal((chunk, Hq, D)).astype(np.float32)
+    st = ora.KVStore(1, Hkv, D, ora.F32)
+    st.append(5, 0, K[:ctx], V[:ctx])
+    st.append(5, 0, K[ctx:], V[ctx:])
+    out, lse = ora.prefill_attention(st, 0, [5], [chunk], q, Hq)
+    qt = torch.from_numpy(q).double().permute(1, 0, 2)                        # [Hq, chunk, D]
+    kt = torch.from_numpy(K).double().permute(1, 0, 2).repeat_interleave(Hq // Hkv, 0)
+    vt = torch.from_numpy(V).double().permute(1, 0, 2).repeat_interleave(Hq // Hkv, 0)
+    mask = torch.arange(ctx + chunk)[None, :] <= (ctx + torch.arange(chunk))[:, None]
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask).permute(1, 0, 2).numpy()
+    assert np.max(np.abs(out - ref)) < 1e-12
+    # a fresh prompt's first token attends itself alone
+    st2 = ora.KVStore(1, Hkv, D, ora.F32)
+    st2.append(1, 0, K[:3], V[:3])
+    o2, l2 = ora.prefill_attention(st2, 0, [1], [3], q[:3], Hq)
+    for h in range(Hq):
+        assert np.allclose(o2[0, h], V[0, h // (Hq // Hkv)], rtol=0, atol=1e-15)
