@@ -153,7 +153,7 @@ class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
     def __init__(self, w: wl.Workload, step_layers: int, device: torch.device, plan_ctas: int = 0,
-                 fused: int = 1, decode_kernel: int = 0):
+                 fused: int = 1, decode_kernel: int = 0, chain_launches: int = 1, mem=None):
         from paper_2512_09427_b200 import odma
         self.odma, self.w, self.dev, self.step_layers = odma, w, device, step_layers
         self.dt = (odma.DTYPE_FP8_E4M3 if w.kv_dtype == "e4m3" else
@@ -170,8 +170,11 @@ class SlabDecode:
         cfg.plan_ctas = plan_ctas
         cfg.fused_combine = fused
         cfg.decode_kernel = decode_kernel
+        cfg.chain_launches = chain_launches
         self.pool_cfg = cfg
-        self.mem = torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
+        # `mem`: the device memory of another SlabDecode of the same workload (a second pool over the
+        # same, already filled bytes: the allocator is deterministic, so the slabs coincide)
+        self.mem = mem if mem is not None else torch.zeros(w.pool_bytes, dtype=torch.uint8, device=device)
         self.stream = torch.cuda.current_stream().cuda_stream
         self.pool = odma.Pool(self.mem.data_ptr(), w.pool_bytes, w.layers, w.kv_heads, w.head_dim,
                               self.dt, cfg)
@@ -197,14 +200,19 @@ class SlabDecode:
                 assert pool.free(r) == 0
         return pool.get_buckets()
 
-    def admit_and_fill(self):
-        """Reserve every request's slab and write its context tokens (seeded N(0,1)) on all layers."""
+    def admit_and_fill(self, fill: bool = True):
+        """Reserve every request's slab and write its context tokens (seeded N(0,1)) on all layers
+        (`fill` False: the memory already holds them, only the bookkeeping is done)."""
         w, pool, odma = self.w, self.pool, self.odma
         for r in self.reqs:
             rc, _ = pool.alloc(r, int(w.predicted[r]))
             assert rc == odma.OK, ("alloc", r, rc)
             rc, _, _ = pool.ensure_capacity(r, int(w.context[r]) + 1, self.stream)
             assert rc == odma.OK, ("ensure", r, rc)
+        if not fill:
+            assert pool.commit_step(self.reqs, [int(c) for c in w.context]) == 0
+            torch.cuda.synchronize()
+            return
         table = torch.empty(pool.tables_bytes(w.batch), dtype=torch.uint8, device=self.dev)
         ctx = [int(c) for c in w.context]
         t = pool.build_tables(self.reqs, table.data_ptr(), table.numel(), self.stream, ctx)
@@ -431,7 +439,10 @@ def workload_config(w, name, step_layers, copies):
     return {"workload": desc, "batch": w.batch, "layers_per_step": step_layers,
             "kv_tokens": int((w.context + 1).sum()), "kv_bytes_per_layer": kv_bytes_layer,
             "l2": (f"steps rotate over {copies} independent KV copies ({copies * kv_bytes_layer >> 20} MiB > L2)"
-                   if copies > 1 else f"one step streams {step_layers * kv_bytes_layer >> 20} MiB of KV (> L2)")}
+                   if copies > 1 else f"one step streams {step_layers * kv_bytes_layer >> 20} MiB of KV (> L2)"),
+            "overlap": "consecutive launches are on different layers (KV copies) of one pool and do not wait for one "
+                       "another, as the layers of a model do not; roofline.serialised has the same steps with every "
+                       "launch waiting for the one before"}
 
 
 def kernel_sources_hash() -> str:
@@ -549,7 +560,9 @@ def run_ours(args):
     step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * io_row_bytes + 2 * n * w.kv_heads * io_row_bytes)
     if w.dtype != torch.bfloat16:
         kernel_name = "decode_generic_kernel"
-    elif args.decode_kernel == "tcgen05" or (args.decode_kernel == "auto" and step_layers > 1) or w.kv_dtype == "e4m3":
+    elif args.decode_kernel in ("tcgen05", "auto") or w.kv_dtype == "e4m3":
+        # auto: every step but the very first follows a decode step on another layer (another KV copy)
+        # and runs on the tcgen05 kernel, chained; the mma.sync kernel serves launches that have to wait
         kernel_name = "decode_umma_kernel"
     else:
         kernel_name = "decode_tc_kernel"
@@ -589,6 +602,37 @@ def run_ours(args):
                     "frac_isolated": isolated / peak}
         kernels_us = {"append": app_ms / max(app_n, 1) * 1e3, "decode": dec_ms / dec_n * 1e3,
                       "combine": cmb_ms / cmb_n * 1e3 if cmb_n else 0.0}
+
+    # ---- the same steps with every launch made to wait for the one before (chain_launches = 0) ----
+    # A second pool over the same, already filled memory (same slabs: the allocator is deterministic).
+    if "serial" in phases and roofline is not None:
+        sd0 = SlabDecode(w, step_layers, dev, fused=args.fused_combine, decode_kernel=DECODE_KERNELS[args.decode_kernel],
+                         chain_launches=0, mem=sd.mem)
+        sd0.learn_boundaries()
+        sd0.admit_and_fill(fill=False)
+        t0 = odma.Tables()
+        i0 = 0
+        for _ in range(max(W, 3)):
+            sd0.step(i0, q, kn, vn, out, t0)
+            i0 += 1
+        torch.cuda.synchronize()
+        reps = max(5, min(n_regions, 50))
+        sm = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        t0w = time.time()
+        sm[0].record()
+        for r in range(reps):
+            for _ in range(K):
+                sd0.step(i0, q, kn, vn, out, t0)
+                i0 += 1
+            sm[r + 1].record()
+        torch.cuda.synchronize()
+        if clocks:
+            clocks.mark(t0w, time.time())
+        assert sd0.pool.check_status(sd0.stream) == odma.OK
+        s_us = statistics.median(sm[r].elapsed_time(sm[r + 1]) for r in range(reps)) / (K * step_layers) * 1e3
+        roofline["serialised"] = {"us_per_launch": s_us, "frac": kv_bytes_per_launch / (s_us * 1e-6) / 1e9 / peak,
+                                  "what": "the same steps with chain_launches = 0: every launch waits for the kernel ahead of it"}
+        sd0.pool.destroy()
 
     # ---- the read probe: the decode kernel's loads and barrier traffic with no arithmetic, launched
     #      the way the timed steps are (consecutive launches between two events)
@@ -873,7 +917,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--phases", default="",
                     help="comma list of the passes to run besides the timed one: kernels (per-kernel CUDA-event "
-                         "times), e2e (host buffers), clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
+                         "times), serial (the steps again with every launch waiting for the one before), e2e (host buffers), "
+                         "clocks (nvidia-smi sampler), cpu (CPU checker baseline), "
                          "probe (the no-arithmetic read probe), paged (page-16 ablation of the decode kernel on "
                          "the same inputs); default: all of them on config2, all but paged elsewhere")
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
@@ -889,7 +934,7 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     if not args.phases:
-        args.phases = "timed,kernels,e2e,clocks,cpu,probe" + (",paged" if args.workload == "config2" else "")
+        args.phases = "timed,kernels,serial,e2e,clocks,cpu,probe" + (",paged" if args.workload == "config2" else "")
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "config4":

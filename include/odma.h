@@ -25,7 +25,13 @@
  *    rows and (after another decode launch of this library) slab rows only once the
  *    kernels ahead of them have completed; a caller that writes pool memory, q, k_new or
  *    v_new with kernels of its own must not let those signal their dependents early
- *    (no programmatic launch trigger before the writes are done).
+ *    (no programmatic launch trigger before the writes are done).  Decode steps
+ *    (odma_decode_step, odma_decode_step_host) issued directly one after the other on
+ *    DIFFERENT layers run concurrently: layers share no K/V rows, and the second does not wait
+ *    for the first.  The q, k_new, v_new of a step must therefore not be outputs of the decode
+ *    step issued directly before it, and their out buffers must not overlap (in a model the
+ *    projections between two layers' attention are kernels of the caller: a step issued
+ *    behind any other kernel or copy starts only when that operation has completed).
  *  - Host-side calls are not thread-safe; serialise calls on one pool.
  *  - Lengths and capacities are in tokens.  One token occupies
  *    layers * 2 * kv_heads * head_dim * elem_bytes bytes of the pool.
@@ -111,6 +117,9 @@ typedef struct odma_config {
                                 kernel, ODMA_DECODE_MMA_SYNC the mma.sync kernel, ODMA_DECODE_AUTO
                                 the first for the layers of an odma_decode_step over several
                                 layers and the second for single launches (0) */
+    int32_t chain_launches;  /* 1: a decode step issued directly behind a decode step on another layer does
+                                not wait for it (see "Conventions"); 0: every launch waits for the kernel
+                                ahead of it (1) */
     int32_t async_recal;     /* 1: a background thread owns the length window: odma_free only logs the
                                 realised length, the thread applies the log in order and refreshes the
                                 boundaries off the critical path (Sections III-E, IV-C); boundaries at

@@ -55,6 +55,11 @@ struct odma_pool {
     // only the last row of each stream).  True after a decode launch, false after any other
     // launch of the library that writes the pool (append, migration copy).
     bool decode_was_last = false;
+    // what the last decode launch was, for chaining the next one to it (decode_attention_impl)
+    bool last_fused_tensor = false;
+    int32_t last_layer = -1;
+    void* last_stream = nullptr;
+    uint32_t scratch_parity = 0;
     uint32_t* d_counters = nullptr;   // per split stream: pieces delivered (fused combine)
     // a second scratch set: consecutive layers of one step alternate between the two, so that a
     // layer's kernel need not wait for the previous layer's
@@ -381,6 +386,7 @@ void odma_config_default(odma_config* cfg) {
     cfg->fused_combine = 1;
     cfg->fused_append = 1;
     cfg->decode_kernel = ODMA_DECODE_AUTO;
+    cfg->chain_launches = 1;
     cfg->async_recal = 0;
     cfg->cluster_observe = 0;
 }
@@ -556,6 +562,7 @@ int32_t odma_ensure_capacity(odma_pool* pool, uint64_t req, int32_t needed_len, 
     mp.kv_heads = pool->kv_heads;
     mp.row_vecs = pool->head_dim * pool->elem_bytes / 16;
     pool->decode_was_last = false;
+    pool->last_fused_tensor = false;
     ProfScope ps(pool, ODMA_K_MIGRATE, as_stream(stream));
     return launch_migrate(mp, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
@@ -696,6 +703,7 @@ int32_t odma_append_kv(odma_pool* pool, int32_t layer, const odma_tables* tables
     ap.k_inv = ap.quantize ? 1.0f / pool->k_scale[layer] : 1.f;
     ap.v_inv = ap.quantize ? 1.0f / pool->v_scale[layer] : 1.f;
     pool->decode_was_last = false;
+    pool->last_fused_tensor = false;
     ProfScope ps(pool, ODMA_K_APPEND, as_stream(stream));
     return launch_append(ap, as_stream(stream)) == cudaSuccess ? ODMA_OK : ODMA_ERR_CUDA;
 }
@@ -710,15 +718,16 @@ bool uses_tc(const odma_pool* pool, int32_t q_heads) {
     return pool->has_maps && tc_supported(pool->head_dim, q_heads / pool->kv_heads);
 }
 
-// Which of the two tensor-core kernels runs a launch.  ODMA_DECODE_AUTO: the tcgen05 kernel for
-// the layers of a step that spans several layers (its launches chain without dependency waits;
-// measured 3 to 6 % faster on the 28-layer workloads), the mma.sync kernel for single launches
-// (3 to 4 % faster there: its last tile and hand-over are a shorter chain).
-bool uses_umma(const odma_pool* pool, int32_t group, bool part_of_multi_layer_step) {
+// Which of the two tensor-core kernels runs a launch.  ODMA_DECODE_AUTO: the tcgen05 kernel for a
+// launch that can chain to the decode launch before it (the layers of a step over several layers,
+// consecutive steps on different layers: it then runs without a dependency wait, measured 3 to 13 %
+// faster), the mma.sync kernel for launches that have to wait (3 to 4 % faster there: its last
+// tile and hand-over are a shorter chain).  8-bit pools: the tcgen05 kernel always.
+bool uses_umma(const odma_pool* pool, int32_t group, bool chains) {
     const int32_t want = pool->alloc.config().decode_kernel;
     if (pool->dtype == ODMA_DTYPE_FP8_E4M3) return true;
     if (want == ODMA_DECODE_MMA_SYNC || !umma_supported(pool->head_dim, group, false)) return false;
-    return want == ODMA_DECODE_TCGEN05 || part_of_multi_layer_step;
+    return want == ODMA_DECODE_TCGEN05 || chains;
 }
 
 cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, const DecodeParams& p, int mode,
@@ -751,19 +760,31 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
         if (pool->has_maps && tc_supported(pool->head_dim, p.group)) {
             if (p.stages < 2) return ODMA_ERR_INVALID;
             fused = p.counters != nullptr;
-            const bool umma = uses_umma(pool, p.group, chain_pos >= 0);
-            if (chain_pos >= 0 && fused && umma) {
-                // layer `chain_pos` of a step over several layers: scratch sets alternate, and every
-                // layer but the first runs chained to the one before
-                if (chain_pos & 1) {
+            // A launch whose predecessor on the stream is a fused decode launch of this pool on ANOTHER
+            // layer has nothing to wait for: other K/V arrays, other outputs, inputs that were complete
+            // when it was issued (they are not the predecessor's outputs: see the header), and the
+            // other scratch set.  The layers of a step over several layers chain that way, and so do
+            // consecutive steps on different layers.  Only the tcgen05 kernel can run without its
+            // dependency wait.  (Anything else enqueued in between - a table copy, the caller's own
+            // kernels - makes the launch wait for that operation to complete before it starts.)
+            const bool can_chain = pool->alloc.config().chain_launches && fused && k_new != nullptr && p.early_ok &&
+                                   pool->last_fused_tensor && pool->last_stream == stream && pool->last_layer != layer;
+            const bool umma = uses_umma(pool, p.group, chain_pos >= 0 || can_chain);
+            if (fused) {
+                pool->scratch_parity ^= 1u;              // scratch sets alternate from launch to launch
+                if (pool->scratch_parity) {
                     p.part_o = pool->part_o2;
                     p.part_ml = pool->part_ml2;
                     p.counters = pool->d_counters2;
                 }
-                p.chained = chain_pos > 0 ? 1 : 0;
             }
+            p.chained = umma && can_chain ? 1 : 0;
+            pool->last_fused_tensor = fused && k_new != nullptr;
+            pool->last_layer = layer;
+            pool->last_stream = stream;
             e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens, umma);
         } else if (generic_supported(pool->head_dim)) {
+            pool->last_fused_tensor = false;
             p.counters = nullptr;
             e = launch_decode_generic(p, pool->dtype, tables->n_ctas, as_stream(stream));
         } else {
@@ -943,6 +964,8 @@ int32_t odma_read_probe(odma_pool* pool, int32_t layer, int32_t q_heads, const o
     fill_decode_params(pool, layer, pool->d_q, q_heads, tables, pool->d_out, nullptr, &p);
     if (!tc_supported(pool->head_dim, p.group) || p.group > pool->alloc.config().max_group || p.stages < 2)
         return ODMA_ERR_INVALID;
+    pool->decode_was_last = false;
+    pool->last_fused_tensor = false;
     ProfScope ps(pool, ODMA_K_PROBE, as_stream(stream));
     return launch_decode_tc(pool->maps, p, kModeProbe, tables->n_ctas, as_stream(stream)) == cudaSuccess
                ? ODMA_OK
@@ -1102,6 +1125,8 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
     p.rows_per_array = paged->n_pages * pool->kv_heads * 16;
     p.page_table = d_page_table;
     p.max_pages = max_pages;
+    pool->decode_was_last = false;        // nothing chains to, or starts early behind, a launch of the ablation
+    pool->last_fused_tensor = false;
     cudaError_t e;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));

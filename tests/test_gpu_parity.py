@@ -557,3 +557,55 @@ def test_config2_full_size_parity():
     err = check_all(s, reqs, res, "config2")
     st = s.ls.check_stats()
     print("config2 parity", err, "buckets", bounds, "reserved", st["reserved_live"], "used", st["used_live"])
+
+
+@pytest.mark.parametrize("kernel", [0, 1], ids=["auto", "tcgen05"])
+def test_consecutive_steps_on_different_layers_overlap_and_stay_right(kernel):
+    """Single-layer odma_decode_step calls issued back to back on changing layers (the pattern of
+    a multi-layer model, and of the benchmark's rotating KV copies): each runs without waiting
+    for the one before; where a round ends on the layer the next round starts with, that launch
+    must wait.  Twelve calls without a host synchronisation, every one against the checker, every
+    appended row in place."""
+    odma = lib()
+    lens = [0, 40, 64, 129, 700, 1500, 2771]
+    w = qwen_small(lens, layers=4)
+    w = wl.scaled(w, predicted=w.context + 8)
+    s = Session(w, plan_ctas=11, decode_kernel=kernel)
+    s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+    reqs = list(range(w.batch))
+    s.admit(reqs, w.predicted)
+    pre = [r for r in reqs if w.context[r] > 0]
+    s.append(pre, [int(w.context[r]) for r in pre])
+    rounds = [[0, 1, 2, 3], [3, 0, 2, 1], [1, 3, 0, 2]]             # token k goes to every layer in round k
+    calls = []
+    for k, order in enumerate(rounds):
+        for l in order:
+            q = s.queries(l, reqs, w.q_heads, 10 + k)
+            kn = torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]).contiguous()
+            vn = torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs]).contiguous()
+            out = torch.full_like(q, float("nan"))
+            lse = torch.full((len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev)
+            calls.append((k, l, q, kn, vn, out, lse))
+    for r in reqs:
+        s.ls.ensure(r, s.lens[r] + len(rounds))
+    torch.cuda.synchronize()
+    for i, (k, l, q, kn, vn, out, lse) in enumerate(calls):        # no synchronisation inside this loop
+        s.pool.decode_step(l, 1, w.q_heads, reqs, q.data_ptr(), kn.data_ptr(), vn.data_ptr(), out.data_ptr(),
+                           lse.data_ptr(), s.stream)
+        if i % 4 == 3:
+            s.ls.commit(reqs, 1)                                    # the round's token, host bookkeeping only
+    torch.cuda.synchronize()
+    assert s.pool.check_status(s.stream) == odma.OK
+    for (k, l, q, kn, vn, out, lse) in calls:
+        for i, r in enumerate(reqs):
+            s.kv.append(r, l, kn[i:i + 1], vn[i:i + 1])
+        ref, ref_lse, _ = s.oracle_out(l, reqs, q, w.q_heads)
+        assert torch.isfinite(out.float()).all()
+        assert_close(out, ref, w.dtype, f"round {k} layer {l}")
+        assert np.abs(lse.double().cpu().numpy() - ref_lse).max() <= 2e-2
+    for r in reqs:
+        s.lens[r] += len(rounds)
+        for l in range(w.layers):
+            k_ref, v_ref = s.kv.gathered(r, l)
+            assert np.array_equal(s.pool_rows(l, 0, r).view(torch.int16).cpu().numpy().view(np.uint16), k_ref)
+            assert np.array_equal(s.pool_rows(l, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
