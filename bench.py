@@ -529,6 +529,14 @@ def run_ours(args):
     for _ in range(W):
         sd.step(step_no, q, kn, vn, out, tables)
         step_no += 1
+    # what one step launches (a step over several layers may be ONE decode launch)
+    sd.pool.profile_enable(True)
+    sd.step(step_no, q, kn, vn, out, tables)
+    step_no += 1
+    torch.cuda.synchronize()
+    dec_per_step = sd.pool.profile_read(odma.K_DECODE)[1]
+    other_per_step = sd.pool.profile_read(odma.K_APPEND)[1] + sd.pool.profile_read(odma.K_COMBINE)[1]
+    sd.pool.profile_enable(False)
     barrier()
     ev0.record()
     for _ in range(max(W, 3)):
@@ -553,11 +561,10 @@ def run_ours(args):
     region_ms = max_over_ranks([marks[r].elapsed_time(marks[r + 1]) for r in range(n_regions)], dist, dev)
     ms = statistics.median(region_ms)
     assert sd.pool.check_status(sd.stream) == odma.OK
-    fused_append = bool(sd.pool_cfg.fused_append) and w.dtype == torch.bfloat16
-    launches_per_step = step_layers * (1 + (0 if fused_append else 1) +
-                                       (1 if tables.n_combine > 0 and not args.fused_combine else 0))
-    kv_bytes_per_launch = tables.kv_tokens * 2 * w.kv_heads * row_bytes
-    step_bytes = step_layers * (kv_bytes_per_launch + 2 * n * w.q_heads * io_row_bytes + 2 * n * w.kv_heads * io_row_bytes)
+    launches_per_step = dec_per_step + other_per_step
+    kv_bytes_layer = tables.kv_tokens * 2 * w.kv_heads * row_bytes
+    kv_bytes_per_launch = kv_bytes_layer * step_layers // dec_per_step     # a launch may cover all layers of the step
+    step_bytes = step_layers * (kv_bytes_layer + 2 * n * w.q_heads * io_row_bytes + 2 * n * w.kv_heads * io_row_bytes)
     if w.dtype != torch.bfloat16:
         kernel_name = "decode_generic_kernel"
     elif args.decode_kernel in ("tcgen05", "auto") or w.kv_dtype == "e4m3":
@@ -588,8 +595,8 @@ def run_ours(args):
         # CUDA events on the launch stream: its average is the figure.  Otherwise the launches
         # bracketed one by one are used (each bracket adds the events' own latency).
         bracketed_us = dec_ms / dec_n * 1e3
-        if launches_per_step == step_layers:
-            us, how, timed_n = ms / (K * step_layers) * 1e3, "median timed region: K steps of consecutive launches between two events", K * step_layers
+        if other_per_step == 0:
+            us, how, timed_n = ms / (K * dec_per_step) * 1e3, "median timed region: K steps of consecutive launches between two events", K * dec_per_step
         else:
             us, how, timed_n = bracketed_us, "each launch bracketed by two events", dec_n
         achieved = kv_bytes_per_launch / (us * 1e-6) / 1e9
@@ -599,7 +606,7 @@ def run_ours(args):
                     "traffic": recorded_traffic(args.workload, kernel_name),
                     "bytes_per_launch": kv_bytes_per_launch, "us_per_launch": us, "timing": how,
                     "launches_timed": timed_n, "us_per_launch_bracketed": bracketed_us,
-                    "frac_isolated": isolated / peak}
+                    "frac_isolated": isolated / peak, "layers_per_launch": step_layers // dec_per_step}
         kernels_us = {"append": app_ms / max(app_n, 1) * 1e3, "decode": dec_ms / dec_n * 1e3,
                       "combine": cmb_ms / cmb_n * 1e3 if cmb_n else 0.0}
 
@@ -629,7 +636,7 @@ def run_ours(args):
         if clocks:
             clocks.mark(t0w, time.time())
         assert sd0.pool.check_status(sd0.stream) == odma.OK
-        s_us = statistics.median(sm[r].elapsed_time(sm[r + 1]) for r in range(reps)) / (K * step_layers) * 1e3
+        s_us = statistics.median(sm[r].elapsed_time(sm[r + 1]) for r in range(reps)) / (K * dec_per_step) * 1e3
         roofline["serialised"] = {"us_per_launch": s_us, "frac": kv_bytes_per_launch / (s_us * 1e-6) / 1e9 / peak,
                                   "what": "the same steps with chain_launches = 0: every launch waits for the kernel ahead of it"}
         sd0.pool.destroy()
@@ -651,8 +658,8 @@ def run_ours(args):
             torch.cuda.synchronize()
         assert sd.pool.check_status(sd.stream) == odma.OK
         p_us = ev0.elapsed_time(ev1) / (reps * step_layers) * 1e3
-        probe_line = {"us_per_launch": p_us, "GBs": kv_bytes_per_launch / (p_us * 1e-6) / 1e9,
-                      "frac": kv_bytes_per_launch / (p_us * 1e-6) / 1e9 / peak, "launches": reps * step_layers,
+        probe_line = {"us_per_launch": p_us, "GBs": kv_bytes_layer / (p_us * 1e-6) / 1e9,
+                      "frac": kv_bytes_layer / (p_us * 1e-6) / 1e9 / peak, "launches": reps * step_layers,
                       "kernel": "decode_tc_kernel<probe>"}
         del own_p
 
@@ -686,7 +693,7 @@ def run_ours(args):
                 torch.cuda.synchronize()
             t_ms, cnt = sd.pool.profile_read(odma.K_DECODE)
             sd.pool.profile_enable(False)
-            res[kind] = {"us_per_launch": t_ms / cnt * 1e3, "GBs": kv_bytes_per_launch / (t_ms / cnt * 1e-3) / 1e9}
+            res[kind] = {"us_per_launch": t_ms / cnt * 1e3, "GBs": kv_bytes_layer / (t_ms / cnt * 1e-3) / 1e9}
         assert sd.pool.check_status(sd.stream) == odma.OK
         paged_line = {"pages": "16 tokens, ids shuffled", "timing": "each launch bracketed by two events", **res,
                       "slab_over_paged": res["paged"]["us_per_launch"] / res["slab"]["us_per_launch"]}

@@ -120,6 +120,10 @@ typedef struct odma_config {
     int32_t chain_launches;  /* 1: a decode step issued directly behind a decode step on another layer does
                                 not wait for it (see "Conventions"); 0: every launch waits for the kernel
                                 ahead of it (1) */
+    int32_t span_layers;     /* 1: odma_decode_step over several layers is ONE launch of the tcgen05 kernel
+                                when that kernel serves the pool and the split streams' partial results of
+                                all layers fit the scratch: the CTAs walk layer after layer over the same
+                                plan; 0: one launch per layer (1) */
     int32_t async_recal;     /* 1: a background thread owns the length window: odma_free only logs the
                                 realised length, the thread applies the log in order and refreshes the
                                 boundaries off the critical path (Sections III-E, IV-C); boundaries at

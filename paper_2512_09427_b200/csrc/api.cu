@@ -57,15 +57,18 @@ struct odma_pool {
     bool decode_was_last = false;
     // what the last decode launch was, for chaining the next one to it (decode_attention_impl)
     bool last_fused_tensor = false;
-    int32_t last_layer = -1;
     void* last_stream = nullptr;
     uint32_t scratch_parity = 0;
     uint32_t* d_counters = nullptr;   // per split stream: pieces delivered (fused combine)
     // a second scratch set: consecutive layers of one step alternate between the two, so that a
     // layer's kernel need not wait for the previous layer's
+    // the second scratch set: the upper halves of the allocations behind part_o, part_ml, d_counters
+    // (one launch over several layers uses both halves as one region, a layer after the other)
     float* part_o2 = nullptr;
     float* part_ml2 = nullptr;
     uint32_t* d_counters2 = nullptr;
+    size_t part_o_floats = 0, part_ml_floats = 0;      // of ONE set
+    int32_t last_lo = -1, last_hi = -1;                // layers the last decode launch covered
     int64_t slots_max = 0;
     int64_t table_words_max = 0;
     bool has_maps = false;
@@ -177,9 +180,6 @@ void free_device_side(odma_pool* p) {
     cudaFree(p->part_ml);
     cudaFree(p->d_status);
     cudaFree(p->d_counters);
-    cudaFree(p->part_o2);
-    cudaFree(p->part_ml2);
-    cudaFree(p->d_counters2);
     cudaFree(p->d_q);
     cudaFree(p->d_k_new);
     cudaFree(p->d_v_new);
@@ -339,6 +339,9 @@ void fill_decode_params(const odma_pool* pool, int32_t layer, const void* q, int
     p->wait_limit_ns = kDefaultWaitLimitNs;
     p->chained = 0;
     p->early_ok = 0;
+    p->n_layers = 1;
+    p->q_stride = p->new_stride = p->out_stride = p->lse_stride = p->part_o_stride = p->part_ml_stride = 0;
+    p->counter_stride = 0;
     p->kv_fp8 = pool->dtype == ODMA_DTYPE_FP8_E4M3 ? 1 : 0;
     p->k_scale = p->v_scale = p->k_inv = p->v_inv = 1.f;
     if (p->kv_fp8) {
@@ -387,6 +390,7 @@ void odma_config_default(odma_config* cfg) {
     cfg->fused_append = 1;
     cfg->decode_kernel = ODMA_DECODE_AUTO;
     cfg->chain_launches = 1;
+    cfg->span_layers = 1;
     cfg->async_recal = 0;
     cfg->cluster_observe = 0;
 }
@@ -465,17 +469,21 @@ int32_t odma_pool_create(void* dev_base, uint64_t bytes, int32_t layers, int32_t
         const size_t pm = static_cast<size_t>(p->slots_max) * cfg.max_group * 2 * 4;
         const size_t qb = static_cast<size_t>(cfg.max_batch) * kv_heads * cfg.max_group * head_dim * iosz;
         const size_t kb = static_cast<size_t>(cfg.max_batch) * kv_heads * head_dim * iosz;
-        bool ok = cudaMalloc(&p->part_o, po) == cudaSuccess && cudaMalloc(&p->part_ml, pm) == cudaSuccess &&
-                  cudaMalloc(&p->part_o2, po) == cudaSuccess && cudaMalloc(&p->part_ml2, pm) == cudaSuccess &&
-                  cudaMalloc(&p->d_counters2, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
-                  cudaMemset(p->d_counters2, 0, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
+        bool ok = cudaMalloc(&p->part_o, 2 * po) == cudaSuccess && cudaMalloc(&p->part_ml, 2 * pm) == cudaSuccess &&
                   cudaMalloc(&p->d_status, 4) == cudaSuccess && cudaMalloc(&p->d_q, qb) == cudaSuccess &&
-                  cudaMalloc(&p->d_counters, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
-                  cudaMemset(p->d_counters, 0, static_cast<size_t>(p->slots_max) * 4) == cudaSuccess &&
+                  cudaMalloc(&p->d_counters, static_cast<size_t>(p->slots_max) * 8) == cudaSuccess &&
+                  cudaMemset(p->d_counters, 0, static_cast<size_t>(p->slots_max) * 8) == cudaSuccess &&
                   cudaMalloc(&p->d_out, qb) == cudaSuccess && cudaMalloc(&p->d_k_new, kb) == cudaSuccess &&
                   cudaMalloc(&p->d_v_new, kb) == cudaSuccess &&
                   cudaMalloc(&p->d_step_table, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
                   cudaMemset(p->d_status, 0, 4) == cudaSuccess;
+        if (ok) {
+            p->part_o_floats = po / 4;
+            p->part_ml_floats = pm / 4;
+            p->part_o2 = p->part_o + p->part_o_floats;
+            p->part_ml2 = p->part_ml + p->part_ml_floats;
+            p->d_counters2 = p->d_counters + p->slots_max;
+        }
         for (auto& s : p->staging) {
             ok = ok && cudaMallocHost(&s.host, static_cast<size_t>(p->table_words_max) * 4) == cudaSuccess &&
                  cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) == cudaSuccess;
@@ -741,7 +749,7 @@ cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, 
 int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int32_t q_heads,
                               const odma_tables* tables, void* out, float* lse, void* stream,
                               const void* k_new, const void* v_new, const InlineLens* lens = nullptr,
-                              int32_t chain_pos = -1) {
+                              int32_t chain_pos = -1, int32_t span = 1) {
     int32_t rc = check_decode_args(pool, layer, q, q_heads, tables, out);
     if (rc != ODMA_OK) return rc;
     DecodeParams p;
@@ -767,10 +775,29 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
             // consecutive steps on different layers.  Only the tcgen05 kernel can run without its
             // dependency wait.  (Anything else enqueued in between - a table copy, the caller's own
             // kernels - makes the launch wait for that operation to complete before it starts.)
-            const bool can_chain = pool->alloc.config().chain_launches && fused && k_new != nullptr && p.early_ok &&
-                                   pool->last_fused_tensor && pool->last_stream == stream && pool->last_layer != layer;
-            const bool umma = uses_umma(pool, p.group, chain_pos >= 0 || can_chain);
-            if (fused) {
+            const bool disjoint = layer + span <= pool->last_lo || layer >= pool->last_hi;
+            const bool can_chain = span == 1 && pool->alloc.config().chain_launches && fused && k_new != nullptr &&
+                                   p.early_ok && pool->last_fused_tensor && pool->last_stream == stream && disjoint;
+            const bool umma = uses_umma(pool, p.group, chain_pos >= 0 || can_chain || span > 1);
+            if (span > 1) {
+                // One launch for `span` layers of a step (the caller has checked that the tcgen05 kernel
+                // serves it and that the scratch of all layers fits): the CTAs walk layer after layer over
+                // the same plan; CTAs drift apart by whole layers, so every layer has its own partial
+                // results and counters, laid one after the other across both scratch halves.  It waits for
+                // the launch before it (the previous step touched the same layers) and nothing chains to it.
+                const size_t n = static_cast<size_t>(tables->n);
+                p.n_layers = span;
+                p.q_stride = p.out_stride = static_cast<int64_t>(n * q_heads * pool->head_dim * pool->io_bytes);
+                p.new_stride = static_cast<int64_t>(n * pool->kv_heads * pool->head_dim * pool->io_bytes);
+                p.lse_stride = static_cast<int64_t>(n * q_heads);
+                p.part_o_stride = static_cast<int64_t>(tables->n_items) * p.group * pool->head_dim;
+                p.part_ml_stride = static_cast<int64_t>(tables->n_items) * p.group * 2;
+                p.counter_stride = tables->n_combine;
+                if (p.kv_fp8)
+                    for (int32_t l = 0; l < span; ++l)
+                        p.span_scales[l] = make_float4(pool->k_scale[layer + l], pool->v_scale[layer + l],
+                                                       1.0f / pool->k_scale[layer + l], 1.0f / pool->v_scale[layer + l]);
+            } else if (fused) {
                 pool->scratch_parity ^= 1u;              // scratch sets alternate from launch to launch
                 if (pool->scratch_parity) {
                     p.part_o = pool->part_o2;
@@ -779,8 +806,9 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
                 }
             }
             p.chained = umma && can_chain ? 1 : 0;
-            pool->last_fused_tensor = fused && k_new != nullptr;
-            pool->last_layer = layer;
+            pool->last_fused_tensor = span == 1 && fused && k_new != nullptr;
+            pool->last_lo = layer;
+            pool->last_hi = layer + span;
             pool->last_stream = stream;
             e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens, umma);
         } else if (generic_supported(pool->head_dim)) {
@@ -855,6 +883,24 @@ int32_t odma_decode_step(odma_pool* pool, int32_t layer, int32_t n_layers, int32
     if (inline_lens) {
         lens.n = n;
         std::copy(pool->v_len.begin(), pool->v_len.begin() + n, lens.len);
+    }
+    // All layers in ONE launch of the tcgen05 kernel when it serves this pool and the partial results
+    // of every layer's split streams fit the scratch (a plan without split streams needs none).
+    const int32_t group = q_heads / pool->kv_heads;
+    const bool span_fits =
+        t.n_combine == 0 ||
+        (static_cast<size_t>(n_layers) * t.n_items * group * pool->head_dim <= 2 * pool->part_o_floats &&
+         static_cast<size_t>(n_layers) * t.n_items * group * 2 <= 2 * pool->part_ml_floats &&
+         static_cast<size_t>(n_layers) * t.n_combine <= 2 * static_cast<size_t>(pool->slots_max));
+    if (fuse && n_layers > 1 && pool->alloc.config().fused_combine && pool->alloc.config().span_layers &&
+        pool->alloc.config().decode_kernel != ODMA_DECODE_MMA_SYNC &&
+        umma_supported(pool->head_dim, group, pool->dtype == ODMA_DTYPE_FP8_E4M3) && span_fits &&
+        (pool->dtype != ODMA_DTYPE_FP8_E4M3 || n_layers <= kMaxSpanScales)) {
+        rc = decode_attention_impl(pool, layer, d_q, q_heads, &t, d_out, lse, stream, d_k_new, d_v_new,
+                                   inline_lens ? &lens : nullptr, 0, n_layers);
+        if (rc != ODMA_OK) return rc;
+        if (tables_out) *tables_out = t;
+        return ODMA_OK;
     }
     for (int32_t l = 0; l < n_layers; ++l) {
         const uint8_t* kn = static_cast<const uint8_t*>(d_k_new) + l * kb;
@@ -944,8 +990,7 @@ int32_t odma_check_status(odma_pool* pool, void* stream) {
     if (word != 0) {
         // a kernel that gave up may have left split streams half counted
         if (cudaMemset(pool->d_status, 0, 4) != cudaSuccess ||
-            cudaMemset(pool->d_counters, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess ||
-            cudaMemset(pool->d_counters2, 0, static_cast<size_t>(pool->slots_max) * 4) != cudaSuccess)
+            cudaMemset(pool->d_counters, 0, static_cast<size_t>(pool->slots_max) * 8) != cudaSuccess)
             return ODMA_ERR_CUDA;
     }
     return (word & kStatusTimeout) ? ODMA_ERR_TIMEOUT : ODMA_OK;

@@ -298,6 +298,12 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const int it_begin = rec.x, it_end = rec.y;
+    // A launch may span several layers of a step: every role walks the CTA's items once per layer, in
+    // one sequence x = 0 .. n_layers * n_it - 1 (item it_begin + x mod n_it of layer x div n_it); ring
+    // positions, buffer parities and query slots simply run on across the layers.
+    const int n_it = it_end - it_begin;
+    const int total = n_it * p.n_layers;
+    auto item_index = [&](int x) { return x < total ? it_begin + x % n_it : it_end; };
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
     const uint32_t p_u32 = smem_u32(pbuf);
@@ -353,8 +359,8 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     if (warp == 1) {
         // ------------------------------------------------------------------ producer
         uint32_t issued_any = 0, issued_odd = 0;     // per stage: loads issued at all / an odd number of times
-        const int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;
-        const int64_t v_array = k_array + p.rows_per_array;
+        int64_t k_array = static_cast<int64_t>(p.layer) * 2 * p.rows_per_array;      // of the layer being issued
+        int64_t v_array = k_array + p.rows_per_array;
         constexpr int COPIES = 2 * HALVES;            // copies per box position: K and V, each column block
         // One tile of a slab stream = up to four groups of 16 rows, fetched with one copy per
         // 128-byte column block of K and of V (a box of 16, 32, 48 or 64 rows; never past
@@ -413,9 +419,11 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
         uint32_t g = 0;                               // tiles issued so far
         fetch(it_begin);
-        for (int it = it_begin; it < it_end && ok; ++it) {
+        for (int x = 0; x < total && ok; ++x) {
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(it + 1);
+            fetch(item_index(x + 1));
+            k_array = static_cast<int64_t>(p.layer + x / n_it) * 2 * p.rows_per_array;
+            v_array = k_array + p.rows_per_array;
             for (int t = 0; t < im.tiles; ++t, ++g) {
                 const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
                 if (g < static_cast<uint32_t>(n_early)) {        // first use of the stage, part 1 under way
@@ -442,12 +450,18 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const uint8_t* qg = static_cast<const uint8_t*>(p.q);
         constexpr int Q_LOADS = (NT * 8 * ROW_CHUNKS + 31) / 32;
         fetch(it_begin);
-        for (int it = it_begin; it < it_end; ++it) {
-            const int k = it - it_begin;
+        for (int x = 0; x < total; ++x) {
+            const int k = x, li = x / n_it;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(it + 1);
+            fetch(item_index(x + 1));
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
-            const uint8_t* src = qg + (static_cast<size_t>(im.req) * p.q_heads + static_cast<size_t>(im.head) * p.group) * D * 2;
+            const uint8_t* src = qg + li * p.q_stride +
+                                 (static_cast<size_t>(im.req) * p.q_heads + static_cast<size_t>(im.head) * p.group) * D * 2;
+            const uint8_t* new_k = static_cast<const uint8_t*>(p.k_new) + li * p.new_stride;
+            const uint8_t* new_v = static_cast<const uint8_t*>(p.v_new) + li * p.new_stride;
+            const int64_t layer_l = p.layer + li;
+            // this layer's scales of an 8-bit pool
+            const float4 sc4 = (F8 && p.n_layers > 1) ? p.span_scales[li] : make_float4(p.k_scale, p.v_scale, p.k_inv, p.v_inv);
             uint4 v[Q_LOADS];
 #pragma unroll
             for (int i = 0; i < Q_LOADS; ++i) {
@@ -460,7 +474,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             const int kvsel = lane / ROW_CHUNKS, c_new = lane - kvsel * ROW_CHUNKS;
             if (mine) {
                 const size_t nrow = (static_cast<size_t>(im.req) * p.kv_heads + im.head) * ROW_CHUNKS;
-                nv = __ldg(reinterpret_cast<const uint4*>(kvsel ? p.v_new : p.k_new) + nrow + c_new);
+                nv = __ldg(reinterpret_cast<const uint4*>(kvsel ? new_v : new_k) + nrow + c_new);
             }
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQEmpty + slot), (use & 1u) ^ 1u, abort_flag, p.status, limit));
             if (!ok) break;
@@ -496,15 +510,15 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                         uint8_t* row = dst + r * 128 + ((((c >> 1) ^ r) & 7) << 4) + (c & 1) * 8;
                         *reinterpret_cast<uint2*>(row) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
                         *reinterpret_cast<uint2*>(row + 1024) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
-                        if (c == 0) qf[r] = __uint_as_float(static_cast<uint32_t>(127 - e) << 23) * (p.k_scale * p.scale_log2);
+                        if (c == 0) qf[r] = __uint_as_float(static_cast<uint32_t>(127 - e) << 23) * (sc4.x * p.scale_log2);
                     }
                 }
                 if (mine) {
                     // the new rows as the slab will hold them: eight codes from this lane's eight numbers
-                    const uint2 codes = quantize8_e4m3(nv, kvsel ? p.v_inv : p.k_inv);
+                    const uint2 codes = quantize8_e4m3(nv, kvsel ? sc4.w : sc4.z);
                     *reinterpret_cast<uint2*>(newbuf + slot * Cfg::kNewBytes + lane * 8) = codes;
                     uint2* slab = reinterpret_cast<uint2*>(const_cast<void*>(p.pool)) +
-                                  ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * (D / 8) + c_new;
+                                  ((layer_l * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * (D / 8) + c_new;
                     *slab = codes;
                 }
             } else {
@@ -520,7 +534,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if (mine) {
                     *reinterpret_cast<uint4*>(newbuf + slot * Cfg::kNewBytes + lane * 16) = nv;
                     uint4* slab = reinterpret_cast<uint4*>(const_cast<void*>(p.pool)) +
-                                  ((static_cast<int64_t>(p.layer) * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
+                                  ((layer_l * 2 + kvsel) * p.rows_per_array + im.row0 + im.n_slab) * ROW_CHUNKS + c_new;
                     *slab = nv;
                 }
             }
@@ -540,10 +554,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         uint32_t c[kLanes] = {0, 0};                  // tiles of each lane issued so far
         uint32_t g = 0;
         fetch(it_begin);
-        for (int it = it_begin; it < it_end && ok; ++it) {
-            const int k = it - it_begin;
+        for (int x = 0; x < total && ok; ++x) {
+            const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(it + 1);
+            fetch(item_index(x + 1));
             const bool both = BOTH && im.tiles >= kBothTiles;
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
@@ -598,10 +612,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
         uint32_t c = 0, j = 0, g = 0;                 // the lane's tiles and items (with tiles) so far; ring position
         fetch(it_begin);
-        for (int it = it_begin; it < it_end && ok; ++it) {
-            const int k = it - it_begin;
+        for (int x = 0; x < total && ok; ++x) {
+            const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(it + 1);
+            fetch(item_index(x + 1));
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
             // the lane's tiles of the item: all of them, or every second one when both lanes work on it
@@ -648,12 +662,19 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         float* x_mine = xchg + L * 32;                      // where this lane leaves (m, l) per head as a helper
         const float* x_other = xchg + (L ^ 1) * 32;
         fetch(it_begin);
-        for (int it = it_begin; it < it_end && ok; ++it) {
-            const int k = it - it_begin;
+        for (int x = 0; x < total && ok; ++x) {
+            const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(it + 1);
+            fetch(item_index(x + 1));
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
+            // this layer's outputs and scratch
+            const int li = x / n_it;
+            __nv_bfloat16* out_l = out + li * (p.out_stride / 2);
+            float* lse_l = p.lse ? p.lse + li * p.lse_stride : nullptr;
+            float* part_o_l = p.part_o + li * p.part_o_stride;
+            float* part_ml_l = p.part_ml + li * p.part_ml_stride;
+            uint32_t* counters_l = p.counters ? p.counters + static_cast<size_t>(li) * p.counter_stride : nullptr;
             // BOTH: an item of kBothTiles tiles or more is worked on by both lanes, its tiles going to
             // them in turn from its home lane (item number mod 2).  The other lane is the helper: it
             // leaves its accumulator in tensor memory and its (m, l) in shared memory, and the home
@@ -957,19 +978,20 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 }
             }
             if (F8) {                                      // codes to values
+                const float v_scale = p.n_layers > 1 ? p.span_scales[li].y : p.v_scale;
 #pragma unroll
-                for (int i = 0; i < D / 4; ++i) oo[0][i] *= p.v_scale;
+                for (int i = 0; i < D / 4; ++i) oo[0][i] *= v_scale;
             }
             auto write_out = [&](int req, int head, int rs, float M, float Lsum, const float (&x)[D / 4]) {
                 const int h = hq + 8 * rs;
                 if (h >= group) return;
                 const float inv = fast_rcp(Lsum);
                 const size_t row = static_cast<size_t>(req) * p.q_heads + static_cast<size_t>(head) * group + h;
-                __nv_bfloat16* dst = out + row * D + kq;
+                __nv_bfloat16* dst = out_l + row * D + kq;
 #pragma unroll
                 for (int i = 0; i < D / 8; ++i)
                     *reinterpret_cast<uint32_t*>(dst + 8 * i) = pack_bf16(x[2 * i] * inv, x[2 * i + 1] * inv);
-                if ((lane & 3) == 0 && p.lse) p.lse[row] = (M + fast_log2(Lsum)) * 0.6931471805599453f;
+                if ((lane & 3) == 0 && lse_l) lse_l[row] = (M + fast_log2(Lsum)) * 0.6931471805599453f;
             };
             if (im.direct) {
 #pragma unroll
@@ -981,12 +1003,12 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 const int h = hq + 8 * rs;
                 if (h >= group) continue;
                 const size_t prow = static_cast<size_t>(im.slot) * group + h;
-                float* po = p.part_o + prow * D + kq;
+                float* po = part_o_l + prow * D + kq;
 #pragma unroll
                 for (int i = 0; i < D / 8; ++i) *reinterpret_cast<float2*>(po + 8 * i) = make_float2(oo[rs][2 * i], oo[rs][2 * i + 1]);
-                if ((lane & 3) == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(m_ref[rs], l_acc[rs]);
+                if ((lane & 3) == 0) *reinterpret_cast<float2*>(part_ml_l + prow * 2) = make_float2(m_ref[rs], l_acc[rs]);
             }
-            if (p.counters == nullptr) continue;           // a combine kernel follows
+            if (counters_l == nullptr) continue;           // a combine kernel follows
             // The CTA that delivers a split stream's last piece merges all of them, in slot
             // order (so the result does not depend on which CTA that is), reading them back
             // through L2 (its own included), the next piece's loads in flight while one is folded.
@@ -995,9 +1017,9 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             int is_last = 0;
             if (lane == 0) {
                 __threadfence();
-                const uint32_t seen = atomicAdd(p.counters + im.comb, 1u);
+                const uint32_t seen = atomicAdd(counters_l + im.comb, 1u);
                 is_last = seen + 1u == static_cast<uint32_t>(cr.w);
-                if (is_last) p.counters[im.comb] = 0u;     // ready for the next launch
+                if (is_last) counters_l[im.comb] = 0u;     // ready for the next launch
             }
             is_last = __shfl_sync(0xFFFFFFFFu, is_last, 0);
             if (!is_last) continue;
@@ -1011,8 +1033,8 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 for (int i = 0; i < D / 4; ++i) fa[i] = 0.f;
                 auto load = [&](int s, float2& ml, float2 (&x)[D / 8]) {
                     const size_t prow = static_cast<size_t>(cr.z + s) * group + h;
-                    ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + prow * 2));
-                    const float* po = p.part_o + prow * D + kq;
+                    ml = __ldcg(reinterpret_cast<const float2*>(part_ml_l + prow * 2));
+                    const float* po = part_o_l + prow * D + kq;
 #pragma unroll
                     for (int i = 0; i < D / 8; ++i) x[i] = __ldcg(reinterpret_cast<const float2*>(po + 8 * i));
                 };

@@ -48,12 +48,22 @@ struct DecodeParams {
     int32_t kv_fp8;             // the pool holds E4M3 codes (one byte per element); q, the new rows and out are bf16
     float k_scale, v_scale;     // 8-bit pool: a stored code stands for value * scale (this layer's scales)
     float k_inv, v_inv;         // fp32 reciprocals: what an appended element is multiplied by before rounding
+    // tcgen05 kernel: one launch for several layers of a step.  The CTA walks its items once per layer
+    // (same plan, the pipeline never drains); layer li of the launch uses K/V arrays of layer + li and
+    // the buffers below advanced by li strides.
+    int32_t n_layers;           // 1 = the usual launch
+    int64_t q_stride, new_stride, out_stride;      // bytes between consecutive layers of q / k_new, v_new / out
+    int64_t lse_stride;                            // floats between consecutive layers of lse
+    int64_t part_o_stride, part_ml_stride;         // floats between consecutive layers' partial results
+    int32_t counter_stride;                        // counters between consecutive layers
+    float4 span_scales[32];                        // 8-bit pools, n_layers > 1: {k_scale, v_scale, k_inv, v_inv} of layer + li
     int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
 };
 
 // Lengths handed to the tensor-core kernel with its arguments instead of through the table in
 // device memory (a step that reuses the previous step's plan then needs no copy at all).
+constexpr int kMaxSpanScales = 32;   // layers of one launch over an 8-bit pool (DecodeParams::span_scales)
 constexpr int kInlineLens = 256;
 struct InlineLens {
     int32_t n;                  // 0: take the lengths the plan was made with (items' n_tokens)

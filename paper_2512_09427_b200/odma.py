@@ -33,7 +33,7 @@ class Config(C.Structure):
                 ("gamma_permille", C.c_int32), ("tau_permille", C.c_int32), ("growth", C.c_int32),
                 ("large_fixed", C.c_int32), ("max_batch", C.c_int32), ("max_group", C.c_int32),
                 ("plan_ctas", C.c_int32), ("fused_combine", C.c_int32), ("fused_append", C.c_int32),
-                ("decode_kernel", C.c_int32), ("chain_launches", C.c_int32), ("async_recal", C.c_int32), ("cluster_observe", C.c_int32)]
+                ("decode_kernel", C.c_int32), ("chain_launches", C.c_int32), ("span_layers", C.c_int32), ("async_recal", C.c_int32), ("cluster_observe", C.c_int32)]
 
 
 class Slab(C.Structure):

@@ -90,14 +90,15 @@ def test_ragged_lengths_span_tiles_key_groups_and_splits(ctas, fused):
     print("e4m3 ragged", ctas, fused, e)
 
 
+@pytest.mark.parametrize("span", [1, 0], ids=["one_launch", "launch_per_layer"])
 @pytest.mark.parametrize("ctas", [0, 5])
-def test_fused_steps_over_chained_layers(ctas):
+def test_fused_steps_over_chained_layers(ctas, span):
     """odma_decode_step: the new token is quantised by the decode kernel, used as its code's value
     and written into the slab; layers chain.  Three steps back to back without a host sync."""
     odma = lib()
     lens = [0, 1, 31, 32, 63, 64, 129, 700, 1500, 2771]
     w = small(lens, layers=4)
-    s, reqs = start(w, plan_ctas=ctas)
+    s, reqs = start(w, plan_ctas=ctas, span_layers=span)
     steps, NL = 3, w.layers
     qs = [torch.stack([s.queries(l, reqs, w.q_heads, k) for l in range(NL)]).contiguous() for k in range(steps)]
     kns = [torch.stack([torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs])

@@ -353,7 +353,7 @@ def test_decode_step_from_host_buffers_matches_the_device_path(pinned):
 
 
 @pytest.mark.parametrize("fused_append", [1, 0])
-def test_decode_step_with_the_append_inside_the_decode_kernel(fused_append):
+def test_decode_step_with_the_append_inside_the_decode_kernel(fused_append, decode_kernel):
     """odma_decode_step: the new token is taken from k_new / v_new by the decode kernel itself
     (never read from the slab) and written into the slab for later steps.  Lengths chosen so
     that some streams consist of the new token alone, some end a tile exactly, some are split."""
@@ -381,7 +381,8 @@ def test_decode_step_with_the_append_inside_the_decode_kernel(fused_append):
         torch.cuda.synchronize()
         assert s.pool.check_status(s.stream) == odma.OK
         assert s.pool.profile_read(odma.K_APPEND)[1] == (0 if fused_append else w.layers)
-        assert s.pool.profile_read(odma.K_DECODE)[1] == w.layers
+        # with the append fused in, both layers of the step are one launch of the tcgen05 kernel
+        assert s.pool.profile_read(odma.K_DECODE)[1] == (1 if fused_append and decode_kernel == 1 else w.layers)
         s.pool.profile_enable(False)
         assert t.n_combine > 0
         s.ls.commit(reqs, 1)
@@ -477,8 +478,9 @@ def test_back_to_back_steps_on_one_layer_without_host_syncs():
         assert np.array_equal(s.pool_rows(0, 1, r).view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
 
 
+@pytest.mark.parametrize("span", [1, 0], ids=["one_launch", "launch_per_layer"])
 @pytest.mark.parametrize("ctas", [0, 5])
-def test_layers_of_one_step_run_chained_without_host_syncs(ctas):
+def test_layers_of_one_step_run_chained_without_host_syncs(ctas, span):
     """odma_decode_step over six layers, three steps enqueued back to back: the kernel of layer
     l > 0 does not wait for the kernel of layer l - 1 (other K/V arrays, other outputs, the other
     scratch set), so kernels of neighbouring layers run side by side.  Every layer of every
@@ -487,7 +489,7 @@ def test_layers_of_one_step_run_chained_without_host_syncs(ctas):
     lens = [0, 40, 64, 129, 700, 1500, 2771]
     w = qwen_small(lens, layers=6)
     w = wl.scaled(w, predicted=w.context + 8)
-    s = Session(w, plan_ctas=ctas)
+    s = Session(w, plan_ctas=ctas, span_layers=span)      # all six layers in one launch, or a chained launch each
     s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
     reqs = list(range(w.batch))
     s.admit(reqs, w.predicted)
