@@ -603,7 +603,7 @@ def run_ours(args):
         isolated = kv_bytes_per_launch / (bracketed_us * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                    "traffic": recorded_traffic(args.workload, kernel_name),
+                    "traffic": recorded_traffic(args.workload + ("-e4m3" if w.kv_dtype == "e4m3" else ""), kernel_name),
                     "bytes_per_launch": kv_bytes_per_launch, "us_per_launch": us, "timing": how,
                     "launches_timed": timed_n, "us_per_launch_bracketed": bracketed_us,
                     "frac_isolated": isolated / peak, "layers_per_launch": step_layers // dec_per_step}
