@@ -818,6 +818,83 @@ def run_config4(args):
     print(json.dumps(line), flush=True)
 
 
+def run_prefill(args):
+    """`--workload prefill`: a chunk of prompt tokens per request appended to Qwen-7B-shaped slabs and
+    attended causally (odma_build_prefill_tables + the decode kernel: one stream per new token).  The
+    timed step is the chunk's attention on one layer; copies of the layer rotate so that L2 starts cold."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    from paper_2512_09427_b200 import odma
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak()
+    K, W = args.steps, args.warmup
+    n_req, ctx, chunk, copies = 8, 1920, 128, 8
+    context = np.full(n_req, ctx, dtype=np.int64)
+    w = wl.Workload(name="prefill", seed=950907, layers=copies, q_heads=28, kv_heads=4, head_dim=128, dtype=torch.bfloat16,
+                    pool_bytes=copies * n_req * 4096 * 2 * 4 * 128 * 2 * 2, safety_pct=10, max_len=4096, context=context,
+                    predicted=context + chunk, static_buckets=(2048, 4096))
+    if args.kv_dtype == "e4m3":
+        w = wl.with_e4m3(w)
+    sd = SlabDecode(w, 1, dev, fused=args.fused_combine, decode_kernel=DECODE_KERNELS[args.decode_kernel])
+    sd.learn_boundaries()
+    sd.admit_and_fill()
+    pool, reqs = sd.pool, sd.reqs
+    # the chunk: appended on every layer copy through the ordinary calls, its plan made first
+    for r in reqs:
+        rc, _, _ = pool.ensure_capacity(r, ctx + chunk, sd.stream)
+        assert rc == odma.OK
+    table = torch.empty(pool.tables_bytes(n_req * chunk), dtype=torch.uint8, device=dev)
+    pt = pool.build_prefill_tables(reqs, [chunk] * n_req, table.data_ptr(), table.numel(), sd.stream)
+    table_app = torch.empty(pool.tables_bytes(n_req), dtype=torch.uint8, device=dev)
+    t_app = pool.build_tables(reqs, table_app.data_ptr(), table_app.numel(), sd.stream, [chunk] * n_req)
+    for layer in range(copies):
+        kk = torch.cat([wl.kv_rows(w.seed, layer, r, wl.KIND_K, ctx, ctx + chunk, 4, 128, w.dtype, dev) for r in reqs])
+        vv = torch.cat([wl.kv_rows(w.seed, layer, r, wl.KIND_V, ctx, ctx + chunk, 4, 128, w.dtype, dev) for r in reqs])
+        pool.append_kv(layer, t_app, kk.data_ptr(), vv.data_ptr(), sd.stream)
+        torch.cuda.synchronize()
+    q = torch.stack([torch.cat([torch.stack([wl.q_rows(w.seed, layer, r, j, 28, 128, w.dtype, dev) for j in range(chunk)])
+                                for r in reqs]) for layer in range(copies)]).contiguous()
+    out = torch.zeros_like(q)
+    def step(i):
+        l = i % copies
+        pool.decode_attention(l, q[l].data_ptr(), 28, pt, out[l].data_ptr(), 0, sd.stream)
+    for i in range(max(W, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    clocks = ClockSampler(dev.index or 0)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+    t0 = time.time()
+    ev[0].record()
+    for r in range(5):
+        for i in range(K):
+            step(r * K + i)
+        ev[r + 1].record()
+    torch.cuda.synchronize()
+    clocks.mark(t0, time.time())
+    assert pool.check_status(sd.stream) == odma.OK
+    ms = statistics.median(ev[r].elapsed_time(ev[r + 1]) for r in range(5)) / K
+    keys = sum(ctx + j + 1 for j in range(chunk)) * n_req                 # (token, key) pairs per KV head
+    flops = 2 * 2 * keys * 28 * 128                                      # two products, 28 query heads
+    read_once = n_req * (ctx + chunk) * 2 * 4 * 128 * w.elem_bytes       # the slabs read once
+    read_per_token = keys * 2 * 4 * 128 * w.elem_bytes                   # what this form reads (per new token, from L2 after the first)
+    line = {"metric": "prefill tokens/s (chunk attention over the slabs, one layer)", "value": n_req * chunk / (ms * 1e-3),
+            "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "e4m3" if w.kv_dtype == "e4m3" else "bf16", "data": "synthetic",
+            "config": {"workload": f"chunked prefill: {n_req} requests, context {ctx}, chunk {chunk} tokens, Qwen-7B-shaped layer "
+                                   f"(28q/4kv heads, head_dim 128), {copies} rotating layer copies",
+                       "streams": int(pt.n), "items": int(pt.n_items), "split_streams": int(pt.n_combine)},
+            "gpu_launches": K,
+            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel" if args.decode_kernel != "tcgen05" and w.kv_dtype != "e4m3" else "decode_umma_kernel",
+                         "achieved": read_per_token / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                         "frac": read_per_token / (ms * 1e-3) / 1e9 / peak, "peak_kind": peak_kind, "traffic": None,
+                         "bytes_per_launch": read_per_token, "us_per_launch": ms * 1e3,
+                         "note": "bytes = the slab prefix of every new token (this form streams it once per token, mostly from L2); "
+                                 "the slabs themselves are " + str(read_once) + " bytes; tensor work " + str(flops) + " flop"},
+            "tflops": flops / (ms * 1e-3) / 1e12, "clocks": clocks.stop()}
+    print(json.dumps(line), flush=True)
+
+
 def run_admission(args):
     """`--workload admission`: the paper's serving protocol (Section V) on the library's native
     simulator.  Two decode launches of the config-2 shape (full batch and half of it) are timed
@@ -918,7 +995,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5", "admission"])
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config4", "config5", "admission", "prefill"])
     ap.add_argument("--requests", type=int, default=4000, help="admission: requests in the Poisson trace")
     ap.add_argument("--rate", type=float, default=0.0, help="admission: arrivals per second (0 = 1.5x what static reservation sustains)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -946,6 +1023,8 @@ def main():
         run_reference(args)
     elif args.workload == "config4":
         run_config4(args)
+    elif args.workload == "prefill":
+        run_prefill(args)
     elif args.workload == "admission":
         run_admission(args)
     else:
