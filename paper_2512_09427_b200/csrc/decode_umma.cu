@@ -234,7 +234,7 @@ __device__ __forceinline__ Item item_of(const int4& a, const int4& b, const Inli
 template <int D, int NT, int MODE, bool F8>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
-                   const __grid_constant__ InlineLens lens) {
+                   const __grid_constant__ InlineLens lens, const __grid_constant__ SpanParams sp) {
     using Cfg = UmmaConfig<D, NT, F8>;
     static_assert(!F8 || (D == 128 && NT == 1 && MODE == kModeSlab), "8-bit slabs: head_dim 128, group <= 8, slab mode");
     constexpr int ES = Cfg::kElem;
@@ -274,6 +274,11 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     const int64_t limit = p.wait_limit_ns;
     const int cta = blockIdx.x;
     const bool fused = p.k_new != nullptr;
+    // The CTA's record and its first item (the record carries a copy) are asked for before anything
+    // else: the set-up below runs under their latency, and no role starts with a load that depends
+    // on another (a chained CTA's first tile is requested one L2 round trip earlier).
+    const int4 rec = __ldg(p.cta + 3 * cta);
+    const int4 first_a = __ldg(p.cta + 3 * cta + 1), first_b = __ldg(p.cta + 3 * cta + 2);
 
     // a query slot is handed back by the MMA thread and the lane's softmax warp (BOTH: and the other lane's,
     // which takes the heads' score factors from it when it helps with the item)
@@ -292,7 +297,6 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    const int4 rec = __ldg(p.cta + 3 * cta);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -303,7 +307,16 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // positions, buffer parities and query slots simply run on across the layers.
     const int n_it = it_end - it_begin;
     const int total = n_it * p.n_layers;
-    auto item_index = [&](int x) { return x < total ? it_begin + x % n_it : it_end; };
+    const bool span = p.n_layers > 1;
+    // the walk: item `it` of layer `li`, advanced by every role at the end of each turn of its loop
+    int it = it_begin, li = 0;
+    auto advance = [&]() {
+        if (++it == it_end) {
+            it = it_begin;
+            ++li;
+        }
+    };
+    auto next_item = [&]() { return it + 1 < it_end ? it + 1 : (li + 1 < p.n_layers ? it_begin : it_end); };
     const uint32_t kv_u32 = smem_u32(kv);
     const uint32_t q_u32 = smem_u32(qbuf);
     const uint32_t p_u32 = smem_u32(pbuf);
@@ -349,7 +362,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // item walk shared by the roles: descriptor of item `it`, the next one already on its way
     int4 nxt_a = make_int4(0, 0, 0, 0), nxt_b = nxt_a;
     auto fetch = [&](int it) {
-        if (it < it_end) {
+        if (it == it_begin) {                          // the copy in the CTA's record
+            nxt_a = first_a;
+            nxt_b = first_b;
+        } else if (it < it_end) {
             nxt_a = __ldg(p.items + 2 * it);
             nxt_b = __ldg(p.items + 2 * it + 1);
         }
@@ -403,8 +419,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         // previous grid finishes.
         int n_early = 0;
         if (MODE != kModePaged && !chained && p.early_ok) {
-            const int4* r = p.cta + 3 * cta;
-            int4 a = __ldg(r + 1), b = __ldg(r + 2);
+            int4 a = first_a, b = first_b;
             for (int it = it_begin; it < it_end && n_early < static_cast<int>(STAGES); ++it) {
                 if (it != it_begin) {
                     a = __ldg(p.items + 2 * it);
@@ -419,10 +434,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
 
         uint32_t g = 0;                               // tiles issued so far
         fetch(it_begin);
-        for (int x = 0; x < total && ok; ++x) {
+        for (int x = 0; x < total && ok; ++x, advance()) {
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(item_index(x + 1));
-            k_array = static_cast<int64_t>(p.layer + x / n_it) * 2 * p.rows_per_array;
+            fetch(next_item());
+            k_array = static_cast<int64_t>(p.layer + li) * 2 * p.rows_per_array;
             v_array = k_array + p.rows_per_array;
             for (int t = 0; t < im.tiles; ++t, ++g) {
                 const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
@@ -450,18 +465,18 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const uint8_t* qg = static_cast<const uint8_t*>(p.q);
         constexpr int Q_LOADS = (NT * 8 * ROW_CHUNKS + 31) / 32;
         fetch(it_begin);
-        for (int x = 0; x < total; ++x) {
-            const int k = x, li = x / n_it;
+        for (int x = 0; x < total; ++x, advance()) {
+            const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(item_index(x + 1));
+            fetch(next_item());
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
-            const uint8_t* src = qg + li * p.q_stride +
+            const uint8_t* src = qg + (span ? li * sp.q_stride : 0) +
                                  (static_cast<size_t>(im.req) * p.q_heads + static_cast<size_t>(im.head) * p.group) * D * 2;
-            const uint8_t* new_k = static_cast<const uint8_t*>(p.k_new) + li * p.new_stride;
-            const uint8_t* new_v = static_cast<const uint8_t*>(p.v_new) + li * p.new_stride;
+            const uint8_t* new_k = static_cast<const uint8_t*>(p.k_new) + (span ? li * sp.new_stride : 0);
+            const uint8_t* new_v = static_cast<const uint8_t*>(p.v_new) + (span ? li * sp.new_stride : 0);
             const int64_t layer_l = p.layer + li;
             // this layer's scales of an 8-bit pool
-            const float4 sc4 = (F8 && p.n_layers > 1) ? p.span_scales[li] : make_float4(p.k_scale, p.v_scale, p.k_inv, p.v_inv);
+            const float4 sc4 = (F8 && span) ? sp.scales[li] : make_float4(p.k_scale, p.v_scale, p.k_inv, p.v_inv);
             uint4 v[Q_LOADS];
 #pragma unroll
             for (int i = 0; i < Q_LOADS; ++i) {
@@ -554,10 +569,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         uint32_t c[kLanes] = {0, 0};                  // tiles of each lane issued so far
         uint32_t g = 0;
         fetch(it_begin);
-        for (int x = 0; x < total && ok; ++x) {
+        for (int x = 0; x < total && ok; ++x, advance()) {
             const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(item_index(x + 1));
+            fetch(next_item());
             const bool both = BOTH && im.tiles >= kBothTiles;
             const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
@@ -612,10 +627,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         const uint32_t t_o = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + 128u;
         uint32_t c = 0, j = 0, g = 0;                 // the lane's tiles and items (with tiles) so far; ring position
         fetch(it_begin);
-        for (int x = 0; x < total && ok; ++x) {
+        for (int x = 0; x < total && ok; ++x, advance()) {
             const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(item_index(x + 1));
+            fetch(next_item());
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
             // the lane's tiles of the item: all of them, or every second one when both lanes work on it
@@ -662,19 +677,18 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         float* x_mine = xchg + L * 32;                      // where this lane leaves (m, l) per head as a helper
         const float* x_other = xchg + (L ^ 1) * 32;
         fetch(it_begin);
-        for (int x = 0; x < total && ok; ++x) {
+        for (int x = 0; x < total && ok; ++x, advance()) {
             const int k = x;
             const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(item_index(x + 1));
+            fetch(next_item());
             const uint32_t g0 = g;
             g += static_cast<uint32_t>(im.tiles);
             // this layer's outputs and scratch
-            const int li = x / n_it;
-            __nv_bfloat16* out_l = out + li * (p.out_stride / 2);
-            float* lse_l = p.lse ? p.lse + li * p.lse_stride : nullptr;
-            float* part_o_l = p.part_o + li * p.part_o_stride;
-            float* part_ml_l = p.part_ml + li * p.part_ml_stride;
-            uint32_t* counters_l = p.counters ? p.counters + static_cast<size_t>(li) * p.counter_stride : nullptr;
+            __nv_bfloat16* out_l = out + (span ? li * (sp.out_stride / 2) : 0);
+            float* lse_l = p.lse ? p.lse + (span ? li * sp.lse_stride : 0) : nullptr;
+            float* part_o_l = p.part_o + (span ? li * sp.part_o_stride : 0);
+            float* part_ml_l = p.part_ml + (span ? li * sp.part_ml_stride : 0);
+            uint32_t* counters_l = p.counters ? p.counters + (span ? static_cast<size_t>(li) * sp.counter_stride : 0) : nullptr;
             // BOTH: an item of kBothTiles tiles or more is worked on by both lanes, its tiles going to
             // them in turn from its home lane (item number mod 2).  The other lane is the helper: it
             // leaves its accumulator in tensor memory and its (m, l) in shared memory, and the home
@@ -978,7 +992,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 }
             }
             if (F8) {                                      // codes to values
-                const float v_scale = p.n_layers > 1 ? p.span_scales[li].y : p.v_scale;
+                const float v_scale = span ? sp.scales[li].y : p.v_scale;
 #pragma unroll
                 for (int i = 0; i < D / 4; ++i) oo[0][i] *= v_scale;
             }
@@ -1092,7 +1106,7 @@ int umma_stages() {
 
 template <int D, int NT, int MODE, bool F8>
 cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas, cudaStream_t stream,
-                             const InlineLens& lens) {
+                             const InlineLens& lens, const SpanParams& sp) {
     using Cfg = UmmaConfig<D, NT, F8>;
     static bool configured[kMaxDevices] = {false};     // the opt-in to large shared memory is per device
     auto kern = decode_umma_kernel<D, NT, MODE, F8>;
@@ -1118,15 +1132,15 @@ cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, maps, p, lens);
+    return cudaLaunchKernelEx(&cfg, kern, maps, p, lens, sp);
 }
 
 template <int D, int NT>
 cudaError_t launch_umma_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s,
-                             const InlineLens& lens) {
+                             const InlineLens& lens, const SpanParams& sp) {
     switch (mode) {
-        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab, false>(maps, p, n_ctas, s, lens);
-        case kModePaged: return launch_umma_inst<D, NT, kModePaged, false>(maps, p, n_ctas, s, lens);
+        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab, false>(maps, p, n_ctas, s, lens, sp);
+        case kModePaged: return launch_umma_inst<D, NT, kModePaged, false>(maps, p, n_ctas, s, lens, sp);
     }
     return cudaErrorInvalidValue;
 }
@@ -1139,20 +1153,23 @@ bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8) {
 }
 
 cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                               cudaStream_t stream, const InlineLens* lens_in) {
+                               cudaStream_t stream, const InlineLens* lens_in, const SpanParams* span_in) {
     static const InlineLens no_lens{};                 // n = 0: lengths as planned
+    static const SpanParams no_span{};                 // never read by a one-layer launch
     const InlineLens& lens = lens_in ? *lens_in : no_lens;
+    if (p.n_layers > 1 && !span_in) return cudaErrorInvalidValue;
+    const SpanParams& sp = span_in ? *span_in : no_span;
     if (p.kv_fp8) {
         if (!umma_supported(p.head_dim, p.group, true) || mode != kModeSlab) return cudaErrorInvalidValue;
-        return launch_umma_inst<128, 1, kModeSlab, true>(maps, p, n_ctas, stream, lens);
+        return launch_umma_inst<128, 1, kModeSlab, true>(maps, p, n_ctas, stream, lens, sp);
     }
     const bool two = p.group > 8;
     if (p.head_dim == 128)
-        return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens)
-                   : launch_umma_mode<128, 1>(maps, p, mode, n_ctas, stream, lens);
+        return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens, sp)
+                   : launch_umma_mode<128, 1>(maps, p, mode, n_ctas, stream, lens, sp);
     if (p.head_dim == 64)
-        return two ? launch_umma_mode<64, 2>(maps, p, mode, n_ctas, stream, lens)
-                   : launch_umma_mode<64, 1>(maps, p, mode, n_ctas, stream, lens);
+        return two ? launch_umma_mode<64, 2>(maps, p, mode, n_ctas, stream, lens, sp)
+                   : launch_umma_mode<64, 1>(maps, p, mode, n_ctas, stream, lens, sp);
     return cudaErrorInvalidValue;
 }
 

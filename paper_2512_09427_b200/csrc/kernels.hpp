@@ -51,19 +51,26 @@ struct DecodeParams {
     // tcgen05 kernel: one launch for several layers of a step.  The CTA walks its items once per layer
     // (same plan, the pipeline never drains); layer li of the launch uses K/V arrays of layer + li and
     // the buffers below advanced by li strides.
-    int32_t n_layers;           // 1 = the usual launch
-    int64_t q_stride, new_stride, out_stride;      // bytes between consecutive layers of q / k_new, v_new / out
-    int64_t lse_stride;                            // floats between consecutive layers of lse
-    int64_t part_o_stride, part_ml_stride;         // floats between consecutive layers' partial results
-    int32_t counter_stride;                        // counters between consecutive layers
-    float4 span_scales[32];                        // 8-bit pools, n_layers > 1: {k_scale, v_scale, k_inv, v_inv} of layer + li
+    int32_t n_layers;           // 1 = the usual launch; more: see SpanParams
     int32_t stages;             // pipeline depth of the tensor-core kernel (2..8)
     int32_t q_slots;            // depth of its query / item-descriptor ring (4..8)
 };
 
+// What a launch over several layers needs beyond DecodeParams; a parameter of its own that a
+// one-layer launch never reads (the parameter block is fetched line by line, on first use, by every
+// CTA: what the usual launch touches stays small).
+constexpr int kMaxSpanScales = 32;   // layers of one launch over an 8-bit pool
+struct SpanParams {
+    int64_t q_stride, new_stride, out_stride;      // bytes between consecutive layers of q / k_new, v_new / out
+    int64_t lse_stride;                            // floats between consecutive layers of lse
+    int64_t part_o_stride, part_ml_stride;         // floats between consecutive layers' partial results
+    int32_t counter_stride;                        // counters between consecutive layers
+    int32_t pad;
+    float4 scales[kMaxSpanScales];                 // 8-bit pools: {k_scale, v_scale, k_inv, v_inv} of layer + li
+};
+
 // Lengths handed to the tensor-core kernel with its arguments instead of through the table in
 // device memory (a step that reuses the previous step's plan then needs no copy at all).
-constexpr int kMaxSpanScales = 32;   // layers of one launch over an 8-bit pool (DecodeParams::span_scales)
 constexpr int kInlineLens = 256;
 struct InlineLens {
     int32_t n;                  // 0: take the lengths the plan was made with (items' n_tokens)
@@ -88,7 +95,7 @@ cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int 
 // An 8-bit (E4M3) pool: head_dim 128, group <= 8, slab mode.
 bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8);
 cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                               cudaStream_t stream, const InlineLens* lens = nullptr);
+                               cudaStream_t stream, const InlineLens* lens = nullptr, const SpanParams* span = nullptr);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
 bool generic_supported(int32_t head_dim);
 
