@@ -223,8 +223,8 @@ def test_config2_in_the_benchmarks_own_launch_configuration(decode_kernel):
 def test_config2_benchmark_pattern_300_overlapping_steps_bit_identical():
     """What bench.py times: the config-2 step repeated on three rotating KV copies (layers of one
     pool) with no synchronisation, so that consecutive launches overlap.  The step on a copy is
-    the same computation every round (the same token re-appended at the same position), so the
-    results of rounds 1 to 99 must be equal bit for bit; rounds 0 and 1 are checked against the
+    the same computation every pass (the same token re-appended at the same position), so the
+    results of passes 1 to 99 must be equal bit for bit; passes 0 and 1 are checked against the
     checker."""
     odma = lib()
     w = wl.config2(layers=3)
@@ -239,11 +239,11 @@ def test_config2_benchmark_pattern_300_overlapping_steps_bit_identical():
     q = torch.stack([s.queries(l, reqs, w.q_heads, 0) for l in range(L)]).contiguous()
     kn = torch.stack([torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r], s.lens[r] + 1) for r in reqs]) for l in range(L)]).contiguous()
     vn = torch.stack([torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]) for l in range(L)]).contiguous()
-    rounds = 100
-    outs = torch.full((rounds, L) + tuple(q.shape[1:]), float("nan"), dtype=q.dtype, device=s.dev)
+    passes = 100
+    outs = torch.full((passes, L) + tuple(q.shape[1:]), float("nan"), dtype=q.dtype, device=s.dev)
     lses = torch.full((rounds, L, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev)
     torch.cuda.synchronize()
-    for k in range(rounds):                      # no synchronisation inside this loop
+    for k in range(passes):                      # no synchronisation inside this loop
         for l in range(L):
             s.pool.decode_step(l, 1, w.q_heads, reqs, q[l].data_ptr(), kn[l].data_ptr(), vn[l].data_ptr(),
                                outs[k, l].data_ptr(), lses[k, l].data_ptr(), s.stream)
@@ -254,12 +254,12 @@ def test_config2_benchmark_pattern_300_overlapping_steps_bit_identical():
     sample = reqs[::7]
     pos = torch.tensor(sample, device=s.dev)
     # The run's very first launch has nothing to chain to and may be served by the other kernel, so
-    # round 0 is checked on its own and round 1 is the one the rest must equal.
+    # pass 0 is checked on its own and pass 1 is the one the rest must equal.
     for l in range(L):
         ref, ref_lse = checker_out(w, l, sample, [s.lens[r] for r in sample], q[l][pos])
         for k in (0, 1):
-            assert_close(outs[k, l][pos], ref, w.dtype, f"config2 copy {l} round {k}")
+            assert_close(outs[k, l][pos], ref, w.dtype, f"config2 copy {l} pass {k}")
             assert np.abs(lses[k, l][pos].double().cpu().numpy() - ref_lse).max() <= 2e-2
     differ = (outs[1:].view(torch.int16) != outs[1].view(torch.int16)).flatten(1).any(dim=1)
-    assert not bool(differ.any()), ("rounds that differ from round 1", differ.nonzero().flatten().tolist()[:10])
+    assert not bool(differ.any()), ("passes that differ from pass 1", differ.nonzero().flatten().tolist()[:10])
     assert bool((lses[1:] == lses[1]).all())
