@@ -196,7 +196,7 @@ def test_config2_in_the_benchmarks_own_launch_configuration(decode_kernel):
     sd.admit_and_fill()
     q, kn, vn, out = sd.make_inputs()
     t = odma.Tables()
-    for i in range(2 * copies):                    # every copy twice: second round reuses the plan
+    for i in range(2 * copies):                    # every copy twice: the second pass reuses the plan
         sd.step(i, q, kn, vn, out, t)
     torch.cuda.synchronize()
     assert sd.pool.check_status(sd.stream) == odma.OK
@@ -241,7 +241,7 @@ def test_config2_benchmark_pattern_300_overlapping_steps_bit_identical():
     vn = torch.stack([torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r], s.lens[r] + 1) for r in reqs]) for l in range(L)]).contiguous()
     passes = 100
     outs = torch.full((passes, L) + tuple(q.shape[1:]), float("nan"), dtype=q.dtype, device=s.dev)
-    lses = torch.full((rounds, L, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev)
+    lses = torch.full((passes, L, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev)
     torch.cuda.synchronize()
     for k in range(passes):                      # no synchronisation inside this loop
         for l in range(L):
