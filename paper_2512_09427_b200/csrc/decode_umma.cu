@@ -325,10 +325,10 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // stream drains, and so may the producer's first loads of rows nobody can be writing; the
     // rest comes after the dependency wait.  The next kernel is let go only after this wait (by
     // warp 7, which does nothing else), so a kernel can overlap with its immediate predecessor
-    // only.  A chained launch (layer l > 0 of a step over several layers) follows this kernel on
-    // layer l - 1: other K/V arrays, other outputs, the other scratch set, inputs that were
-    // complete when the step was issued; none of its roles waits, and its CTAs do real work on
-    // every SM the previous layer's CTAs have left.  (Warp 7 still waits before letting the next
+    // only.  A chained launch follows a decode launch of the same pool on ANOTHER layer (the next
+    // layer of a step, or a step on another layer): other K/V arrays, other outputs, the other
+    // scratch set, inputs that were complete when it was issued; none of its roles waits, and its
+    // CTAs do real work on every SM the predecessor's CTAs have left.  (Warp 7 still waits before letting the next
     // launch go: the kernel two launches back, which used the same scratch set, is complete
     // before any CTA of this one starts.)
     const bool chained = p.chained != 0;

@@ -42,9 +42,9 @@ struct DecodeParams {
     int32_t early_ok;           // the previous kernel of the stream that wrote this pool was a decode kernel (it
                                 // appends one row per stream): rows up to two before a stream's end may be
                                 // requested before the dependency wait; 0: nothing is read before it
-    int32_t chained;            // tcgen05 kernel: the previous kernel of the stream is this kernel on the
-                                // previous layer of the same step (same plan, other K/V arrays, other
-                                // outputs, the other scratch set): nothing of this launch waits for it
+    int32_t chained;            // tcgen05 kernel: the previous kernel of the stream is a decode launch of this
+                                // pool on another layer (other K/V arrays, other outputs, the other
+                                // scratch set): nothing of this launch waits for it
     int32_t kv_fp8;             // the pool holds E4M3 codes (one byte per element); q, the new rows and out are bf16
     float k_scale, v_scale;     // 8-bit pool: a stored code stands for value * scale (this layer's scales)
     float k_inv, v_inv;         // fp32 reciprocals: what an appended element is multiplied by before rounding
