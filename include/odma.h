@@ -78,6 +78,7 @@ enum { ODMA_DTYPE_F32 = 0, ODMA_DTYPE_BF16 = 1, ODMA_DTYPE_FP8_E4M3 = 2 };
 
 /* which tensor-core decode kernel a bf16 pool runs (odma_config.decode_kernel) */
 enum { ODMA_DECODE_AUTO = 0, ODMA_DECODE_TCGEN05 = 1, ODMA_DECODE_MMA_SYNC = 2 };
+enum { ODMA_READOUT_AUTO = 0, ODMA_READOUT_LATE = 1, ODMA_READOUT_AT_ONCE = 2 };
 
 /* kernels that odma_profile_read can report */
 enum { ODMA_K_APPEND = 0, ODMA_K_DECODE = 1, ODMA_K_COMBINE = 2, ODMA_K_MIGRATE = 3,
@@ -134,6 +135,12 @@ typedef struct odma_config {
                                 (every replica then feeds the same merged sequence and derives the
                                 same boundaries: the bucket configuration a cluster manager keeps
                                 consistent, Section III-E); 0: it enters the window at once (0) */
+    int32_t readout;         /* tcgen05 kernel, 16-bit slabs: ODMA_READOUT_LATE an item's result is read out
+                                of tensor memory and stored after the softmax of the first tile of the next
+                                item of the same half of the CTA (same results; faster where a CTA works
+                                through many short items, slower on few long ones), ODMA_READOUT_AT_ONCE as
+                                soon as the item ends, ODMA_READOUT_AUTO late for launches in which a CTA
+                                walks three items or more of at most 128 tokens on average (0) */
 } odma_config;
 
 typedef struct odma_slab {

@@ -129,6 +129,7 @@ int32_t Allocator::init(uint64_t bytes, int32_t layers, int32_t kv_heads, int32_
     outbox_.clear();
     if (cfg.async_recal < 0 || cfg.async_recal > 1 || cfg.cluster_observe < 0 || cfg.cluster_observe > 1)
         return ODMA_ERR_INVALID;
+    if (cfg.readout < ODMA_READOUT_AUTO || cfg.readout > ODMA_READOUT_AT_ONCE) return ODMA_ERR_INVALID;
     if (cfg.async_recal) {
         async_.reset(new Async());
         async_->th = std::thread([this] { worker(); });

@@ -391,6 +391,7 @@ void odma_config_default(odma_config* cfg) {
     cfg->span_layers = 1;
     cfg->async_recal = 0;
     cfg->cluster_observe = 0;
+    cfg->readout = ODMA_READOUT_AUTO;
 }
 
 const char* odma_strerror(int32_t code) {
@@ -736,10 +737,26 @@ bool uses_umma(const odma_pool* pool, int32_t group, bool chains) {
     return want == ODMA_DECODE_TCGEN05 || chains;
 }
 
+// The tcgen05 kernel has a variant that reads an item's result out of tensor memory one step late,
+// under the softmax of the lane's next item.  It pays where a CTA works through many short items
+// per launch (measured on 1,024 streams of one or two tiles, all layers in one launch: 12.2 -> 11.2
+// us per layer) and costs on longer ones (512 streams of ~300 tokens: 15.9 -> 16.4 us; 276 pieces
+// of ~500 tokens: 14.0 -> 15.3 us), so a launch picks by the plan's counts unless the
+// configuration says which.
+constexpr int64_t kLateItemsPerCta = 3;      // items a CTA walks in the launch, at least
+constexpr int64_t kLateTokensPerItem = 128;  // tokens per item on average, at most
+
 cudaError_t launch_tensor_decode(const odma_pool* pool, const TensorMaps& maps, const DecodeParams& p, int mode,
-                                 int n_ctas, cudaStream_t stream, const InlineLens* lens, bool umma,
+                                 const odma_tables* t, cudaStream_t stream, const InlineLens* lens, bool umma,
                                  const SpanParams* span = nullptr) {
-    return umma ? launch_decode_umma(maps, p, mode, n_ctas, stream, lens, span)
+    const int n_ctas = t->n_ctas;
+    const int32_t want = pool->alloc.config().readout;
+    bool defer = want == ODMA_READOUT_LATE;
+    if (want == ODMA_READOUT_AUTO)
+        defer = static_cast<int64_t>(p.n_layers) * t->n_items >= kLateItemsPerCta * n_ctas &&
+                t->kv_tokens * pool->kv_heads <= kLateTokensPerItem * t->n_items;
+    defer = defer && mode == kModeSlab && !p.kv_fp8;
+    return umma ? launch_decode_umma(maps, p, mode, n_ctas, stream, lens, span, defer)
                 : launch_decode_tc(maps, p, mode, n_ctas, stream, lens);
 }
 
@@ -811,7 +828,7 @@ int32_t decode_attention_impl(odma_pool* pool, int32_t layer, const void* q, int
             pool->last_lo = layer;
             pool->last_hi = layer + span;
             pool->last_stream = stream;
-            e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables->n_ctas, as_stream(stream), lens, umma,
+            e = launch_tensor_decode(pool, pool->maps, p, kModeSlab, tables, as_stream(stream), lens, umma,
                                      span > 1 ? &sp : nullptr);
         } else if (generic_supported(pool->head_dim)) {
             pool->last_fused_tensor = false;
@@ -1177,7 +1194,7 @@ int32_t odma_decode_attention_paged(odma_paged* paged, int32_t layer, const void
     cudaError_t e;
     {
         ProfScope ps(pool, ODMA_K_DECODE, as_stream(stream));
-        e = launch_tensor_decode(pool, paged->maps, p, kModePaged, tables->n_ctas, as_stream(stream), nullptr,
+        e = launch_tensor_decode(pool, paged->maps, p, kModePaged, tables, as_stream(stream), nullptr,
                                  uses_umma(pool, p.group, false));
     }
     if (e != cudaSuccess) return ODMA_ERR_CUDA;

@@ -231,12 +231,13 @@ __device__ __forceinline__ Item item_of(const int4& a, const int4& b, const Inli
     return it;
 }
 
-template <int D, int NT, int MODE, bool F8>
+template <int D, int NT, int MODE, bool F8, bool DEFER>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                    const __grid_constant__ InlineLens lens, const __grid_constant__ SpanParams sp) {
     using Cfg = UmmaConfig<D, NT, F8>;
     static_assert(!F8 || (D == 128 && NT == 1 && MODE == kModeSlab), "8-bit slabs: head_dim 128, group <= 8, slab mode");
+    static_assert(!DEFER || (!F8 && MODE == kModeSlab), "late read-out: 16-bit slabs");
     constexpr int ES = Cfg::kElem;
     constexpr int HALVES = Cfg::kHalves;
     constexpr int HALF_BYTES = kTile * 128;           // one 128-byte column block of a K or V tile
@@ -676,237 +677,20 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         uint32_t n_helped = 0, n_merged = 0;                // items this lane helped with / merged the other lane's part of
         float* x_mine = xchg + L * 32;                      // where this lane leaves (m, l) per head as a helper
         const float* x_other = xchg + (L ^ 1) * 32;
-        fetch(it_begin);
-        for (int x = 0; x < total && ok; ++x, advance()) {
-            const int k = x;
-            const Item im = item_of(nxt_a, nxt_b, lens, fused);
-            fetch(next_item());
-            const uint32_t g0 = g;
-            g += static_cast<uint32_t>(im.tiles);
-            // this layer's outputs and scratch
-            __nv_bfloat16* out_l = out + (span ? li * (sp.out_stride / 2) : 0);
-            float* lse_l = p.lse ? p.lse + (span ? li * sp.lse_stride : 0) : nullptr;
-            float* part_o_l = p.part_o + (span ? li * sp.part_o_stride : 0);
-            float* part_ml_l = p.part_ml + (span ? li * sp.part_ml_stride : 0);
-            uint32_t* counters_l = p.counters ? p.counters + (span ? static_cast<size_t>(li) * sp.counter_stride : 0) : nullptr;
-            // BOTH: an item of kBothTiles tiles or more is worked on by both lanes, its tiles going to
-            // them in turn from its home lane (item number mod 2).  The other lane is the helper: it
-            // leaves its accumulator in tensor memory and its (m, l) in shared memory, and the home
-            // lane merges the two parts and finishes the item.  Every item's query slot is visited by
-            // both softmax warps (each sees every phase of the slot's barriers, and a helper takes the
-            // heads' score factors from it).
-            const bool both = BOTH && im.tiles >= kBothTiles, home = (k & 1) == L;
-            if (!BOTH && !home) continue;
-            const int t_first = both ? (L ^ k) & 1 : 0, t_step = both ? 2 : 1;
-            const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
-            if (!ok) break;
-            if (!both && !home) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
-                continue;
-            }
-            // The token appended this step: its scaled score per head from the query rows and the
-            // new K row in shared memory (each thread adds up the elements it will also hold of the
-            // output, the quad completes the sum); its value row, packed, for when the item ends.
-            float s_new[NT];
-            uint32_t v_new[D / 8];
-#pragma unroll
-            for (int rs = 0; rs < NT; ++rs) s_new[rs] = -INFINITY;
-            float qfac = scale;                            // F8: the head's score factor (query power of two, key scale)
-            if (F8) qfac = reinterpret_cast<const float*>(newbuf + slot * Cfg::kNewBytes + 2 * D)[hq];
-            if (im.has_new && home && F8) {
-                // queries as hi + lo / 16 from rows hq and hq + 8 of the slot, the new rows as codes
-                const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes + hq * 128;
-                const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
-                float dot = 0.f;
-#pragma unroll
-                for (int i = 0; i < D / 8; ++i) {
-                    const float2 kk = unpack_e4m3(*reinterpret_cast<const uint16_t*>(nk + 8 * i + kq));
-                    v_new[i] = *reinterpret_cast<const uint16_t*>(nk + D + 8 * i + kq);
-                    const int off = (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
-                    const float2 qh = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + off));
-                    const float2 ql = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + 1024 + off));
-                    dot = fmaf(fmaf(ql.x, 0.0625f, qh.x), kk.x, dot);
-                    dot = fmaf(fmaf(ql.y, 0.0625f, qh.y), kk.y, dot);
-                }
-                dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 1);
-                dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 2);
-                s_new[0] = dot * qfac;
-            } else if (im.has_new && home) {
-                const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes;
-                const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
-                const uint8_t* nvp = nk + D * 2;
-                float dot[NT];
-#pragma unroll
-                for (int rs = 0; rs < NT; ++rs) dot[rs] = 0.f;
-#pragma unroll
-                for (int i = 0; i < D / 8; ++i) {
-                    const uint32_t kk = *reinterpret_cast<const uint32_t*>(nk + (8 * i + kq) * 2);
-                    v_new[i] = *reinterpret_cast<const uint32_t*>(nvp + (8 * i + kq) * 2);
-#pragma unroll
-                    for (int rs = 0; rs < NT; ++rs) {
-                        const uint32_t qq = *reinterpret_cast<const uint32_t*>(
-                            qs + (i >> 3) * Cfg::kQHalfBytes + rs * 1024 + hq * 128 + (((i & 7) ^ hq) << 4) + kq * 2);
-                        dot[rs] = fmaf(__uint_as_float(qq << 16), __uint_as_float(kk << 16), dot[rs]);
-                        dot[rs] = fmaf(__uint_as_float(qq & 0xFFFF0000u), __uint_as_float(kk & 0xFFFF0000u), dot[rs]);
-                    }
-                }
-#pragma unroll
-                for (int rs = 0; rs < NT; ++rs) {
-                    dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 1);
-                    dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 2);
-                    s_new[rs] = dot[rs] * scale;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
 
-            float m_ref[NT], l_acc[NT];
-#pragma unroll
-            for (int rs = 0; rs < NT; ++rs) {
-                m_ref[rs] = s_new[rs];
-                l_acc[rs] = 0.f;
-            }
-            for (int t = t_first; t < im.tiles; t += t_step) {
-                const uint32_t b = c & 1u, u = c >> 1;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t r[32];
-                tmem_ld_x8(t_s + b * 64u, r);
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(lane_bar(L, S_EMPTY + b));
-                const int valid = min(kTile, im.n_slab - t * kTile);
-                // scaled scores, keys at or beyond the item's end selected to -inf; tile maximum per head
-                float sc[NT][16], mx[NT];
-#pragma unroll
-                for (int rs = 0; rs < NT; ++rs) {
-                    mx[rs] = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            float s = F8 ? fmaf(__uint_as_float(r[4 * i + 2 + e]), 0.0625f, __uint_as_float(r[4 * i + e])) * qfac
-                                         : __uint_as_float(r[4 * i + 2 * rs + e]) * scale;
-                            if (8 * i + kq + e >= valid) s = -INFINITY;
-                            sc[rs][2 * i + e] = s;
-                            mx[rs] = fmaxf(mx[rs], s);
-                        }
-                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 1));
-                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 2));
-                }
-                if (t == t_first) {
-#pragma unroll
-                    for (int rs = 0; rs < NT; ++rs) m_ref[rs] = fmaxf(m_ref[rs], mx[rs]);
-                } else {
-                    bool grow = false;
-#pragma unroll
-                    for (int rs = 0; rs < NT; ++rs) grow = grow || mx[rs] > m_ref[rs] + RESCALE_ABOVE;
-                    if (__any_sync(0xFFFFFFFFu, grow)) {
-                        // Rare: raise the reference of the heads that need it and rescale their
-                        // rows of the accumulator.  Every second product issued so far must be
-                        // complete (the previous tile's releases its P buffer when it is); none
-                        // can be issued before this tile's P is handed over.
-                        const uint32_t pc = c - 1u;
-                        ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + (pc & 1u)), (pc >> 1) & 1u, abort_flag,
-                                                              p.status, limit));
-                        if (!ok) break;
-                        tc_fence_after();
-                        float f[2] = {1.f, 1.f};
-#pragma unroll
-                        for (int rs = 0; rs < NT; ++rs) {
-                            const float mn = mx[rs] > m_ref[rs] + RESCALE_ABOVE ? mx[rs] : m_ref[rs];
-                            f[rs] = fast_exp2(m_ref[rs] - mn);
-                            l_acc[rs] *= f[rs];
-                            m_ref[rs] = mn;
-                        }
-                        if (F8) f[1] = f[0];             // rows h and h + 8 are the two terms of one head
-#pragma unroll
-                        for (int blk = 0; blk < D / 32; ++blk) {
-                            uint32_t o[16];
-                            tmem_ld_x4(t_o + blk * 32u, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * f[0]);
-                                o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * f[0]);
-                                o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * f[1]);
-                                o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * f[1]);
-                            }
-                            tmem_st_x4(t_o + blk * 32u, o);
-                        }
-                        tmem_wait_st();
-                        tc_fence_before();
-                    }
-                }
-                // P = 2^(s - m) as bf16, 64 keys per head row, in the K-major swizzled layout; the row sums stay fp32
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit));
-                if (!ok) break;
-                uint8_t* pb = p_lane + b * Cfg::kPBufBytes;
-#pragma unroll
-                for (int rs = 0; rs < NT; ++rs) {
-                    float sum = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float p0 = fast_exp2(sc[rs][2 * i] - m_ref[rs]), p1 = fast_exp2(sc[rs][2 * i + 1] - m_ref[rs]);
-                        sum += p0 + p1;
-                        if (F8) {
-                            // 16 P = hi + lo / 16: hi to row hq, lo to row hq + 8; keys 8i + kq, + 1 are bytes of the row
-                            const float y0 = p0 * 16.f, y1 = p1 * 16.f;
-                            const uint32_t hi = pack_e4m3(y0, y1);
-                            const float2 h = unpack_e4m3(hi);
-                            const uint32_t lo = pack_e4m3((y0 - h.x) * 16.f, (y1 - h.y) * 16.f);
-                            uint8_t* dst = pb + hq * 128 + (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
-                            *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(hi);
-                            *reinterpret_cast<uint16_t*>(dst + 1024) = static_cast<uint16_t>(lo);
-                        } else {
-                            *reinterpret_cast<uint32_t*>(pb + rs * 1024 + hq * 128 + ((i ^ hq) << 4) + kq * 2) = pack_bf16(p0, p1);
-                        }
-                    }
-                    l_acc[rs] += sum;
-                }
-                if (valid & (PV_KEYS - 1)) {
-                    // the second product takes whole groups of 16 (8-bit slabs: 32) keys: value rows between
-                    // the item's end and the end of its last group are zeroed (P is zero there; the rows hold
-                    // whatever the slab or the stage did, which may not be a finite number)
-                    uint8_t* vt = kv + ((g0 + static_cast<uint32_t>(t)) % STAGES) * Cfg::kStageBytes + Cfg::kKvTileBytes;
-                    const int zero_rows = PV_KEYS - (valid & (PV_KEYS - 1));
-                    for (int idx = lane; idx < zero_rows * KV_CHUNKS; idx += 32) {
-                        const int zr = valid + idx / KV_CHUNKS, cc = idx % KV_CHUNKS;
-                        *reinterpret_cast<uint4*>(vt + (cc >> 3) * HALF_BYTES + zr * 128 + (((cc & 7) ^ (zr & 7)) << 4)) =
-                            make_uint4(0u, 0u, 0u, 0u);
-                    }
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(lane_bar(L, P_FULL + b));
-                ++c;
-            }
-            if (!ok) break;
-            if (BOTH && !home) {
-                // helper: once its accumulator is complete, (m, l) per head goes to shared memory;
-                // the home lane reads the accumulator itself and signs it off
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
-                if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, X_EMPTY), (n_helped & 1u) ^ 1u, abort_flag, p.status, limit));
-                if (!ok) break;
-                ++j;
-                ++n_helped;
-                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 1);
-                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 2);
-                if ((lane & 3) == 0) *reinterpret_cast<float2*>(x_mine + hq * 2) = make_float2(m_ref[0], l_acc[0]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(lane_bar(L, X_FULL));
-                continue;
-            }
-
-            // ---- the item's result: O from tensor memory, then out / partial / merge
+        // ---- an item's result: O from tensor memory, then out / partial / merge.  `fli` is the layer
+        // the item belongs to (its outputs and scratch), `both` whether the other lane helped with it.
+        auto finish = [&](const Item& im, int fli, bool both, float (&m_ref)[NT], float (&l_acc)[NT],
+                          const float (&s_new)[NT], const uint32_t (&v_new)[D / 8]) {
+            __nv_bfloat16* out_l = out + (span ? fli * (sp.out_stride / 2) : 0);
+            float* lse_l = p.lse ? p.lse + (span ? fli * sp.lse_stride : 0) : nullptr;
+            float* part_o_l = p.part_o + (span ? fli * sp.part_o_stride : 0);
+            float* part_ml_l = p.part_ml + (span ? fli * sp.part_ml_stride : 0);
+            uint32_t* counters_l = p.counters ? p.counters + (span ? static_cast<size_t>(fli) * sp.counter_stride : 0) : nullptr;
             float oo[NT][D / 4];                          // [rs][2i + e]: head hq + 8 rs, element 8i + kq + e
             if (im.tiles > 0) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
-                if (!ok) break;
+                if (!ok) return;
                 tc_fence_after();
 #pragma unroll
                 for (int blk = 0; blk < D / 64; ++blk) {
@@ -947,7 +731,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 // columns of tensor memory; both are signed off on its behalf
                 const int LO = L ^ 1;
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(LO, X_FULL), n_merged & 1u, abort_flag, p.status, limit));
-                if (!ok) break;
+                if (!ok) return;
                 ++n_merged;
                 tc_fence_after();
                 const float2 ml = *reinterpret_cast<const float2*>(x_other + hq * 2);
@@ -992,7 +776,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 }
             }
             if (F8) {                                      // codes to values
-                const float v_scale = span ? sp.scales[li].y : p.v_scale;
+                const float v_scale = span ? sp.scales[fli].y : p.v_scale;
 #pragma unroll
                 for (int i = 0; i < D / 4; ++i) oo[0][i] *= v_scale;
             }
@@ -1010,7 +794,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
             if (im.direct) {
 #pragma unroll
                 for (int rs = 0; rs < NT; ++rs) write_out(im.req, im.head, rs, m_ref[rs], l_acc[rs], oo[rs]);
-                continue;
+                return;
             }
 #pragma unroll
             for (int rs = 0; rs < NT; ++rs) {
@@ -1022,7 +806,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 for (int i = 0; i < D / 8; ++i) *reinterpret_cast<float2*>(po + 8 * i) = make_float2(oo[rs][2 * i], oo[rs][2 * i + 1]);
                 if ((lane & 3) == 0) *reinterpret_cast<float2*>(part_ml_l + prow * 2) = make_float2(m_ref[rs], l_acc[rs]);
             }
-            if (counters_l == nullptr) continue;           // a combine kernel follows
+            if (counters_l == nullptr) return;             // a combine kernel follows
             // The CTA that delivers a split stream's last piece merges all of them, in slot
             // order (so the result does not depend on which CTA that is), reading them back
             // through L2 (its own included), the next piece's loads in flight while one is folded.
@@ -1036,7 +820,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if (is_last) counters_l[im.comb] = 0u;     // ready for the next launch
             }
             is_last = __shfl_sync(0xFFFFFFFFu, is_last, 0);
-            if (!is_last) continue;
+            if (!is_last) return;
             __threadfence();
 #pragma unroll
             for (int rs = 0; rs < NT; ++rs) {
@@ -1076,6 +860,279 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 }
                 write_out(cr.x, cr.y, rs, fm, fl, fa);
             }
+        };
+
+        // DEFER (launches in which a lane works through several short items): an item's result is
+        // taken from tensor memory one step late.  Once an item's last P is handed over, the warp
+        // goes on to the lane's NEXT item (its new token's score, the softmax of its first tile) and
+        // only then reads out and stores the earlier item, whose second products have run meanwhile.
+        // (Only the first tile: the next item's second products cannot start before the accumulator
+        // is read out.)  The loop takes one turn more than there are items, for the last result.
+        Item pd_im = {};
+        int pd_li = 0;
+        bool pd_valid = false;
+        float pd_m[NT], pd_l[NT], pd_s[NT];
+        uint32_t pd_v[D / 8];
+        fetch(it_begin);
+        for (int x = 0; x < total + (DEFER ? 1 : 0) && ok; ++x, advance()) {
+            const int k = x;
+            const bool have = x < total;
+            Item im = item_of(nxt_a, nxt_b, lens, fused);
+            if (have) {
+                fetch(next_item());
+            } else {
+                im.tiles = 0;
+                im.has_new = false;
+            }
+            const uint32_t g0 = g;
+            g += static_cast<uint32_t>(im.tiles);
+            // BOTH: an item of kBothTiles tiles or more is worked on by both lanes, its tiles going to
+            // them in turn from its home lane (item number mod 2).  The other lane is the helper: it
+            // leaves its accumulator in tensor memory and its (m, l) in shared memory, and the home
+            // lane merges the two parts and finishes the item.  Every item's query slot is visited by
+            // both softmax warps (each sees every phase of the slot's barriers, and a helper takes the
+            // heads' score factors from it).
+            const bool both = BOTH && im.tiles >= kBothTiles, home = (k & 1) == L;
+            if (!BOTH && !home && have) continue;
+            const int t_first = both ? (L ^ k) & 1 : 0, t_step = both ? 2 : 1;
+            const uint32_t slot = static_cast<uint32_t>(k) % kQSlots, use = static_cast<uint32_t>(k) / kQSlots;
+            float s_new[NT];
+            uint32_t v_new[D / 8];
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) s_new[rs] = -INFINITY;
+            float qfac = scale;                            // F8: the head's score factor (query power of two, key scale)
+            if (have) {
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(kBarQFull + slot), use & 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                if (!both && !home) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
+                    continue;
+                }
+                // The token appended this step: its scaled score per head from the query rows and the
+                // new K row in shared memory (each thread adds up the elements it will also hold of the
+                // output, the quad completes the sum); its value row, packed, for when the item ends.
+                if (F8) qfac = reinterpret_cast<const float*>(newbuf + slot * Cfg::kNewBytes + 2 * D)[hq];
+                if (im.has_new && home && F8) {
+                    // queries as hi + lo / 16 from rows hq and hq + 8 of the slot, the new rows as codes
+                    const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes + hq * 128;
+                    const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
+                    float dot = 0.f;
+#pragma unroll
+                    for (int i = 0; i < D / 8; ++i) {
+                        const float2 kk = unpack_e4m3(*reinterpret_cast<const uint16_t*>(nk + 8 * i + kq));
+                        v_new[i] = *reinterpret_cast<const uint16_t*>(nk + D + 8 * i + kq);
+                        const int off = (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
+                        const float2 qh = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + off));
+                        const float2 ql = unpack_e4m3(*reinterpret_cast<const uint16_t*>(qs + 1024 + off));
+                        dot = fmaf(fmaf(ql.x, 0.0625f, qh.x), kk.x, dot);
+                        dot = fmaf(fmaf(ql.y, 0.0625f, qh.y), kk.y, dot);
+                    }
+                    dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 1);
+                    dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 2);
+                    s_new[0] = dot * qfac;
+                } else if (im.has_new && home) {
+                    const uint8_t* qs = qbuf + slot * Cfg::kQSlotBytes;
+                    const uint8_t* nk = newbuf + slot * Cfg::kNewBytes;
+                    const uint8_t* nvp = nk + D * 2;
+                    float dot[NT];
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) dot[rs] = 0.f;
+#pragma unroll
+                    for (int i = 0; i < D / 8; ++i) {
+                        const uint32_t kk = *reinterpret_cast<const uint32_t*>(nk + (8 * i + kq) * 2);
+                        v_new[i] = *reinterpret_cast<const uint32_t*>(nvp + (8 * i + kq) * 2);
+#pragma unroll
+                        for (int rs = 0; rs < NT; ++rs) {
+                            const uint32_t qq = *reinterpret_cast<const uint32_t*>(
+                                qs + (i >> 3) * Cfg::kQHalfBytes + rs * 1024 + hq * 128 + (((i & 7) ^ hq) << 4) + kq * 2);
+                            dot[rs] = fmaf(__uint_as_float(qq << 16), __uint_as_float(kk << 16), dot[rs]);
+                            dot[rs] = fmaf(__uint_as_float(qq & 0xFFFF0000u), __uint_as_float(kk & 0xFFFF0000u), dot[rs]);
+                        }
+                    }
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) {
+                        dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 1);
+                        dot[rs] += __shfl_xor_sync(0xFFFFFFFFu, dot[rs], 2);
+                        s_new[rs] = dot[rs] * scale;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarQEmpty + slot));
+            }
+
+            float m_ref[NT], l_acc[NT];
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                m_ref[rs] = s_new[rs];
+                l_acc[rs] = 0.f;
+            }
+            // one tile of the item (`first`: the lane's first tile of it); false when a wait ran out
+            auto do_tile = [&](int t, bool first) -> bool {
+                const uint32_t b = c & 1u, u = c >> 1;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait_spin(lane_bar(L, S_FULL + b), u & 1u, abort_flag, p.status, limit));
+                if (!ok) return false;
+                tc_fence_after();
+                uint32_t r[32];
+                tmem_ld_x8(t_s + b * 64u, r);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, S_EMPTY + b));
+                const int valid = min(kTile, im.n_slab - t * kTile);
+                // scaled scores, keys at or beyond the item's end selected to -inf; tile maximum per head
+                float sc[NT][16], mx[NT];
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    mx[rs] = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float s = F8 ? fmaf(__uint_as_float(r[4 * i + 2 + e]), 0.0625f, __uint_as_float(r[4 * i + e])) * qfac
+                                         : __uint_as_float(r[4 * i + 2 * rs + e]) * scale;
+                            if (8 * i + kq + e >= valid) s = -INFINITY;
+                            sc[rs][2 * i + e] = s;
+                            mx[rs] = fmaxf(mx[rs], s);
+                        }
+                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 1));
+                    mx[rs] = fmaxf(mx[rs], __shfl_xor_sync(0xFFFFFFFFu, mx[rs], 2));
+                }
+                if (first) {
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) m_ref[rs] = fmaxf(m_ref[rs], mx[rs]);
+                } else {
+                    bool grow = false;
+#pragma unroll
+                    for (int rs = 0; rs < NT; ++rs) grow = grow || mx[rs] > m_ref[rs] + RESCALE_ABOVE;
+                    if (__any_sync(0xFFFFFFFFu, grow)) {
+                        // Rare: raise the reference of the heads that need it and rescale their
+                        // rows of the accumulator.  Every second product issued so far must be
+                        // complete (the previous tile's releases its P buffer when it is); none
+                        // can be issued before this tile's P is handed over.
+                        const uint32_t pc = c - 1u;
+                        ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + (pc & 1u)), (pc >> 1) & 1u, abort_flag,
+                                                              p.status, limit));
+                        if (!ok) return false;
+                        tc_fence_after();
+                        float f[2] = {1.f, 1.f};
+#pragma unroll
+                        for (int rs = 0; rs < NT; ++rs) {
+                            const float mn = mx[rs] > m_ref[rs] + RESCALE_ABOVE ? mx[rs] : m_ref[rs];
+                            f[rs] = fast_exp2(m_ref[rs] - mn);
+                            l_acc[rs] *= f[rs];
+                            m_ref[rs] = mn;
+                        }
+                        if (F8) f[1] = f[0];             // rows h and h + 8 are the two terms of one head
+#pragma unroll
+                        for (int blk = 0; blk < D / 32; ++blk) {
+                            uint32_t o[16];
+                            tmem_ld_x4(t_o + blk * 32u, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                o[4 * i] = __float_as_uint(__uint_as_float(o[4 * i]) * f[0]);
+                                o[4 * i + 1] = __float_as_uint(__uint_as_float(o[4 * i + 1]) * f[0]);
+                                o[4 * i + 2] = __float_as_uint(__uint_as_float(o[4 * i + 2]) * f[1]);
+                                o[4 * i + 3] = __float_as_uint(__uint_as_float(o[4 * i + 3]) * f[1]);
+                            }
+                            tmem_st_x4(t_o + blk * 32u, o);
+                        }
+                        tmem_wait_st();
+                        tc_fence_before();
+                    }
+                }
+                // P = 2^(s - m) as bf16, 64 keys per head row, in the K-major swizzled layout; the row sums stay fp32
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, P_EMPTY + b), (u & 1u) ^ 1u, abort_flag, p.status, limit));
+                if (!ok) return false;
+                uint8_t* pb = p_lane + b * Cfg::kPBufBytes;
+#pragma unroll
+                for (int rs = 0; rs < NT; ++rs) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float p0 = fast_exp2(sc[rs][2 * i] - m_ref[rs]), p1 = fast_exp2(sc[rs][2 * i + 1] - m_ref[rs]);
+                        sum += p0 + p1;
+                        if (F8) {
+                            // 16 P = hi + lo / 16: hi to row hq, lo to row hq + 8; keys 8i + kq, + 1 are bytes of the row
+                            const float y0 = p0 * 16.f, y1 = p1 * 16.f;
+                            const uint32_t hi = pack_e4m3(y0, y1);
+                            const float2 h = unpack_e4m3(hi);
+                            const uint32_t lo = pack_e4m3((y0 - h.x) * 16.f, (y1 - h.y) * 16.f);
+                            uint8_t* dst = pb + hq * 128 + (((i >> 1) ^ hq) << 4) + (i & 1) * 8 + kq;
+                            *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(hi);
+                            *reinterpret_cast<uint16_t*>(dst + 1024) = static_cast<uint16_t>(lo);
+                        } else {
+                            *reinterpret_cast<uint32_t*>(pb + rs * 1024 + hq * 128 + ((i ^ hq) << 4) + kq * 2) = pack_bf16(p0, p1);
+                        }
+                    }
+                    l_acc[rs] += sum;
+                }
+                if (valid & (PV_KEYS - 1)) {
+                    // the second product takes whole groups of 16 (8-bit slabs: 32) keys: value rows between
+                    // the item's end and the end of its last group are zeroed (P is zero there; the rows hold
+                    // whatever the slab or the stage did, which may not be a finite number)
+                    uint8_t* vt = kv + ((g0 + static_cast<uint32_t>(t)) % STAGES) * Cfg::kStageBytes + Cfg::kKvTileBytes;
+                    const int zero_rows = PV_KEYS - (valid & (PV_KEYS - 1));
+                    for (int idx = lane; idx < zero_rows * KV_CHUNKS; idx += 32) {
+                        const int zr = valid + idx / KV_CHUNKS, cc = idx % KV_CHUNKS;
+                        *reinterpret_cast<uint4*>(vt + (cc >> 3) * HALF_BYTES + zr * 128 + (((cc & 7) ^ (zr & 7)) << 4)) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, P_FULL + b));
+                ++c;
+                return true;
+            };
+            int t = t_first;
+            if (DEFER && t < im.tiles) {
+                if (!do_tile(t, true)) break;
+                t += t_step;
+            }
+            if (DEFER && pd_valid) {
+                finish(pd_im, pd_li, false, pd_m, pd_l, pd_s, pd_v);
+                pd_valid = false;
+                if (!ok) break;
+            }
+            for (; t < im.tiles; t += t_step)
+                if (!do_tile(t, !DEFER && t == t_first)) break;
+            if (!ok || !have) break;
+            if (BOTH && !home) {
+                // helper: once its accumulator is complete, (m, l) per head goes to shared memory;
+                // the home lane reads the accumulator itself and signs it off
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, O_FULL), j & 1u, abort_flag, p.status, limit));
+                if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(lane_bar(L, X_EMPTY), (n_helped & 1u) ^ 1u, abort_flag, p.status, limit));
+                if (!ok) break;
+                ++j;
+                ++n_helped;
+                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 1);
+                l_acc[0] += __shfl_xor_sync(0xFFFFFFFFu, l_acc[0], 2);
+                if ((lane & 3) == 0) *reinterpret_cast<float2*>(x_mine + hq * 2) = make_float2(m_ref[0], l_acc[0]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(lane_bar(L, X_FULL));
+                continue;
+            }
+
+            if (!DEFER) {
+                finish(im, li, both, m_ref, l_acc, s_new, v_new);
+                if (!ok) break;
+                continue;
+            }
+            pd_im = im;
+            pd_li = li;
+            pd_valid = true;
+#pragma unroll
+            for (int rs = 0; rs < NT; ++rs) {
+                pd_m[rs] = m_ref[rs];
+                pd_l[rs] = l_acc[rs];
+                pd_s[rs] = s_new[rs];
+            }
+            if (im.has_new) {
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) pd_v[i] = v_new[i];
+            }
         }
     }
 
@@ -1104,12 +1161,12 @@ int umma_stages() {
     return std::min(n, Cfg::kStagesMax);
 }
 
-template <int D, int NT, int MODE, bool F8>
+template <int D, int NT, int MODE, bool F8, bool DEFER>
 cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas, cudaStream_t stream,
                              const InlineLens& lens, const SpanParams& sp) {
     using Cfg = UmmaConfig<D, NT, F8>;
     static bool configured[kMaxDevices] = {false};     // the opt-in to large shared memory is per device
-    auto kern = decode_umma_kernel<D, NT, MODE, F8>;
+    auto kern = decode_umma_kernel<D, NT, MODE, F8, DEFER>;
     p.stages = umma_stages<D, NT, F8>();
     if (p.stages < 2) return cudaErrorInvalidValue;
     const int smem = Cfg::smem_bytes(p.stages);
@@ -1137,10 +1194,12 @@ cudaError_t launch_umma_inst(const TensorMaps& maps, DecodeParams p, int n_ctas,
 
 template <int D, int NT>
 cudaError_t launch_umma_mode(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas, cudaStream_t s,
-                             const InlineLens& lens, const SpanParams& sp) {
+                             const InlineLens& lens, const SpanParams& sp, bool defer) {
     switch (mode) {
-        case kModeSlab: return launch_umma_inst<D, NT, kModeSlab, false>(maps, p, n_ctas, s, lens, sp);
-        case kModePaged: return launch_umma_inst<D, NT, kModePaged, false>(maps, p, n_ctas, s, lens, sp);
+        case kModeSlab:
+            return defer ? launch_umma_inst<D, NT, kModeSlab, false, true>(maps, p, n_ctas, s, lens, sp)
+                         : launch_umma_inst<D, NT, kModeSlab, false, false>(maps, p, n_ctas, s, lens, sp);
+        case kModePaged: return launch_umma_inst<D, NT, kModePaged, false, false>(maps, p, n_ctas, s, lens, sp);
     }
     return cudaErrorInvalidValue;
 }
@@ -1153,7 +1212,7 @@ bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8) {
 }
 
 cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                               cudaStream_t stream, const InlineLens* lens_in, const SpanParams* span_in) {
+                               cudaStream_t stream, const InlineLens* lens_in, const SpanParams* span_in, bool defer) {
     static const InlineLens no_lens{};                 // n = 0: lengths as planned
     static const SpanParams no_span{};                 // never read by a one-layer launch
     const InlineLens& lens = lens_in ? *lens_in : no_lens;
@@ -1161,15 +1220,15 @@ cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, in
     const SpanParams& sp = span_in ? *span_in : no_span;
     if (p.kv_fp8) {
         if (!umma_supported(p.head_dim, p.group, true) || mode != kModeSlab) return cudaErrorInvalidValue;
-        return launch_umma_inst<128, 1, kModeSlab, true>(maps, p, n_ctas, stream, lens, sp);
+        return launch_umma_inst<128, 1, kModeSlab, true, false>(maps, p, n_ctas, stream, lens, sp);
     }
     const bool two = p.group > 8;
     if (p.head_dim == 128)
-        return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens, sp)
-                   : launch_umma_mode<128, 1>(maps, p, mode, n_ctas, stream, lens, sp);
+        return two ? launch_umma_mode<128, 2>(maps, p, mode, n_ctas, stream, lens, sp, defer)
+                   : launch_umma_mode<128, 1>(maps, p, mode, n_ctas, stream, lens, sp, defer);
     if (p.head_dim == 64)
-        return two ? launch_umma_mode<64, 2>(maps, p, mode, n_ctas, stream, lens, sp)
-                   : launch_umma_mode<64, 1>(maps, p, mode, n_ctas, stream, lens, sp);
+        return two ? launch_umma_mode<64, 2>(maps, p, mode, n_ctas, stream, lens, sp, defer)
+                   : launch_umma_mode<64, 1>(maps, p, mode, n_ctas, stream, lens, sp, defer);
     return cudaErrorInvalidValue;
 }
 

@@ -92,10 +92,12 @@ cudaError_t launch_decode_tc(const TensorMaps& maps, const DecodeParams& p, int 
                              cudaStream_t stream, const InlineLens* lens = nullptr);
 // The same decode step on the tcgen05 tensor cores (decode_umma.cu): slab and paged modes;
 // `stages` and `q_slots` of the parameter block are ignored (the kernel sizes its own rings).
-// An 8-bit (E4M3) pool: head_dim 128, group <= 8, slab mode.
+// An 8-bit (E4M3) pool: head_dim 128, group <= 8, slab mode.  `defer` (16-bit slabs, slab mode)
+// picks the variant that reads an item's result out under the softmax of the lane's next item.
 bool umma_supported(int32_t head_dim, int32_t group, bool kv_fp8);
 cudaError_t launch_decode_umma(const TensorMaps& maps, const DecodeParams& p, int mode, int n_ctas,
-                               cudaStream_t stream, const InlineLens* lens = nullptr, const SpanParams* span = nullptr);
+                               cudaStream_t stream, const InlineLens* lens = nullptr, const SpanParams* span = nullptr,
+                               bool defer = false);
 cudaError_t launch_decode_generic(const DecodeParams& p, int dtype, int n_ctas, cudaStream_t stream);
 bool generic_supported(int32_t head_dim);
 

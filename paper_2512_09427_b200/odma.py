@@ -23,6 +23,7 @@ MAX_BUCKETS = 8
 OK, ERR_INVALID, ERR_NOMEM, ERR_UNKNOWN_REQ, ERR_DUP_REQ, ERR_OVERFLOW, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(9)
 DTYPE_F32, DTYPE_BF16, DTYPE_FP8_E4M3 = 0, 1, 2
 DECODE_AUTO, DECODE_TCGEN05, DECODE_MMA_SYNC = 0, 1, 2
+READOUT_AUTO, READOUT_LATE, READOUT_AT_ONCE = 0, 1, 2
 K_APPEND, K_DECODE, K_COMBINE, K_MIGRATE, K_PROBE = range(5)
 
 
@@ -33,7 +34,7 @@ class Config(C.Structure):
                 ("gamma_permille", C.c_int32), ("tau_permille", C.c_int32), ("growth", C.c_int32),
                 ("large_fixed", C.c_int32), ("max_batch", C.c_int32), ("max_group", C.c_int32),
                 ("plan_ctas", C.c_int32), ("fused_combine", C.c_int32), ("fused_append", C.c_int32),
-                ("decode_kernel", C.c_int32), ("chain_launches", C.c_int32), ("span_layers", C.c_int32), ("async_recal", C.c_int32), ("cluster_observe", C.c_int32)]
+                ("decode_kernel", C.c_int32), ("chain_launches", C.c_int32), ("span_layers", C.c_int32), ("async_recal", C.c_int32), ("cluster_observe", C.c_int32), ("readout", C.c_int32)]
 
 
 class Slab(C.Structure):

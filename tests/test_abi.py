@@ -34,7 +34,7 @@ def test_defaults_are_the_papers_constants():
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(odma.Slab) == 24
     assert ctypes.sizeof(odma.Stats) == 16 * 8
-    assert ctypes.sizeof(odma.Config) == (6 + 8 + 1 + 14) * 4
+    assert ctypes.sizeof(odma.Config) == (6 + 8 + 1 + 15) * 4
     assert ctypes.sizeof(odma.Tables) == 8 + 16 * 4 + 8 + 8
 
 

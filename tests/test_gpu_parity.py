@@ -10,12 +10,13 @@ from paper_2512_09427_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(autouse=True, params=[1, 2], ids=["tcgen05", "mma_sync"])
+@pytest.fixture(autouse=True, params=[(1, 2), (1, 1), (2, 0)], ids=["tcgen05", "tcgen05_late_readout", "mma_sync"])
 def decode_kernel(request):
-    """Every test of this module runs once on each bf16 tensor-core decode kernel."""
+    """Every test of this module runs once on each bf16 tensor-core decode kernel, on the tcgen05
+    kernel with both orders of reading an item's result out."""
     import helpers
-    helpers.CFG_DEFAULTS["decode_kernel"] = request.param
-    yield request.param
+    helpers.CFG_DEFAULTS["decode_kernel"], helpers.CFG_DEFAULTS["readout"] = request.param
+    yield request.param[0]
     helpers.CFG_DEFAULTS.clear()
 
 RAGGED = [1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 500, 1000, 2771]
@@ -210,6 +211,62 @@ def test_fused_and_separate_combine_agree_bit_for_bit():
         assert s.last_tables.n_combine > 0
         outs.append(res[0])
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("span", [1, 0], ids=["one_launch", "launch_per_layer"])
+@pytest.mark.parametrize("ctas", [1, 3, 0])
+def test_late_and_immediate_readout_agree_bit_for_bit(ctas, span, decode_kernel):
+    """The tcgen05 kernel reads an item's result out at once or under the next item of the same half
+    of the CTA: the same arithmetic in another order of hand-overs, so every output bit, every
+    log-sum-exp and every appended row agree.  Many short items per CTA (up to 60 per half and
+    layer), items of no tile at all, split streams, three layers, two steps without a host sync."""
+    if decode_kernel != 1:
+        pytest.skip("tcgen05 kernel only")
+    odma = lib()
+    lens = [0, 1, 2, 15, 16, 17, 40, 63, 64, 65, 100, 127, 128, 129, 130, 200, 31, 33, 5, 7, 9, 11, 300, 2771, 70, 90, 3, 0, 64, 128]
+    w = qwen_small(lens, layers=3)
+    w = wl.scaled(w, predicted=w.context + 8)
+    got = []
+    for readout in (odma.READOUT_LATE, odma.READOUT_AT_ONCE):
+        s = Session(w, plan_ctas=ctas, span_layers=span, readout=readout)
+        s.pool.set_buckets(list(w.static_buckets)); s.ls.oracle.set_buckets(list(w.static_buckets))
+        reqs = list(range(w.batch))
+        s.admit(reqs, w.predicted)
+        pre = [r for r in reqs if w.context[r] > 0]
+        s.append(pre, [int(w.context[r]) for r in pre])
+        steps, NL = 2, w.layers
+        qs = [torch.stack([s.queries(l, reqs, w.q_heads, k) for l in range(NL)]).contiguous() for k in range(steps)]
+        kns = [torch.stack([torch.cat([s.rows(l, r, wl.KIND_K, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs])
+                            for l in range(NL)]).contiguous() for k in range(steps)]
+        vns = [torch.stack([torch.cat([s.rows(l, r, wl.KIND_V, s.lens[r] + k, s.lens[r] + k + 1) for r in reqs])
+                            for l in range(NL)]).contiguous() for k in range(steps)]
+        outs = [torch.full_like(qs[0], float("nan")) for _ in range(steps)]
+        lses = [torch.full((NL, len(reqs), w.q_heads), float("nan"), dtype=torch.float32, device=s.dev) for _ in range(steps)]
+        torch.cuda.synchronize()
+        t = odma.Tables()
+        for k in range(steps):
+            s.pool.decode_step(0, NL, w.q_heads, reqs, qs[k].data_ptr(), kns[k].data_ptr(), vns[k].data_ptr(),
+                               outs[k].data_ptr(), lses[k].data_ptr(), s.stream, t)
+            s.ls.commit(reqs, 1)
+        torch.cuda.synchronize()
+        assert s.pool.check_status(s.stream) == odma.OK
+        if ctas == 0:
+            assert t.n_combine > 0
+        if readout == odma.READOUT_LATE:                    # and the late order against the checker
+            for k in range(steps):
+                for l in range(NL):
+                    for i, r in enumerate(reqs):
+                        s.kv.append(r, l, kns[k][l, i:i + 1], vns[k][l, i:i + 1])
+                    ref, ref_lse, _ = s.oracle_out(l, reqs, qs[k][l], w.q_heads)
+                    assert_close(outs[k][l], ref, w.dtype, f"late step {k} layer {l}")
+                    assert np.abs(lses[k][l].double().cpu().numpy() - ref_lse).max() <= 2e-2
+        for r in reqs:
+            s.lens[r] += steps
+        rows = [s.pool_rows(l, kind, r).clone() for l in range(NL) for kind in (0, 1) for r in reqs]
+        got.append((outs, lses, rows))
+    (o1, l1, r1), (o2, l2, r2) = got
+    for a, b in zip(o1 + l1 + r1, o2 + l2 + r2):
+        assert torch.equal(a, b)
 
 
 def test_bf16_multi_layer_and_second_step():
