@@ -86,6 +86,11 @@ def test_async_thread_stops_with_the_pool_and_bad_flags_are_refused():
         host_pool(w, async_recal=2)
     with pytest.raises(odma.OdmaError):
         host_pool(w, cluster_observe=-1)
+    for bad in (-1, 3):                                 # the decode kernel's read-out order: auto, late, at once
+        with pytest.raises(odma.OdmaError):
+            host_pool(w, readout=bad)
+    for good in (odma.READOUT_AUTO, odma.READOUT_LATE, odma.READOUT_AT_ONCE):
+        host_pool(w, readout=good).destroy()
 
 
 def test_observe_and_drain_single_process():
