@@ -17,7 +17,8 @@
 // Two items are in flight per CTA ("lanes": items go to them in turn), each with its own
 // softmax warp, two S buffers and one O accumulator in tensor memory and two P buffers in
 // shared memory, so one item's hand-over runs under the other's streaming.  Warp roles:
-//     0, 4   softmax + finish of lane 0 / 1: S from tensor memory (one thread holds 16 keys of
+//     0, 4   (0, 5 in the late-read-out variant, whose second products of lane 0 are issued by warp 4)
+//            softmax + finish of lane 0 / 1: S from tensor memory (one thread holds 16 keys of
 //            one head), masking, running reference maximum, P = 2^(s - m) to shared memory; on
 //            an item's last tile the value rows between the item's end and the next multiple of
 //            16 are zeroed (the second product runs over whole groups of 16 keys); when the item
@@ -269,6 +270,17 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
     // 8-bit slabs: the softmax warp is the slowest role (a tile arrives in half the time), so an item of
     // kBothTiles tiles or more is worked on by both lanes, its tiles going to them in turn
     constexpr bool BOTH = F8;
+    // The late-read-out variant puts the two softmax warps on different schedulers (both lanes are at
+    // work most of the time there, and on one scheduler each slows the other down).  Tensor-memory
+    // lanes 0..31 belong to warps 0 and 4, lanes 32..63 to warps 1 and 5; an M = 64 accumulator keeps
+    // rows 16..31 in lanes 32..47.  So lane 1's A operands (queries, P) are described from 2 KB (16
+    // rows) before their first row: its heads are rows 16.. of its products, and warp 5 reads them.
+    // (Rows 0..15 are then whatever lies there; they are never looked at.)  Measured with the read-out
+    // at once, the same arrangement lost 3 % on long streams, and the 8-bit kernel needs both softmax
+    // warps on lanes 0..15 (a home lane reads the helper lane's accumulator): both keep warps 0 and 4.
+    constexpr bool SPLIT = DEFER;
+    constexpr int W_SOFT1 = SPLIT ? 5 : 4, W_PV0 = SPLIT ? 4 : 5, W_PV1 = 6;
+    constexpr uint32_t ROWS16 = 16u * 128u;            // bytes of 16 operand rows
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -585,6 +597,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 continue;
             }
             const uint32_t qb = q_u32 + slot * Cfg::kQSlotBytes;
+            const uint32_t qb1 = qb - ROWS16;            // lane 1 (SPLIT): the heads as rows 16..
             for (int t = 0; t < im.tiles; ++t, ++g) {
                 const uint32_t stage = g % STAGES, phase = (g / STAGES) & 1u;
                 const int L = (both ? k + t : k) & 1;
@@ -603,7 +616,7 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 if (elected) {
 #pragma unroll
                     for (int ks = 0; ks < QK_STEPS; ++ks)
-                        umma<F8>(t_s, smem_desc(qb + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
+                        umma<F8>(t_s, smem_desc((SPLIT && L ? qb1 : qb) + (ks >> 2) * Cfg::kQHalfBytes + (ks & 3) * 32, 16, 1024),
                                   smem_desc(kbase + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
                     umma_commit(lane_bar(L, S_FULL + b));
                     if (t == im.tiles - 1) umma_commit(bar(kBarQEmpty + slot));
@@ -616,12 +629,12 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         if (elected) umma_commit(bar(kBarDrain));
         __syncwarp();
         mbar_wait_slow(bar(kBarDrain), 0, nullptr, p.status, limit / 4 + 1);
-    } else if (warp == 5 || warp == 6) {
+    } else if (warp == W_PV0 || warp == W_PV1) {
         // ------------------------------------------------------------------ MMA issue, second products of one lane
         // A tile's P has been written (and, for an item's first tile, the lane's O of the item
         // before has been read out); the commits hand the stage back to the producer and the P
         // buffer to the softmax warp, and after an item's last tile tell it that O is complete.
-        const int L = warp - 5;
+        const int L = warp == W_PV0 ? 0 : 1;
         uint32_t elected;
         asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(elected));
         constexpr uint32_t IDESC_PV = F8 ? umma_idesc8(64, D, true) : umma_idesc(64, D, true);
@@ -648,7 +661,8 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
                 const bool last = t + t_step >= im.tiles;                      // the lane's last tile of the item
                 const int ksteps = (t == im.tiles - 1 ? im.n_slab - t * kTile + PV_KEYS - 1 : kTile) / PV_KEYS;
                 const uint32_t vbase = kv_u32 + st * Cfg::kStageBytes + Cfg::kKvTileBytes;
-                const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + static_cast<int>(b)) * Cfg::kPBufBytes);
+                const uint32_t pb = p_u32 + static_cast<uint32_t>((L * 2 + static_cast<int>(b)) * Cfg::kPBufBytes) -
+                                    (SPLIT && L ? ROWS16 : 0u);
                 if (elected) {
                     for (int ks = 0; ks < ksteps; ++ks)
                         umma<F8>(t_o, smem_desc(pb + ks * 32, 16, 1024), smem_desc(vbase + ks * (PV_KEYS * 128), HALF_BYTES, 1024), IDESC_PV,
@@ -664,10 +678,11 @@ decode_umma_kernel(const __grid_constant__ TensorMaps tm, const DecodeParams p,
         if (elected) umma_commit(bar(kBarDrain + 1 + L));
         __syncwarp();
         mbar_wait_slow(bar(kBarDrain + 1 + L), 0, nullptr, p.status, limit / 4 + 1);
-    } else if (warp == 0 || warp == 4) {
+    } else if (warp == 0 || warp == W_SOFT1) {
         // ------------------------------------------------------------------ softmax + finish
         const int L = warp == 0 ? 0 : 1;
-        const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols), t_o = t_s + 128u;
+        // (SPLIT: lane 1's rows are in tensor-memory lanes 32.., the lane field of the address is bits 16..)
+        const uint32_t t_s = tmem + static_cast<uint32_t>(L * kTmemLaneCols) + (SPLIT && L ? (32u << 16) : 0u), t_o = t_s + 128u;
         uint8_t* p_lane = pbuf + L * 2 * Cfg::kPBufBytes;
         const int hq = lane >> 2, kq = (lane & 3) * 2;      // head row within 8; first of the thread's two keys within 8
         const float scale = p.scale_log2;
