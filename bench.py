@@ -151,6 +151,9 @@ def config4_drift(rank: int = 0):
     return stats, halves
 
 
+READOUT = 0          # --readout: the tcgen05 kernel's read-out order (0 = the library picks per launch)
+
+
 class SlabDecode:
     """A device pool filled with the workload's KV, plus the step's input buffers."""
 
@@ -173,6 +176,7 @@ class SlabDecode:
         cfg.fused_combine = fused
         cfg.decode_kernel = decode_kernel
         cfg.chain_launches = chain_launches
+        cfg.readout = READOUT
         self.pool_cfg = cfg
         # `mem`: the device memory of another SlabDecode of the same workload (a second pool over the
         # same, already filled bytes: the allocator is deterministic, so the slabs coincide)
@@ -1013,6 +1017,8 @@ def main():
     ap.add_argument("--fused-combine", type=int, default=1, help="1: split streams merged inside the decode kernel")
     ap.add_argument("--decode-kernel", default="auto", choices=list(DECODE_KERNELS),
                     help="which bf16 decode kernel the pool runs (auto: the library's choice per shape)")
+    ap.add_argument("--readout", default="auto", choices=["auto", "late", "at_once"],
+                    help="tcgen05 kernel, 16-bit slabs: when an item's result is read out of tensor memory (auto: per launch, by the plan's counts)")
     ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "e4m3"],
                     help="element type of the slabs: bf16 (the configs as stated) or E4M3 codes with per-layer scales")
     ap.add_argument("--copies", type=int, default=0, help="config2: rotating KV copies (0 = enough for 3x L2)")
@@ -1020,6 +1026,8 @@ def main():
                     help="config3/config5: step through this many layers only (0 = all 28; a reduced size for profiler "
                          "captures, not the benchmark configuration)")
     args = ap.parse_args()
+    global READOUT
+    READOUT = {"auto": 0, "late": 1, "at_once": 2}[args.readout]
     if args.warmup < 3:
         args.warmup = 3
     if not args.phases:
